@@ -1,0 +1,210 @@
+/*
+ * moska.h -- C ABI of the MoSKA decode-attention hot path for NVIDIA B200 (sm_100a).
+ *
+ * MoSKA (Mixture of Shared KV Attention) splits the KV context of a batch of decoding requests
+ * into a large SHARED store, partitioned into chunks that many requests attend to, and a
+ * per-request UNIQUE KV.  One decode step of one attention layer is
+ *
+ *   route  ->  group_by_chunk  ->  { shared_attn  ||  unique_attn }  ->  merge
+ *
+ * (Section III-A "Shared KV Attention", Section III-B "The MoSKA Architecture", Fig. 2.)
+ *
+ * Conventions that hold for every entry point
+ * -------------------------------------------
+ *  * All tensor arguments are DEVICE pointers owned by the caller, unless a parameter is
+ *    documented as a host pointer.  The library never allocates, frees or keeps a pointer
+ *    after the call returns.  Scratch memory comes from a caller-provided workspace.
+ *  * Every call only enqueues work on `stream` and returns without synchronising.  Nothing
+ *    produced on the device is read back by the host.
+ *  * bf16 tensors are passed as `const uint16_t*` (raw bfloat16 bit patterns).
+ *  * Symbols: B requests, Hq query heads, Hkv KV heads, G = Hq / Hkv (1..8), D head dimension
+ *    (64 or 128), C shared chunks of L tokens each, k chunks routed per (request, KV head).
+ *    Query row r = b * Hq + hq; its KV head is h = hq / G.
+ *  * Partial results: every query row owns `n_slots = shared_slots + n_unique_splits` slots.
+ *        o_part   float [B][Hq][n_slots][D]   softmax-normalised partial output
+ *        lse_part float [B][Hq][n_slots]      natural-log sum of exp(scale * q.k) over the
+ *                                             tokens of that slot; -inf marks an empty slot
+ *    Shared attention writes slots [0, shared_slots), unique attention writes slots
+ *    [shared_slots, n_slots).  Both write EVERY slot of their range (empty ones as -inf, o = 0),
+ *    so the caller never has to clear the buffers.
+ *  * Return value: MOSKA_OK or a negative moska_status.  moska_last_error() gives a text for
+ *    the last failure on the calling thread.  Invalid arguments are detected on the host
+ *    before anything is launched.
+ */
+#ifndef MOSKA_H_
+#define MOSKA_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum moska_status {
+    MOSKA_OK              = 0,
+    MOSKA_ERR_INVALID_ARG = -1, /* null pointer, k > C, Hq % Hkv != 0, misaligned pointer ...   */
+    MOSKA_ERR_UNSUPPORTED = -2, /* D not in {64,128}, G > 8, L % 128 != 0, device is not sm_100 */
+    MOSKA_ERR_WORKSPACE   = -3, /* workspace missing or smaller than moska_workspace_bytes()    */
+    MOSKA_ERR_CUDA        = -4  /* a CUDA runtime call or kernel launch failed                  */
+} moska_status;
+
+/* Problem shape of one decode step of one layer. */
+typedef struct moska_shape {
+    int32_t B;               /* concurrent requests                                              */
+    int32_t Hq;              /* query heads                                                      */
+    int32_t Hkv;             /* KV heads, Hq % Hkv == 0, G = Hq / Hkv <= 8                       */
+    int32_t D;               /* head dimension: 64 or 128                                        */
+    int32_t C;               /* number of shared chunks                                          */
+    int32_t L;               /* tokens per shared chunk, a multiple of 128                       */
+    int32_t k;               /* chunks routed per (request, KV head), 1 <= k <= C                */
+    int32_t shared_slots;    /* partial slots written by shared attention: k in routed mode;     */
+                             /* in dense mode (no routing) the C chunks are cut into this many   */
+                             /* runs of ceil(C / shared_slots) consecutive chunks                */
+    int32_t n_unique_splits; /* partial slots written by unique attention (split-K), >= 1        */
+} moska_shape;
+
+typedef void* moska_stream; /* a cudaStream_t */
+
+/* Library version, major * 100 + minor. */
+int moska_version(void);
+
+/* Text of the last error raised on the calling thread ("" if none). Host pointer, never NULL. */
+const char* moska_last_error(void);
+
+/* n_slots = shared_slots + n_unique_splits; negative status if the shape is invalid. Host only. */
+int moska_partial_slots(const moska_shape* shape);
+
+/* Bytes of workspace that moska_route / moska_group_by_chunk / moska_shared_attn need for this
+ * shape (one workspace serves all three; 256-byte aligned base required).  Host only, pure.   */
+size_t moska_workspace_bytes(const moska_shape* shape);
+
+/* A reasonable n_unique_splits for a batch whose longest unique context has `max_len` tokens.
+ * Host only, pure.                                                                              */
+int moska_default_unique_splits(int32_t B, int32_t Hkv, int32_t max_len);
+
+/*
+ * Chunk embeddings used by the router (Section III-B: "precomputed chunk embeddings"; the
+ * embedding of a chunk is the arithmetic mean of its L keys, per KV head).  Offline step.
+ *   k_shared   bf16  [Hkv][C][L][D]   (16-byte aligned)
+ *   summaries  float [Hkv][C][D]      out
+ */
+int moska_build_chunk_summaries(const uint16_t* k_shared, float* summaries,
+                                const moska_shape* shape, moska_stream stream);
+
+/*
+ * Router (Section III-B): relevance of chunk c for (request b, KV head h) is the inner product
+ * of the pooled query  qbar[b][h] = sum_{g<G} q[b][h*G+g]  with summaries[h][c]; the k chunks
+ * with the largest score are selected, exact ties going to the lower chunk index.
+ *   q           bf16  [B][Hq][D]
+ *   summaries   float [Hkv][C][D]
+ *   topk_idx    int32 [B][Hkv][k]   out, chunk indices in ASCENDING order
+ *   topk_score  float [B][Hkv][k]   out, score of topk_idx[...] (same order); may be NULL
+ * One warp scores and selects for one (b, h).  No workspace.
+ */
+int moska_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
+                const moska_shape* shape, moska_stream stream);
+
+/*
+ * Query aggregation (Section III-A: the N concurrent queries that hit the same shared chunk are
+ * gathered into one query matrix).  Let p = (b*Hkv + h)*k + j be the flat position of the j-th
+ * routed chunk of (b, h) and key(p) = h*C + topk_idx[p].  This is a stable counting sort of the
+ * positions by key:
+ *   seg_offsets  int32 [Hkv*C + 1]  out, exclusive scan of the number of positions per key
+ *   seg_entries  int32 [B*Hkv*k]    out, positions p, key-major, ascending p inside one key
+ * The result is deterministic.  It also writes the tile work lists that moska_shared_attn
+ * consumes into `ws` (give both calls the same, unmodified workspace).
+ */
+int moska_group_by_chunk(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
+                         const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream);
+
+/*
+ * Shared KV Attention (Section III-A, Fig. 2a): for every non-empty segment (h, c) the query rows
+ * of all requests routed to chunk c form the rows of one Q matrix; S = scale * Q Kc^T, row-wise
+ * softmax statistics and O = softmax(S) Vc are computed as one batched tensor-core product, so
+ * the chunk's K/V tile leaves HBM once per step however many requests use it.
+ * For entry p = (b*Hkv+h)*k + j and each g < G it writes slot j of row (b, h*G+g).
+ *   q                      bf16 [B][Hq][D]
+ *   k_shared, v_shared     bf16 [Hkv][C][L][D]   (128-byte aligned)
+ *   topk_idx/seg_offsets/seg_entries   as produced by moska_route / moska_group_by_chunk,
+ *       or all three NULL for DENSE mode: no routing, every row attends every chunk; run s of
+ *       ceil(C/shared_slots) consecutive chunks goes to slot s (needs no prior grouping call).
+ *   o_part, lse_part       see "Partial results" above; slots [0, shared_slots) are written
+ *   softmax_scale          multiplies q.k before the softmax (usually 1/sqrt(D))
+ */
+int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
+                      const int32_t* topk_idx, const int32_t* seg_offsets,
+                      const int32_t* seg_entries, float* o_part, float* lse_part,
+                      float softmax_scale, const moska_shape* shape, void* ws, size_t ws_bytes,
+                      moska_stream stream);
+
+/*
+ * Unique KV Attention (Section III-A: per-request attention over private KV, a memory-bound
+ * GEMV-like pass).  Split-K over the request's tokens: each of the n_unique_splits slots holds
+ * the partial result over a disjoint token range (which range is an implementation detail);
+ * slots without tokens are written as lse = -inf, o = 0.
+ *   k_unique, v_unique  bf16 [T_total][Hkv][D]  token-major ragged store (16-byte aligned)
+ *   kv_start            int64 [B]  first token of request b in the store
+ *   kv_len              int32 [B]  number of tokens of request b (0 allowed)
+ */
+int moska_unique_attn(const uint16_t* q, const uint16_t* k_unique, const uint16_t* v_unique,
+                      const int64_t* kv_start, const int32_t* kv_len, float* o_part,
+                      float* lse_part, float softmax_scale, const moska_shape* shape,
+                      moska_stream stream);
+
+/*
+ * Combination of the shared and unique partial results.  The paper leaves this step implicit;
+ * the log-sum-exp merge is the only combination that equals softmax attention over the union of
+ * the tokens (Section III-A/III-B).  Per row: M = max_i lse_i, w_i = exp(lse_i - M),
+ * out = sum_i w_i o_i / sum_i w_i, lse = M + ln sum_i w_i.  Slots with lse = -inf contribute
+ * nothing; if every slot is -inf then out = 0 and lse = -inf (never NaN).
+ *   out      bf16  [B][Hq][D]        out
+ *   out_f32  float [B][Hq][D]        out, unrounded copy; may be NULL
+ *   lse_out  float [B][Hq]           out; may be NULL
+ */
+int moska_merge(const float* o_part, const float* lse_part, uint16_t* out, float* out_f32,
+                float* lse_out, const moska_shape* shape, moska_stream stream);
+
+/*
+ * Measured comparison, not part of the method: the unbatched form that Shared KV Attention
+ * replaces (Section I, Section III-A: one memory-bound GEMV pass per request over each routed
+ * chunk).  Same results as moska_shared_attn, same slots; reads every routed chunk once per
+ * (request, KV head) instead of once per step.  topk_idx == NULL selects dense mode.
+ */
+int moska_gemv_baseline(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
+                        const int32_t* topk_idx, float* o_part, float* lse_part,
+                        float softmax_scale, const moska_shape* shape, moska_stream stream);
+
+/*
+ * One whole decode step on device buffers: route -> group -> shared || unique -> merge, in that
+ * order on `stream` (shared and unique attention overlap on an internal second stream when
+ * `side_stream` is not NULL).  Dense mode (no routing) when summaries == NULL.
+ * Scratch buffers topk_idx [B*Hkv*k], seg_offsets [Hkv*C+1], seg_entries [B*Hkv*k], o_part,
+ * lse_part and ws are caller-owned as in the individual calls.
+ */
+int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t* k_shared,
+                      const uint16_t* v_shared, const uint16_t* k_unique,
+                      const uint16_t* v_unique, const int64_t* kv_start, const int32_t* kv_len,
+                      int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
+                      float* o_part, float* lse_part, uint16_t* out, float* lse_out,
+                      float softmax_scale, const moska_shape* shape, void* ws, size_t ws_bytes,
+                      moska_stream stream, moska_stream side_stream);
+
+/*
+ * moska_decode_step for a caller whose step inputs live in HOST memory: copies q_host (bf16
+ * [B][Hq][D], ideally pinned) into q_dev, runs the step, copies `out` back into out_host (bf16
+ * [B][Hq][D]) and waits for the stream.  The KV stores and all scratch stay on the device.
+ */
+int moska_decode_step_host(const uint16_t* q_host, uint16_t* q_dev, const float* summaries,
+                           const uint16_t* k_shared, const uint16_t* v_shared,
+                           const uint16_t* k_unique, const uint16_t* v_unique,
+                           const int64_t* kv_start, const int32_t* kv_len, int32_t* topk_idx,
+                           int32_t* seg_offsets, int32_t* seg_entries, float* o_part,
+                           float* lse_part, uint16_t* out_dev, uint16_t* out_host,
+                           float softmax_scale, const moska_shape* shape, void* ws,
+                           size_t ws_bytes, moska_stream stream, moska_stream side_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOSKA_H_ */
