@@ -1,0 +1,292 @@
+// extern "C" boundary of the MoSKA library: argument validation and launch sequencing only.
+#include <cstring>
+
+#include "common.cuh"
+
+namespace moska {
+
+char* last_error_buffer()
+{
+    static thread_local char buf[512] = {0};
+    return buf;
+}
+
+int fail(int status, const char* fmt, ...)
+{
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(last_error_buffer(), 512, fmt, ap);
+    va_end(ap);
+    return status;
+}
+
+int check_shape(const moska_shape* s, bool needs_k)
+{
+    if (s == nullptr) return fail(MOSKA_ERR_INVALID_ARG, "shape is NULL");
+    if (s->B < 0 || s->Hq <= 0 || s->Hkv <= 0 || s->C <= 0 || s->L <= 0)
+        return fail(MOSKA_ERR_INVALID_ARG, "B >= 0 and Hq, Hkv, C, L > 0 required");
+    if (s->Hq % s->Hkv != 0)
+        return fail(MOSKA_ERR_INVALID_ARG, "Hq = %d is not a multiple of Hkv = %d", s->Hq, s->Hkv);
+    if (s->Hq / s->Hkv > 8)
+        return fail(MOSKA_ERR_UNSUPPORTED, "G = Hq / Hkv = %d > 8", s->Hq / s->Hkv);
+    if (s->D != 64 && s->D != 128)
+        return fail(MOSKA_ERR_UNSUPPORTED, "D = %d, only 64 and 128 are built", s->D);
+    if (s->L % 128 != 0) return fail(MOSKA_ERR_UNSUPPORTED, "L = %d is not a multiple of 128", s->L);
+    if (needs_k && (s->k < 1 || s->k > s->C))
+        return fail(MOSKA_ERR_INVALID_ARG, "k = %d outside [1, C = %d]", s->k, s->C);
+    if (s->shared_slots < 1 || s->n_unique_splits < 1)
+        return fail(MOSKA_ERR_INVALID_ARG, "shared_slots and n_unique_splits must be >= 1");
+    if ((long long)s->B * s->Hkv * (long long)(s->k > 0 ? s->k : 1) > 0x7fffffffLL ||
+        (long long)s->Hkv * s->C >= 0x7fffffffLL)
+        return fail(MOSKA_ERR_UNSUPPORTED, "index range exceeds int32");
+    return MOSKA_OK;
+}
+
+int check_device()
+{
+    static thread_local int cached_dev = -1;
+    static thread_local int cached_major = 0;
+    int dev = 0;
+    MOSKA_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev != cached_dev) {
+        MOSKA_CUDA_TRY(cudaDeviceGetAttribute(&cached_major, cudaDevAttrComputeCapabilityMajor, dev));
+        cached_dev = dev;
+    }
+    if (cached_major != 10)
+        return fail(MOSKA_ERR_UNSUPPORTED, "device %d is compute capability %d.x, sm_100 required",
+                    dev, cached_major);
+    return MOSKA_OK;
+}
+
+}  // namespace moska
+
+using namespace moska;
+
+#define MOSKA_TRY(expr)              \
+    do {                             \
+        int st__ = (expr);           \
+        if (st__ != MOSKA_OK) return st__; \
+    } while (0)
+
+#define REQUIRE_PTR(p, align)                                                                   \
+    do {                                                                                        \
+        if ((p) == nullptr) return fail(MOSKA_ERR_INVALID_ARG, "%s is NULL", #p);               \
+        if (!aligned((p), (align)))                                                             \
+            return fail(MOSKA_ERR_INVALID_ARG, "%s is not %d-byte aligned", #p, (int)(align));  \
+    } while (0)
+
+extern "C" {
+
+int moska_version(void) { return 100; }
+
+const char* moska_last_error(void) { return last_error_buffer(); }
+
+int moska_partial_slots(const moska_shape* shape)
+{
+    MOSKA_TRY(check_shape(shape, false));
+    return shape->shared_slots + shape->n_unique_splits;
+}
+
+size_t moska_workspace_bytes(const moska_shape* shape)
+{
+    if (check_shape(shape, true) != MOSKA_OK) return 0;
+    return ws_layout(shape).total;
+}
+
+int moska_default_unique_splits(int32_t B, int32_t Hkv, int32_t max_len)
+{
+    // Enough CTAs to fill 148 SMs several times over, but at least 512 tokens per split so the
+    // per-CTA prologue and combine stay small next to the streaming loop.
+    if (B <= 0 || Hkv <= 0 || max_len <= 0) return 1;
+    const long long want_ctas = 148LL * 12;
+    long long n = (want_ctas + (long long)B * Hkv - 1) / ((long long)B * Hkv);
+    const long long cap = (max_len + 511) / 512;
+    if (n > cap) n = cap;
+    if (n < 1) n = 1;
+    if (n > 64) n = 64;
+    return (int)n;
+}
+
+int moska_build_chunk_summaries(const uint16_t* k_shared, float* summaries,
+                                const moska_shape* shape, moska_stream stream)
+{
+    MOSKA_TRY(check_shape(shape, false));
+    MOSKA_TRY(check_device());
+    REQUIRE_PTR(k_shared, 16);
+    REQUIRE_PTR(summaries, 16);
+    return launch_summaries(k_shared, summaries, shape, (cudaStream_t)stream);
+}
+
+int moska_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
+                const moska_shape* shape, moska_stream stream)
+{
+    MOSKA_TRY(check_shape(shape, true));
+    MOSKA_TRY(check_device());
+    REQUIRE_PTR(q, 16);
+    REQUIRE_PTR(summaries, 16);
+    REQUIRE_PTR(topk_idx, 4);
+    return launch_route(q, summaries, topk_idx, topk_score, shape, (cudaStream_t)stream);
+}
+
+int moska_group_by_chunk(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
+                         const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream)
+{
+    MOSKA_TRY(check_shape(shape, true));
+    MOSKA_TRY(check_device());
+    REQUIRE_PTR(topk_idx, 4);
+    REQUIRE_PTR(seg_offsets, 4);
+    REQUIRE_PTR(seg_entries, 4);
+    if (ws == nullptr || !aligned(ws, 256) || ws_bytes < ws_layout(shape).total)
+        return fail(MOSKA_ERR_WORKSPACE, "workspace missing, misaligned or smaller than %zu bytes",
+                    ws_layout(shape).total);
+    return launch_group(topk_idx, seg_offsets, seg_entries, shape, ws, (cudaStream_t)stream);
+}
+
+int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
+                      const int32_t* topk_idx, const int32_t* seg_offsets,
+                      const int32_t* seg_entries, float* o_part, float* lse_part,
+                      float softmax_scale, const moska_shape* shape, void* ws, size_t ws_bytes,
+                      moska_stream stream)
+{
+    const bool dense = (topk_idx == nullptr && seg_offsets == nullptr && seg_entries == nullptr);
+    MOSKA_TRY(check_shape(shape, !dense));
+    MOSKA_TRY(check_device());
+    REQUIRE_PTR(q, 16);
+    REQUIRE_PTR(k_shared, 128);
+    REQUIRE_PTR(v_shared, 128);
+    REQUIRE_PTR(o_part, 16);
+    REQUIRE_PTR(lse_part, 4);
+    if (!dense) {
+        REQUIRE_PTR(topk_idx, 4);
+        REQUIRE_PTR(seg_offsets, 4);
+        REQUIRE_PTR(seg_entries, 4);
+        if (shape->shared_slots != shape->k)
+            return fail(MOSKA_ERR_INVALID_ARG, "routed mode needs shared_slots == k");
+        if (ws == nullptr || !aligned(ws, 256) || ws_bytes < ws_layout(shape).total)
+            return fail(MOSKA_ERR_WORKSPACE, "workspace missing, misaligned or smaller than %zu bytes",
+                        ws_layout(shape).total);
+    } else if (shape->shared_slots > shape->C) {
+        return fail(MOSKA_ERR_INVALID_ARG, "dense mode needs shared_slots <= C");
+    }
+    return launch_shared_small(q, k_shared, v_shared, seg_entries, o_part, lse_part, softmax_scale,
+                               shape, ws, dense, (cudaStream_t)stream);
+}
+
+int moska_unique_attn(const uint16_t* q, const uint16_t* k_unique, const uint16_t* v_unique,
+                      const int64_t* kv_start, const int32_t* kv_len, float* o_part,
+                      float* lse_part, float softmax_scale, const moska_shape* shape,
+                      moska_stream stream)
+{
+    MOSKA_TRY(check_shape(shape, false));
+    MOSKA_TRY(check_device());
+    REQUIRE_PTR(q, 16);
+    REQUIRE_PTR(k_unique, 16);
+    REQUIRE_PTR(v_unique, 16);
+    REQUIRE_PTR(kv_start, 8);
+    REQUIRE_PTR(kv_len, 4);
+    REQUIRE_PTR(o_part, 16);
+    REQUIRE_PTR(lse_part, 4);
+    return launch_unique(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part, softmax_scale,
+                         shape, (cudaStream_t)stream);
+}
+
+int moska_merge(const float* o_part, const float* lse_part, uint16_t* out, float* out_f32,
+                float* lse_out, const moska_shape* shape, moska_stream stream)
+{
+    MOSKA_TRY(check_shape(shape, false));
+    MOSKA_TRY(check_device());
+    REQUIRE_PTR(o_part, 16);
+    REQUIRE_PTR(lse_part, 4);
+    REQUIRE_PTR(out, 8);
+    if (out_f32 != nullptr && !aligned(out_f32, 16))
+        return fail(MOSKA_ERR_INVALID_ARG, "out_f32 is not 16-byte aligned");
+    return launch_merge(o_part, lse_part, out, out_f32, lse_out, shape, (cudaStream_t)stream);
+}
+
+int moska_gemv_baseline(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
+                        const int32_t* topk_idx, float* o_part, float* lse_part,
+                        float softmax_scale, const moska_shape* shape, moska_stream stream)
+{
+    const bool dense = topk_idx == nullptr;
+    MOSKA_TRY(check_shape(shape, !dense));
+    MOSKA_TRY(check_device());
+    REQUIRE_PTR(q, 16);
+    REQUIRE_PTR(k_shared, 16);
+    REQUIRE_PTR(v_shared, 16);
+    REQUIRE_PTR(o_part, 16);
+    REQUIRE_PTR(lse_part, 4);
+    if (!dense && shape->shared_slots != shape->k)
+        return fail(MOSKA_ERR_INVALID_ARG, "routed mode needs shared_slots == k");
+    if (dense && shape->shared_slots > shape->C)
+        return fail(MOSKA_ERR_INVALID_ARG, "dense mode needs shared_slots <= C");
+    return launch_gemv_baseline(q, k_shared, v_shared, topk_idx, o_part, lse_part, softmax_scale,
+                                shape, (cudaStream_t)stream);
+}
+
+int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t* k_shared,
+                      const uint16_t* v_shared, const uint16_t* k_unique,
+                      const uint16_t* v_unique, const int64_t* kv_start, const int32_t* kv_len,
+                      int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
+                      float* o_part, float* lse_part, uint16_t* out, float* lse_out,
+                      float softmax_scale, const moska_shape* shape, void* ws, size_t ws_bytes,
+                      moska_stream stream, moska_stream side_stream)
+{
+    const bool dense = summaries == nullptr;
+    cudaStream_t st = (cudaStream_t)stream, side = (cudaStream_t)side_stream;
+    // Fork/join events for the optional second stream, created once per host thread.
+    static thread_local cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    if (side != nullptr && ev_fork == nullptr) {
+        MOSKA_CUDA_TRY(cudaEventCreateWithFlags(&ev_fork, cudaEventDisableTiming));
+        MOSKA_CUDA_TRY(cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming));
+    }
+    // Unique attention depends on nothing upstream: start it first on the side stream.
+    if (side != nullptr) {
+        MOSKA_CUDA_TRY(cudaEventRecord(ev_fork, st));
+        MOSKA_CUDA_TRY(cudaStreamWaitEvent(side, ev_fork, 0));
+        MOSKA_TRY(moska_unique_attn(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part,
+                                    softmax_scale, shape, side));
+        MOSKA_CUDA_TRY(cudaEventRecord(ev_join, side));
+    }
+    if (!dense) {
+        MOSKA_TRY(moska_route(q, summaries, topk_idx, nullptr, shape, st));
+        MOSKA_TRY(moska_group_by_chunk(topk_idx, seg_offsets, seg_entries, shape, ws, ws_bytes, st));
+        MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, topk_idx, seg_offsets, seg_entries,
+                                    o_part, lse_part, softmax_scale, shape, ws, ws_bytes, st));
+    } else {
+        MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, nullptr, nullptr, nullptr, o_part,
+                                    lse_part, softmax_scale, shape, ws, ws_bytes, st));
+    }
+    if (side != nullptr) {
+        MOSKA_CUDA_TRY(cudaStreamWaitEvent(st, ev_join, 0));
+    } else {
+        MOSKA_TRY(moska_unique_attn(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part,
+                                    softmax_scale, shape, st));
+    }
+    return moska_merge(o_part, lse_part, out, nullptr, lse_out, shape, st);
+}
+
+int moska_decode_step_host(const uint16_t* q_host, uint16_t* q_dev, const float* summaries,
+                           const uint16_t* k_shared, const uint16_t* v_shared,
+                           const uint16_t* k_unique, const uint16_t* v_unique,
+                           const int64_t* kv_start, const int32_t* kv_len, int32_t* topk_idx,
+                           int32_t* seg_offsets, int32_t* seg_entries, float* o_part,
+                           float* lse_part, uint16_t* out_dev, uint16_t* out_host,
+                           float softmax_scale, const moska_shape* shape, void* ws,
+                           size_t ws_bytes, moska_stream stream, moska_stream side_stream)
+{
+    MOSKA_TRY(check_shape(shape, summaries != nullptr));
+    if (q_host == nullptr || q_dev == nullptr || out_dev == nullptr || out_host == nullptr)
+        return fail(MOSKA_ERR_INVALID_ARG, "q_host, q_dev, out_dev and out_host must not be NULL");
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t bytes = sizeof(uint16_t) * (size_t)shape->B * shape->Hq * shape->D;
+    MOSKA_CUDA_TRY(cudaMemcpyAsync(q_dev, q_host, bytes, cudaMemcpyHostToDevice, st));
+    MOSKA_TRY(moska_decode_step(q_dev, summaries, k_shared, v_shared, k_unique, v_unique, kv_start,
+                                kv_len, topk_idx, seg_offsets, seg_entries, o_part, lse_part,
+                                out_dev, nullptr, softmax_scale, shape, ws, ws_bytes, stream,
+                                side_stream));
+    MOSKA_CUDA_TRY(cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, st));
+    MOSKA_CUDA_TRY(cudaStreamSynchronize(st));
+    return MOSKA_OK;
+}
+
+}  // extern "C"

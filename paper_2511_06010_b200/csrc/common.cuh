@@ -1,0 +1,93 @@
+// Shared host/device helpers of the MoSKA CUDA library (sm_100a only).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <cstdarg>
+#include <cstdio>
+
+#include "moska.h"
+
+namespace moska {
+
+// ---- error reporting -------------------------------------------------------------------------
+char* last_error_buffer();  // thread-local, 512 bytes
+int fail(int status, const char* fmt, ...);
+
+#define MOSKA_CUDA_TRY(expr)                                                              \
+    do {                                                                                  \
+        cudaError_t err__ = (expr);                                                       \
+        if (err__ != cudaSuccess)                                                         \
+            return ::moska::fail(MOSKA_ERR_CUDA, "%s failed: %s", #expr,                  \
+                                 cudaGetErrorString(err__));                              \
+    } while (0)
+
+#define MOSKA_LAUNCH_CHECK(name)                                                          \
+    do {                                                                                  \
+        cudaError_t err__ = cudaGetLastError();                                           \
+        if (err__ != cudaSuccess)                                                         \
+            return ::moska::fail(MOSKA_ERR_CUDA, "launch of %s failed: %s", name,         \
+                                 cudaGetErrorString(err__));                              \
+    } while (0)
+
+// Validates the shape fields every entry point relies on; returns MOSKA_OK or a negative status.
+int check_shape(const moska_shape* s, bool needs_k);
+// MOSKA_OK if the current device is compute capability 10.x.
+int check_device();
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---- workspace layout (route / group / shared attention) ---------------------------------------
+// One work item of shared attention: `n_entries` consecutive entries of segment `key`,
+// starting at seg_entries[entry_begin].
+struct TileItem {
+    int32_t key;          // h * C + c
+    int32_t entry_begin;  // absolute index into seg_entries
+    int32_t n_entries;    // requests in this tile (rows = n_entries * G)
+    int32_t pad;
+};
+
+struct WsHeader {
+    int32_t n_small_tiles;  // items in the small-tile list
+    int32_t n_big_tiles;    // items in the big-tile list
+    int32_t status;         // 0, or a negative code set by a device-side range check
+    int32_t pad[61];
+};
+static_assert(sizeof(WsHeader) == 256, "header is one 256-byte block");
+
+struct WsLayout {
+    int32_t n_blocks;         // request blocks of the counting sort
+    int32_t n_keys;           // Hkv * C
+    int32_t small_entries;    // requests per small tile
+    int32_t big_entries;      // requests per big tile
+    int32_t big_min_entries;  // a remainder of at least this many requests still forms a big tile
+    int64_t max_small, max_big;
+    size_t off_hist, off_totals, off_small, off_big, total;
+};
+WsLayout ws_layout(const moska_shape* s);
+
+constexpr int kSmallTileRows = 16;  // query rows of one small tile (two 8-row MMA column blocks)
+constexpr int kBigTileRows = 128;   // query rows of one tensor-core (tcgen05) tile
+
+// ---- internal launchers (one per .cu file) -----------------------------------------------------
+int launch_summaries(const uint16_t* k_shared, float* summaries, const moska_shape* s,
+                     cudaStream_t st);
+int launch_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
+                 const moska_shape* s, cudaStream_t st);
+int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
+                 const moska_shape* s, void* ws, cudaStream_t st);
+int launch_shared_small(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
+                        const int32_t* seg_entries, float* o_part, float* lse_part, float scale,
+                        const moska_shape* s, void* ws, bool dense, cudaStream_t st);
+int launch_unique(const uint16_t* q, const uint16_t* k_unique, const uint16_t* v_unique,
+                  const int64_t* kv_start, const int32_t* kv_len, float* o_part, float* lse_part,
+                  float scale, const moska_shape* s, cudaStream_t st);
+int launch_gemv_baseline(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
+                         const int32_t* topk_idx, float* o_part, float* lse_part, float scale,
+                         const moska_shape* s, cudaStream_t st);
+int launch_merge(const float* o_part, const float* lse_part, uint16_t* out, float* out_f32,
+                 float* lse_out, const moska_shape* s, cudaStream_t st);
+
+}  // namespace moska

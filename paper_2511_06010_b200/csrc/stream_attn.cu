@@ -1,0 +1,234 @@
+// Kernels built on the streaming decode-attention block: Unique KV Attention, the unbatched
+// per-request GEMV baseline over shared chunks, and Shared KV Attention for small query tiles.
+#include "common.cuh"
+#include "stream_attn.cuh"
+
+namespace moska {
+using namespace stream;
+
+namespace {
+
+template <int NT>
+__device__ __forceinline__ void clear_rows(TileRows<NT>& rows)
+{
+    for (int i = threadIdx.x; i < NT * 8; i += kThreads) {
+        rows.q[i] = nullptr;
+        rows.o[i] = nullptr;
+        rows.lse[i] = nullptr;
+    }
+}
+
+// Token range of split `s` of a request with `len` unique tokens: equal parts rounded up to a
+// whole number of CTA passes (kWarps * 16 tokens), so trailing splits of short requests are empty.
+__device__ __forceinline__ void split_range(int len, int n_splits, int s, int& t0, int& t1)
+{
+    constexpr int kQuantum = kWarps * kTileTokens;
+    int per = (len + n_splits - 1) / n_splits;
+    per = (per + kQuantum - 1) / kQuantum * kQuantum;
+    t0 = min(len, s * per);
+    t1 = min(len, t0 + per);
+}
+
+// ---- Unique KV Attention (Section III-A): one CTA per (request, KV head, split) ----------------
+template <int D>
+__global__ void __launch_bounds__(kThreads, 3)
+unique_attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_unique,
+                   const uint16_t* __restrict__ v_unique, const int64_t* __restrict__ kv_start,
+                   const int32_t* __restrict__ kv_len, float* __restrict__ o_part,
+                   float* __restrict__ lse_part, float scale, int Hq, int Hkv, int n_splits,
+                   int slot0, int n_slots)
+{
+    __shared__ TileRows<1> rows;
+    __shared__ CombineSmem<D, 1> sm;
+    const int G = Hq / Hkv;
+    // KV heads of the same (request, split) sit in neighbouring CTAs: together they read whole
+    // token rows of the [T][Hkv][D] store.
+    const int h = blockIdx.x % Hkv;
+    const int s = (blockIdx.x / Hkv) % n_splits;
+    const int b = blockIdx.x / (Hkv * n_splits);
+    clear_rows(rows);
+    __syncthreads();
+    if (threadIdx.x < G) {
+        const int64_t r = (int64_t)b * Hq + h * G + threadIdx.x;
+        rows.q[threadIdx.x] = q + r * D;
+        rows.o[threadIdx.x] = o_part + (r * n_slots + slot0 + s) * D;
+        rows.lse[threadIdx.x] = lse_part + r * n_slots + slot0 + s;
+    }
+    __syncthreads();
+    int t0, t1;
+    split_range(kv_len[b], n_splits, s, t0, t1);
+    const int64_t stride = (int64_t)Hkv * D;
+    const uint16_t* kb = k_unique + kv_start[b] * stride + (int64_t)h * D;
+    const uint16_t* vb = v_unique + kv_start[b] * stride + (int64_t)h * D;
+    attend_stream<D, 1>(rows, kb, vb, stride, t0, t1, scale, sm);
+}
+
+// ---- per-request GEMV baseline over shared chunks: one CTA per (request, KV head, slot) ---------
+template <int D>
+__global__ void __launch_bounds__(kThreads, 3)
+gemv_baseline_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_shared,
+                     const uint16_t* __restrict__ v_shared, const int32_t* __restrict__ topk_idx,
+                     float* __restrict__ o_part, float* __restrict__ lse_part, float scale,
+                     int Hq, int Hkv, int C, int L, int k, int shared_slots, int n_slots)
+{
+    __shared__ TileRows<1> rows;
+    __shared__ CombineSmem<D, 1> sm;
+    const int G = Hq / Hkv;
+    const int j = blockIdx.x % shared_slots;
+    const int h = (blockIdx.x / shared_slots) % Hkv;
+    const int b = blockIdx.x / (shared_slots * Hkv);
+    clear_rows(rows);
+    __syncthreads();
+    if (threadIdx.x < G) {
+        const int64_t r = (int64_t)b * Hq + h * G + threadIdx.x;
+        rows.q[threadIdx.x] = q + r * D;
+        rows.o[threadIdx.x] = o_part + (r * n_slots + j) * D;
+        rows.lse[threadIdx.x] = lse_part + r * n_slots + j;
+    }
+    __syncthreads();
+    int64_t tok0;
+    int n_tok;
+    if (topk_idx != nullptr) {  // routed: slot j is chunk topk_idx[b][h][j]
+        tok0 = ((int64_t)h * C + topk_idx[((int64_t)b * Hkv + h) * k + j]) * L;
+        n_tok = L;
+    } else {                    // dense: slot j is the j-th run of consecutive chunks
+        const int run = (C + shared_slots - 1) / shared_slots;
+        const int c0 = min(C, j * run), c1 = min(C, c0 + run);
+        tok0 = ((int64_t)h * C + c0) * L;
+        n_tok = (c1 - c0) * L;
+    }
+    attend_stream<D, 1>(rows, k_shared + tok0 * D, v_shared + tok0 * D, D, 0, n_tok, scale, sm);
+}
+
+// ---- Shared KV Attention, small tiles (Section III-A) ------------------------------------------
+// Routed mode: one CTA per work item = up to 16/G requests of one (KV head, chunk) segment; the
+// chunk's K/V is streamed once for all of them.  Dense mode: one CTA per (KV head, run of chunks,
+// group of 16/G requests).
+template <int D>
+__global__ void __launch_bounds__(kThreads, 2)
+shared_small_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_shared,
+                    const uint16_t* __restrict__ v_shared, const int32_t* __restrict__ seg_entries,
+                    const WsHeader* __restrict__ hdr, const TileItem* __restrict__ items,
+                    float* __restrict__ o_part, float* __restrict__ lse_part, float scale, int B,
+                    int Hq, int Hkv, int C, int L, int k, int shared_slots, int n_slots, int dense)
+{
+    constexpr int NT = kSmallTileRows / 8;
+    __shared__ TileRows<NT> rows;
+    __shared__ CombineSmem<D, NT> sm;
+    const int G = Hq / Hkv;
+    const int per_tile = kSmallTileRows / G;  // requests per tile
+    clear_rows(rows);
+    __syncthreads();
+    int64_t tok0;
+    int n_tok;
+    if (!dense) {
+        if ((int)blockIdx.x >= hdr->n_small_tiles) return;
+        const TileItem it = items[blockIdx.x];
+        const int h = it.key / C;
+        if (threadIdx.x < it.n_entries * G) {
+            const int p = seg_entries[it.entry_begin + threadIdx.x / G];
+            const int g = threadIdx.x % G;
+            const int j = p % k, b = p / (k * Hkv);
+            const int64_t r = (int64_t)b * Hq + h * G + g;
+            rows.q[threadIdx.x] = q + r * D;
+            rows.o[threadIdx.x] = o_part + (r * n_slots + j) * D;
+            rows.lse[threadIdx.x] = lse_part + r * n_slots + j;
+        }
+        tok0 = (int64_t)it.key * L;
+        n_tok = L;
+    } else {
+        const int b_tiles = (B + per_tile - 1) / per_tile;
+        const int bt = blockIdx.x % b_tiles;
+        const int j = (blockIdx.x / b_tiles) % shared_slots;
+        const int h = blockIdx.x / (b_tiles * shared_slots);
+        const int b = bt * per_tile + threadIdx.x / G;
+        if (threadIdx.x < per_tile * G && b < B) {
+            const int64_t r = (int64_t)b * Hq + h * G + threadIdx.x % G;
+            rows.q[threadIdx.x] = q + r * D;
+            rows.o[threadIdx.x] = o_part + (r * n_slots + j) * D;
+            rows.lse[threadIdx.x] = lse_part + r * n_slots + j;
+        }
+        const int run = (C + shared_slots - 1) / shared_slots;
+        const int c0 = min(C, j * run), c1 = min(C, c0 + run);
+        tok0 = ((int64_t)h * C + c0) * L;
+        n_tok = (c1 - c0) * L;
+    }
+    __syncthreads();
+    attend_stream<D, NT>(rows, k_shared + tok0 * D, v_shared + tok0 * D, D, 0, n_tok, scale, sm);
+}
+
+}  // namespace
+
+int launch_unique(const uint16_t* q, const uint16_t* k_unique, const uint16_t* v_unique,
+                  const int64_t* kv_start, const int32_t* kv_len, float* o_part, float* lse_part,
+                  float scale, const moska_shape* s, cudaStream_t st)
+{
+    const int n_slots = s->shared_slots + s->n_unique_splits;
+    const long long grid = (long long)s->B * s->Hkv * s->n_unique_splits;
+    if (grid == 0) return MOSKA_OK;
+    if (grid > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "unique attention grid too large");
+    if (s->D == 128)
+        unique_attn_kernel<128><<<(unsigned)grid, kThreads, 0, st>>>(
+            q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part, scale, s->Hq, s->Hkv,
+            s->n_unique_splits, s->shared_slots, n_slots);
+    else
+        unique_attn_kernel<64><<<(unsigned)grid, kThreads, 0, st>>>(
+            q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part, scale, s->Hq, s->Hkv,
+            s->n_unique_splits, s->shared_slots, n_slots);
+    MOSKA_LAUNCH_CHECK("unique_attn_kernel");
+    return MOSKA_OK;
+}
+
+int launch_gemv_baseline(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
+                         const int32_t* topk_idx, float* o_part, float* lse_part, float scale,
+                         const moska_shape* s, cudaStream_t st)
+{
+    const int n_slots = s->shared_slots + s->n_unique_splits;
+    const long long grid = (long long)s->B * s->Hkv * s->shared_slots;
+    if (grid == 0) return MOSKA_OK;
+    if (grid > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "baseline grid too large");
+    if (s->D == 128)
+        gemv_baseline_kernel<128><<<(unsigned)grid, kThreads, 0, st>>>(
+            q, k_shared, v_shared, topk_idx, o_part, lse_part, scale, s->Hq, s->Hkv, s->C, s->L,
+            s->k, s->shared_slots, n_slots);
+    else
+        gemv_baseline_kernel<64><<<(unsigned)grid, kThreads, 0, st>>>(
+            q, k_shared, v_shared, topk_idx, o_part, lse_part, scale, s->Hq, s->Hkv, s->C, s->L,
+            s->k, s->shared_slots, n_slots);
+    MOSKA_LAUNCH_CHECK("gemv_baseline_kernel");
+    return MOSKA_OK;
+}
+
+int launch_shared_small(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
+                        const int32_t* seg_entries, float* o_part, float* lse_part, float scale,
+                        const moska_shape* s, void* ws, bool dense, cudaStream_t st)
+{
+    const int n_slots = s->shared_slots + s->n_unique_splits;
+    const int G = s->Hq / s->Hkv;
+    long long grid;
+    const WsHeader* hdr = nullptr;
+    const TileItem* items = nullptr;
+    if (dense) {
+        const int per_tile = kSmallTileRows / G;
+        grid = (long long)s->Hkv * s->shared_slots * ((s->B + per_tile - 1) / per_tile);
+    } else {
+        const WsLayout lay = ws_layout(s);
+        grid = lay.max_small;
+        hdr = reinterpret_cast<const WsHeader*>(ws);
+        items = reinterpret_cast<const TileItem*>(static_cast<const char*>(ws) + lay.off_small);
+    }
+    if (grid == 0) return MOSKA_OK;
+    if (grid > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "shared attention grid too large");
+    if (s->D == 128)
+        shared_small_kernel<128><<<(unsigned)grid, kThreads, 0, st>>>(
+            q, k_shared, v_shared, seg_entries, hdr, items, o_part, lse_part, scale, s->B, s->Hq,
+            s->Hkv, s->C, s->L, s->k, s->shared_slots, n_slots, dense ? 1 : 0);
+    else
+        shared_small_kernel<64><<<(unsigned)grid, kThreads, 0, st>>>(
+            q, k_shared, v_shared, seg_entries, hdr, items, o_part, lse_part, scale, s->B, s->Hq,
+            s->Hkv, s->C, s->L, s->k, s->shared_slots, n_slots, dense ? 1 : 0);
+    MOSKA_LAUNCH_CHECK("shared_small_kernel");
+    return MOSKA_OK;
+}
+
+}  // namespace moska

@@ -1,0 +1,76 @@
+"""CPU-side checks of the C ABI: the library builds, loads, exports every declared symbol, and
+rejects bad arguments on the host before touching a GPU.  No compute call is made here."""
+import ctypes
+import os
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def M():
+    from paper_2511_06010_b200 import build
+
+    build.build()
+    from paper_2511_06010_b200 import binding
+
+    return binding
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "moska.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(moska_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported_and_bound(M):
+    names = declared_symbols()
+    assert len(names) >= 12
+    lib = ctypes.CDLL(M.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in moska.h but not exported"
+        assert n in M.EXPORTS, f"{n} has no Python binding"
+        assert hasattr(M, n[len("moska_"):]), f"binding function for {n} missing"
+    assert M.version() >= 100
+
+
+def test_pure_host_helpers(M):
+    s = M.shape(64, 32, 8, 128, 128, 512, 8, n_unique_splits=4)
+    assert M.partial_slots(s) == 12
+    assert M.workspace_bytes(s) > 256 and M.workspace_bytes(s) % 256 == 0
+    assert 1 <= M.default_unique_splits(64, 8, 4096) <= 8
+    assert M.default_unique_splits(1024, 8, 32768) >= 1
+    assert M.default_unique_splits(4, 1, 100) == 1
+
+
+@pytest.mark.parametrize("kwargs,status", [
+    (dict(Hq=30), -1),            # Hq % Hkv != 0
+    (dict(D=96), -2),             # unsupported head dim
+    (dict(Hq=128), -2),           # G = 16 > 8
+    (dict(L=100), -2),            # L not a multiple of 128
+    (dict(k=0), -1),
+    (dict(k=129), -1),            # k > C
+])
+def test_bad_shapes_are_rejected_on_the_host(M, kwargs, status):
+    base = dict(B=4, Hq=32, Hkv=8, D=128, C=128, L=512, k=8)
+    base.update(kwargs)
+    s = M.shape(**base)
+    with pytest.raises(M.MoskaError) as e:
+        M.route(0x1000, 0x1000, 0x1000, None, s, stream=0)
+    assert e.value.status == status
+    assert M.last_error() != ""
+
+
+def test_null_pointer_and_workspace_errors_come_before_any_launch(M):
+    s = M.shape(4, 32, 8, 128, 128, 512, 8)
+    with pytest.raises(M.MoskaError) as e:
+        M.merge(None, 0x1000, 0x1000, None, None, s, stream=0)
+    # NULL is reported as invalid argument unless the device check (no GPU here) comes first
+    assert e.value.status in (M.ERR_INVALID_ARG, M.ERR_CUDA, M.ERR_UNSUPPORTED)
+    bad = M.shape(4, 32, 8, 128, 128, 512, 8, shared_slots=0)
+    with pytest.raises(M.MoskaError) as e:
+        M.partial_slots(bad)
+    assert e.value.status == M.ERR_INVALID_ARG
+    assert M.workspace_bytes(bad) == 0

@@ -1,0 +1,278 @@
+"""GPU parity: every stage of the CUDA path, called through the C ABI, against the fp64 oracle.
+
+Small cases are compared element by element; the full-size benchmark workloads are compared on
+sampled requests (all of their rows), routing and grouping always in full.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2511_06010_b200 import workloads as W
+from tests import parity_utils as PU
+
+pytestmark = pytest.mark.gpu
+
+
+def _mods():
+    from paper_2511_06010_b200 import binding as M
+    from paper_2511_06010_b200.engine import MoskaLayer
+
+    return M, MoskaLayer
+
+
+def _subproblem(q, topk, sh, un, kv_len, sample):
+    """Host copies of what the oracle needs for the sampled requests only: their queries, their
+    unique tokens (compacted) and the shared chunks they were routed to (compacted, indices
+    remapped in order).  Pure indexing."""
+    sample = np.asarray(sample)
+    q_s = q[sample].cpu()
+    topk_s = topk[sample].cpu().numpy()                       # [n][Hkv][k]
+    Hkv = topk_s.shape[1]
+    unions = [np.unique(topk_s[:, h]) for h in range(Hkv)]
+    Cc = max(len(u) for u in unions)
+    L, D = sh.k_shared.shape[2], sh.k_shared.shape[3]
+    ks = torch.zeros(Hkv, Cc, L, D, dtype=torch.bfloat16)
+    vs = torch.zeros(Hkv, Cc, L, D, dtype=torch.bfloat16)
+    remap = np.empty_like(topk_s)
+    for h, u in enumerate(unions):
+        idx = torch.from_numpy(u).to(sh.k_shared.device)
+        ks[h, :len(u)] = sh.k_shared[h].index_select(0, idx).cpu()
+        vs[h, :len(u)] = sh.v_shared[h].index_select(0, idx).cpu()
+        remap[:, h] = np.searchsorted(u, topk_s[:, h])
+    lens = kv_len.cpu().numpy()[sample].astype(np.int32)
+    starts_dev = un.kv_start.cpu().numpy()[sample]
+    new_start = np.concatenate([[0], np.cumsum(lens)[:-1]]).astype(np.int64)
+    T = max(1, int(lens.sum()))
+    ku = torch.zeros(T, Hkv, D, dtype=torch.bfloat16)
+    vu = torch.zeros(T, Hkv, D, dtype=torch.bfloat16)
+    for i in range(len(sample)):
+        s0, n = int(starts_dev[i]), int(lens[i])
+        ku[new_start[i]:new_start[i] + n] = un.k_unique[s0:s0 + n].cpu()
+        vu[new_start[i]:new_start[i] + n] = un.v_unique[s0:s0 + n].cpu()
+    return q_s, remap.astype(np.int32), ks, vs, ku, vu, new_start, lens
+
+
+def run_case(w: W.Workload, sample=None, lengths=None, n_unique_splits=None, step=0,
+             check_baseline=True, two_streams=False):
+    """All stages of one decode step of workload `w` against the oracle."""
+    M, MoskaLayer = _mods()
+    dev = "cuda"
+    sh = W.make_shared_store(w, dev)
+    un = W.make_unique_store(w, dev, lengths)
+    q = W.make_queries(w, sh, step, dev)
+    kv_len = (un.kv_len + step).to(torch.int32)
+    max_len = int(kv_len.max().item()) if w.B else 1
+    layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, max_len, dense=w.dense,
+                       n_unique_splits=n_unique_splits)
+    S = layer.shape
+    scale = layer.scale
+    sample = np.arange(w.B) if sample is None else np.asarray(sample)
+    report = {}
+
+    # ---- summaries + routing + grouping: always in full, bit-exact (near-tie rule for routing)
+    if not w.dense:
+        layer.build_summaries(sh.k_shared)
+        summ_ref = O.chunk_summaries(sh.k_shared.cpu())
+        summ_gpu = layer.summaries.cpu().numpy().astype(np.float64)
+        np.testing.assert_allclose(summ_gpu, summ_ref, rtol=0, atol=4e-6)
+        layer.route(q)
+        ref_idx, ref_sc, ref_all = O.route(q.cpu(), summ_ref, w.k, return_all=True)
+        gpu_idx = layer.topk_idx.cpu().numpy()
+        report["routing_excused_rows"] = PU.check_routing(gpu_idx, ref_idx, ref_all)
+        gpu_sc = layer.topk_score.cpu().numpy().astype(np.float64)
+        picked = np.take_along_axis(ref_all, gpu_idx.astype(np.int64), axis=-1)
+        np.testing.assert_allclose(gpu_sc, picked, rtol=1e-4, atol=1e-3)
+        layer.group()
+        off_ref, ent_ref = O.group_by_chunk(gpu_idx, w.C, fast=True)
+        assert np.array_equal(layer.seg_offsets.cpu().numpy(), off_ref)
+        assert np.array_equal(layer.seg_entries.cpu().numpy()[: len(ent_ref)], ent_ref)
+        status = layer.ws[:12].view(torch.int32).cpu().numpy()
+        assert status[2] == 0, "device-side range check of the grouping fired"
+        topk = layer.topk_idx
+    else:
+        topk = torch.arange(w.C, dtype=torch.int32, device=dev).repeat(w.B, w.Hkv, 1)
+
+    q_s, topk_s, ks, vs, ku, vu, st_s, len_s = _subproblem(q, topk, sh, un, kv_len, sample)
+    n_sh = S.shared_slots
+
+    # ---- shared attention: one partial per (row, slot)
+    def shared_reference():
+        if not w.dense:
+            return O.shared_partials(q_s, ks, vs, topk_s, scale)
+        run = -(-w.C // n_sh)
+        o_ref = np.zeros((len(sample), w.Hq, n_sh, w.D))
+        l_ref = np.full((len(sample), w.Hq, n_sh), -np.inf)
+        for s in range(n_sh):
+            c0, c1 = min(w.C, s * run), min(w.C, (s + 1) * run)
+            if c1 == c0:
+                continue
+            tk = np.tile(np.arange(c0, c1, dtype=np.int32), (len(sample), w.Hkv, 1))
+            o_ref[:, :, s], l_ref[:, :, s] = O.attend_direct(
+                q_s, ks, vs, ku, vu, st_s, len_s, tk, scale, use_unique=False)
+        return o_ref, l_ref
+
+    o_ref, l_ref = shared_reference()
+    layer.o_part.fill_(float("nan"))
+    layer.lse_part.fill_(float("nan"))
+    layer.shared(q, sh.k_shared, sh.v_shared)
+    torch.cuda.synchronize()
+    o_gpu = layer.o_part[sample][:, :, :n_sh].cpu().numpy()
+    l_gpu = layer.lse_part[sample][:, :, :n_sh].cpu().numpy()
+    report["shared_lse"] = PU.check_lse(l_gpu, l_ref, "shared lse")
+    report["shared_o"] = PU.check_attention(o_gpu, o_ref, "shared partial o")
+    assert torch.isfinite(layer.o_part[:, :, :n_sh]).all(), "a shared slot was left unwritten"
+
+    # ---- per-request GEMV baseline: same result, same slots
+    if check_baseline:
+        layer.o_part[:, :, :n_sh].fill_(float("nan"))
+        layer.lse_part[:, :, :n_sh].fill_(float("nan"))
+        layer.gemv_baseline(q, sh.k_shared, sh.v_shared)
+        torch.cuda.synchronize()
+        PU.check_lse(layer.lse_part[sample][:, :, :n_sh].cpu().numpy(), l_ref, "baseline lse")
+        PU.check_attention(layer.o_part[sample][:, :, :n_sh].cpu().numpy(), o_ref, "baseline o")
+
+    # ---- unique attention: the split partials, merged in fp64, equal the unique partial
+    layer.unique(q, un.k_unique, un.v_unique, un.kv_start, kv_len)
+    torch.cuda.synchronize()
+    o_un = layer.o_part[sample][:, :, n_sh:].cpu().numpy()
+    l_un = layer.lse_part[sample][:, :, n_sh:].cpu().numpy()
+    assert not np.isnan(l_un).any() and np.isfinite(o_un).all(), "a unique slot was left unwritten"
+    o_um, l_um = O.merge(o_un, l_un)
+    o_uref, l_uref = O.attend_direct(q_s, ks, vs, ku, vu, st_s, len_s, topk_s, scale,
+                                     use_shared=False)
+    report["unique_lse"] = PU.check_lse(l_um, l_uref, "unique lse")
+    report["unique_o"] = PU.check_attention(o_um, o_uref, "unique partial o")
+
+    # ---- merge of the GPU partials vs the oracle's merge of the same partials (fp32 out)
+    layer.merge()
+    torch.cuda.synchronize()
+    o_all = layer.o_part[sample].cpu().numpy()
+    l_all = layer.lse_part[sample].cpu().numpy()
+    m_ref, ml_ref = O.merge(o_all, l_all)
+    PU.check_attention(layer.out_f32[sample].cpu().numpy(), m_ref, "merge", max_abs=1e-5, row_rel=1e-5)
+    PU.check_lse(layer.lse_out[sample].cpu().numpy(), ml_ref, "merge lse", tol=1e-4)
+
+    # ---- the whole step through moska_decode_step vs the definition (one softmax over the union)
+    layer.out.zero_()
+    out = layer.step(q, sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, un.kv_start, kv_len,
+                     two_streams=two_streams)
+    torch.cuda.synchronize()
+    ref_out, ref_lse = O.attend_direct(q_s, ks, vs, ku, vu, st_s, len_s, topk_s, scale)
+    report["out"] = PU.check_attention(out[sample].float().cpu().numpy(), ref_out, "decode step out")
+    report["lse"] = PU.check_lse(layer.lse_out[sample].cpu().numpy(), ref_lse, "decode step lse")
+    return report
+
+
+# ------------------------------------------------------------------------------------------------
+def test_cfg0_every_element():
+    r = run_case(W.CONFIGS[0])
+    assert r["routing_excused_rows"] == 0
+
+
+def test_small_ragged_tails_and_empty_requests():
+    """Unique lengths around every tile boundary, including empty requests; D = 64 and 128."""
+    lens = np.array([0, 1, 15, 16, 17, 63, 64, 65, 127, 129, 1000, 5], dtype=np.int64)
+    for D, Hq, Hkv in ((64, 4, 1), (128, 8, 2), (128, 8, 1), (64, 6, 2)):
+        w = W.Workload("ragged", B=len(lens), Hq=Hq, Hkv=Hkv, D=D, C=6, L=128, k=3,
+                       unique_len=0, seed=3)
+        run_case(w, lengths=lens, n_unique_splits=3)
+        run_case(w, lengths=lens, n_unique_splits=1)
+
+
+def test_single_request_and_k_equals_C():
+    w = W.Workload("b1", B=1, Hq=8, Hkv=2, D=128, C=4, L=256, k=4, unique_len=40, seed=4)
+    # k == C through the ROUTED path: must reproduce dense attention
+    M, MoskaLayer = _mods()
+    sh = W.make_shared_store(w, "cuda")
+    un = W.make_unique_store(w, "cuda")
+    q = W.make_queries(w, sh, 0, "cuda")
+    layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, 40, dense=False)
+    layer.build_summaries(sh.k_shared)
+    out = layer.step(q, sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, un.kv_start, un.kv_len)
+    torch.cuda.synchronize()
+    assert np.array_equal(layer.topk_idx.cpu().numpy()[0, 0], np.arange(4))
+    tk = np.tile(np.arange(4, dtype=np.int32), (1, 2, 1))
+    ref, _ = O.attend_direct(q.cpu(), sh.k_shared.cpu(), sh.v_shared.cpu(), un.k_unique.cpu(),
+                             un.v_unique.cpu(), un.kv_start.cpu(), un.kv_len.cpu(), tk, layer.scale)
+    PU.check_attention(out.float().cpu().numpy(), ref, "k == C routed")
+    # and the dense entry (no routing) gives the same
+    run_case(W.scaled(w, B=3))
+
+
+def test_exact_ties_route_to_lower_chunk():
+    """Duplicate chunks give bit-identical fp32 scores; the lower index must win."""
+    M, MoskaLayer = _mods()
+    w = W.Workload("ties", B=8, Hq=4, Hkv=2, D=64, C=8, L=128, k=3, unique_len=16, seed=5)
+    sh = W.make_shared_store(w, "cuda")
+    sh.k_shared[:, 5] = sh.k_shared[:, 1]
+    sh.k_shared[:, 6] = sh.k_shared[:, 1]
+    q = W.make_queries(w, sh, 0, "cuda")
+    layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, 16)
+    layer.build_summaries(sh.k_shared)
+    layer.route(q)
+    summ = O.chunk_summaries(sh.k_shared.cpu())
+    ref_idx, _ = O.route(q.cpu(), summ, w.k)
+    assert np.array_equal(layer.topk_idx.cpu().numpy(), ref_idx)
+    # all-zero queries: every score is exactly 0 -> chunks 0..k-1
+    layer.route(torch.zeros_like(q))
+    assert np.array_equal(layer.topk_idx.cpu().numpy(),
+                          np.tile(np.arange(3, dtype=np.int32), (8, 2, 1)))
+
+
+def test_run_twice_bitwise_identical():
+    M, MoskaLayer = _mods()
+    w = W.scaled(W.CONFIGS[1], B=16, C=32, unique_len=700)
+    sh = W.make_shared_store(w, "cuda")
+    un = W.make_unique_store(w, "cuda")
+    q = W.make_queries(w, sh, 0, "cuda")
+    layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, 700)
+    layer.build_summaries(sh.k_shared)
+    outs = []
+    for _ in range(2):
+        layer.step(q, sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, un.kv_start, un.kv_len)
+        torch.cuda.synchronize()
+        outs.append((layer.out.clone(), layer.seg_entries.clone(), layer.o_part.clone()))
+    for a, b in zip(outs[0], outs[1]):
+        assert torch.equal(a, b)
+
+
+def test_reduced_configs_every_element():
+    """The five workloads at reduced batch / corpus size, every output element checked."""
+    run_case(W.scaled(W.CONFIGS[1], B=12, C=32, unique_len=1000))
+    run_case(W.scaled(W.CONFIGS[2], B=24, C=64, k=8, unique_len=777))
+    run_case(W.scaled(W.CONFIGS[3], B=20, C=8, k=8, unique_len=300))
+    lens = np.random.default_rng(0).integers(100, 3000, size=20)
+    run_case(W.scaled(W.CONFIGS[4], B=20, C=48, k=8, unique_len=0, unique_len_max=0), lengths=lens,
+             two_streams=True)
+
+
+def _sample(w, n):
+    return np.sort(np.random.default_rng(7).choice(w.B, size=min(n, w.B), replace=False))
+
+
+def test_full_cfg1_sampled():
+    w = W.CONFIGS[1]
+    run_case(w, sample=_sample(w, 6))
+
+
+def test_full_cfg2_sampled():
+    w = W.CONFIGS[2]
+    run_case(w, sample=_sample(w, 4), check_baseline=False)
+
+
+def test_full_cfg3_dense_sampled():
+    w = W.CONFIGS[3]
+    run_case(w, sample=_sample(w, 2), check_baseline=False)
+
+
+def test_full_cfg4_sampled_steps():
+    w = W.CONFIGS[4]
+    free, _ = torch.cuda.mem_get_info()
+    if free < 110e9:
+        pytest.skip("not enough free device memory for the 71 GB ragged unique store")
+    for step in (0, w.steps - 1):
+        run_case(w, sample=_sample(w, 3), check_baseline=False, step=step, two_streams=True)
+        torch.cuda.empty_cache()
