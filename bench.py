@@ -1,0 +1,440 @@
+#!/usr/bin/env python
+"""Benchmark of the MoSKA decode-attention hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config I] [--impl reference]
+
+One step = one decode step of one attention layer over one batch of synthetic requests:
+route -> group -> shared attention || unique attention -> merge, through the C ABI.  Prints ONE
+JSON line (rank 0).  With N > 1 (torchrun) every rank runs the same workload on its own batch of
+requests against its own copy of the shared store (no data-path collective; weak scaling).
+
+`--impl reference` times the fp64 CPU oracle on the host cores instead (bounded sample per step).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2511_06010_b200 import distributed as DD
+from paper_2511_06010_b200 import workloads as W
+
+METRIC = "decode_queries_per_s_per_layer"
+UNIT = "queries/s"
+L2_BYTES = 126e6
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from ncu captures of the same kernels
+# (summaries under profiles/).  Keyed by (kernel, workload name).
+NCU_TRAFFIC_BYTES = {}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                smax.append(float(r[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+def algorithmic_work(w: W.Workload, lens: np.ndarray, n_unique_splits: int, shared_slots: int,
+                     touched_segments: int):
+    """Bytes and flops the method must move/compute per step (no padding, no re-reads)."""
+    rows = w.B * w.Hq
+    P = w.B * w.Hkv * w.k
+    unique_bytes = int(lens.sum()) * w.Hkv * 4 * w.D + rows * w.D * 2 + rows * n_unique_splits * (w.D + 1) * 4
+    shared_flops = P * w.G * w.L * 4 * w.D
+    shared_bytes = touched_segments * 4 * w.D * w.L + rows * w.D * 2 + rows * shared_slots * (w.D + 1) * 4
+    gemv_bytes = P * 4 * w.D * w.L + rows * w.D * 2 + rows * shared_slots * (w.D + 1) * 4
+    return dict(unique_bytes=unique_bytes, shared_flops=shared_flops, shared_bytes=shared_bytes,
+                gemv_bytes=gemv_bytes)
+
+
+def time_events(fn, iters: int, flush=None):
+    """Average milliseconds of fn() on the current stream, CUDA events, optional L2 flush between."""
+    total = 0.0
+    for _ in range(iters):
+        if flush is not None:
+            flush()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        b.synchronize()
+        total += a.elapsed_time(b)
+    return total / iters
+
+
+def cpu_oracle_step(w, sh_host, un_host, q_host, kv_len, summ_ref, sample):
+    """One oracle decode step (route + group + attention by definition) for the sampled requests."""
+    from oracle import oracle as O
+
+    qs = q_host[sample]
+    scale = 1.0 / float(np.sqrt(w.D))
+    if w.dense:
+        topk = np.tile(np.arange(w.C, dtype=np.int32), (len(sample), w.Hkv, 1))
+    else:
+        topk, _ = O.route(qs, summ_ref, w.k)
+        O.group_by_chunk(topk, w.C, fast=True)
+    out, _ = O.attend_direct(qs, sh_host[0], sh_host[1], un_host[0], un_host[1],
+                             un_host[2][sample], kv_len[sample], topk, scale)
+    return out
+
+
+def run_reference(args, w):
+    """The CPU oracle as the reference arm: each step is a bounded sample of the workload."""
+    rank, _, world = DD.env_world()
+    if rank != 0:
+        return
+    from oracle import oracle as O
+
+    O.build()
+    n_sample = min(w.B, args.ref_sample)
+    ws = W.scaled(w, B=n_sample)
+    sh = W.make_shared_store(ws, "cpu")
+    un = W.make_unique_store(ws, "cpu")
+    q = W.make_queries(ws, sh, 0, "cpu")
+    summ = None if w.dense else O.chunk_summaries(sh.k_shared)
+    sample = np.arange(n_sample)
+    kv_len = un.kv_len.numpy()
+    host = ((sh.k_shared, sh.v_shared), (un.k_unique, un.v_unique, un.kv_start.numpy()))
+    for _ in range(args.warmup):
+        cpu_oracle_step(ws, host[0], host[1], q, kv_len, summ, sample)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        cpu_oracle_step(ws, host[0], host[1], q, kv_len, summ, sample)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = n_sample / dt
+    sample_txt = f"first {n_sample} of {w.B} requests per step, all heads, full context per request"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": {"workload": w.name, "batch": w.B, "sample": sample_txt},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+                         "sample": sample_txt},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+def run_cuda(args, w):
+    rank, local_rank, world = DD.init("nccl")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    from paper_2511_06010_b200 import build as B
+
+    if rank == 0:
+        B.build()
+    DD.barrier()
+    from paper_2511_06010_b200 import binding as M
+    from paper_2511_06010_b200.engine import MoskaLayer
+
+    # every rank: its own request batch (seed offset), its own copy of the shared store
+    wr = W.scaled(w, seed=w.seed + 7919 * rank) if world > 1 else w
+    free, _ = torch.cuda.mem_get_info()
+    lens0 = W.unique_lengths(wr)
+    need = (2 * w.Hkv * w.C * w.L * w.D + 2 * int((lens0 + w.steps).sum()) * w.Hkv * w.D) * 2
+    if need * 1.15 > free:
+        raise SystemExit(f"workload {w.name} needs {need/1e9:.1f} GB, only {free/1e9:.1f} GB free")
+    sh = W.make_shared_store(wr, dev)
+    un = W.make_unique_store(wr, dev)
+    n_q = max(1, w.steps)
+    qs = [W.make_queries(wr, sh, s, dev) for s in range(n_q)]
+    kv_lens = [(un.kv_len + s).to(torch.int32) for s in range(n_q)]
+    max_len = int(lens0.max()) + w.steps
+    layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, max_len, dense=w.dense)
+    S = layer.shape
+    if not w.dense:
+        layer.build_summaries(sh.k_shared)
+    torch.cuda.synchronize()
+
+    two_streams = not args.one_stream
+    input_bytes = (sh.k_shared.numel() + un.k_unique.numel()) * 4
+    flush_buf = None
+    if input_bytes < 2 * L2_BYTES:
+        flush_buf = torch.empty(int(3 * L2_BYTES), dtype=torch.uint8, device=dev)
+    flush = (lambda: flush_buf.fill_(1)) if flush_buf is not None else None
+
+    def step(i, prof=None):
+        s = i % n_q
+        layer.step(qs[s], sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, un.kv_start,
+                   kv_lens[s], two_streams=two_streams, prof=prof)
+
+    for i in range(max(3, args.warmup)):
+        step(i)
+    torch.cuda.synchronize()
+
+    prof = M.profiler_create(args.steps)
+    sampler = ClockSampler(local_rank)
+    DD.barrier()
+    torch.cuda.synchronize()
+    sampler.start()
+    if flush is None:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(args.steps):
+            step(i, prof)
+        e1.record()
+        torch.cuda.synchronize()
+        total_ms = e0.elapsed_time(e1)
+    else:
+        total_ms = 0.0
+        for i in range(args.steps):
+            flush()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            step(i, prof)
+            e1.record()
+            e1.synchronize()
+            total_ms += e0.elapsed_time(e1)
+    DD.barrier()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    stage_ms, n_rec = M.profiler_read(prof)
+    M.profiler_destroy(prof)
+    stage_ms = {k: v / max(1, n_rec) for k, v in stage_ms.items()}
+    ms_per_step = total_ms / args.steps
+    value, ms_max = DD.whole_job_throughput(w.B * args.steps, total_ms, dev)
+    ms_per_step_max = ms_max / args.steps
+
+    # ---- end to end through the host-buffer entry point (pinned q in, out back, every step)
+    q_host = [q.cpu().pin_memory() for q in qs]
+    out_host = torch.empty(w.B, w.Hq, w.D, dtype=torch.bfloat16).pin_memory()
+    q_dev = torch.empty_like(qs[0])
+    for i in range(3):
+        layer.step_host(q_host[i % n_q], q_dev, out_host, sh.k_shared, sh.v_shared, un.k_unique,
+                        un.v_unique, un.kv_start, kv_lens[i % n_q], two_streams=two_streams)
+    DD.barrier()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(args.steps):
+        if flush is not None:
+            flush()
+        layer.step_host(q_host[i % n_q], q_dev, out_host, sh.k_shared, sh.v_shared, un.k_unique,
+                        un.v_unique, un.kv_start, kv_lens[i % n_q], two_streams=two_streams)
+    e1.record()
+    torch.cuda.synchronize()
+    e2e_ms = e0.elapsed_time(e1)
+    e2e_value, _ = DD.whole_job_throughput(w.B * args.steps, e2e_ms, dev)
+    io_bytes = w.B * w.Hq * w.D * 2
+
+    if rank != 0:
+        DD.finalize()
+        return
+
+    # ---- per-kernel detail (rank 0, outside the timed region)
+    peaks = measured_peaks()
+    lens = kv_lens[0].cpu().numpy().astype(np.int64)
+    if w.dense:
+        touched, P = w.Hkv * w.C, w.B * w.Hkv * w.C
+    else:
+        off = layer.seg_offsets.cpu().numpy()
+        touched, P = int((np.diff(off) > 0).sum()), w.B * w.Hkv * w.k
+    work = algorithmic_work(w, lens, S.n_unique_splits, S.shared_slots, touched)
+    iters = max(3, min(args.steps, 10))
+    gemv_ms = None
+    if not args.no_baseline:
+        big = w.dense and w.B * w.C > 20000   # 256 GiB of re-reads in the dense config: sample it
+        if big:
+            sub = MoskaLayer(8, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, max_len, dense=True,
+                             dense_slots=S.shared_slots)
+            qsub = qs[0][:8].contiguous()
+            gemv_ms = time_events(lambda: sub.gemv_baseline(qsub, sh.k_shared, sh.v_shared), 3) * (w.B / 8)
+        else:
+            layer.gemv_baseline(qs[0], sh.k_shared, sh.v_shared)
+            gemv_ms = time_events(lambda: layer.gemv_baseline(qs[0], sh.k_shared, sh.v_shared), iters, flush)
+    # every kernel alone on the GPU (same inputs, after the timed region): separates a kernel's own
+    # speed from the bandwidth and SM sharing of the two overlapped streams
+    iso = {}
+    if not w.dense:
+        iso["route"] = time_events(lambda: layer.route(qs[0]), iters, flush)
+        iso["group"] = time_events(lambda: layer.group(), iters, flush)
+    iso["shared"] = time_events(lambda: layer.shared(qs[0], sh.k_shared, sh.v_shared), iters, flush)
+    iso["unique"] = time_events(lambda: layer.unique(qs[0], un.k_unique, un.v_unique, un.kv_start,
+                                                     kv_lens[0]), iters, flush)
+    iso["merge"] = time_events(lambda: layer.merge(), iters, flush)
+    shared_ms, unique_ms = stage_ms["shared"], stage_ms["unique"]
+    shared_tflops = work["shared_flops"] / (shared_ms * 1e-3) / 1e12 if shared_ms > 0 else None
+    unique_gbs = work["unique_bytes"] / (unique_ms * 1e-3) / 1e9 if unique_ms > 0 else None
+    shared_gbs = work["shared_bytes"] / (shared_ms * 1e-3) / 1e9 if shared_ms > 0 else None
+
+    # dominant kernel and the roofline that bounds it
+    t_flops = work["shared_flops"] / (peaks["bf16_tflops_sustained"] * 1e12)
+    t_bytes = work["shared_bytes"] / (peaks["hbm_gbs"] * 1e9)
+    if unique_ms >= shared_ms:
+        kernel = "unique_attn_kernel"
+        roof = dict(bound="hbm", achieved=unique_gbs, peak=peaks["hbm_gbs"], unit="GB/s")
+    elif t_flops > t_bytes:
+        kernel = "shared_attn"
+        roof = dict(bound="tensor", achieved=shared_tflops, peak=peaks["bf16_tflops_sustained"],
+                    unit="TFLOP/s")
+    else:
+        kernel = "shared_attn"
+        roof = dict(bound="hbm", achieved=shared_gbs, peak=peaks["hbm_gbs"], unit="GB/s")
+    roof["frac"] = roof["achieved"] / roof["peak"] if roof["achieved"] else None
+    roof["traffic"] = NCU_TRAFFIC_BYTES.get((kernel, w.name))
+    roof["kernel"] = kernel
+    roof["peak_source"] = "of " + peaks["source"]
+    roof["avg_launch_ms"] = unique_ms if kernel.startswith("unique") else shared_ms
+
+    # ---- CPU baseline: the oracle as it stands on the host cores, bounded sample (N = 1 only)
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import oracle as O
+
+        O.build()
+        n_s = min(w.B, args.cpu_sample)
+        sample = np.arange(n_s)
+        qh = qs[0].cpu()
+        lens_s = kv_lens[0].cpu().numpy()
+        end = int((un.kv_start[n_s - 1] + un.capacity[n_s - 1]).item())
+        un_host = (un.k_unique[:end].cpu(), un.v_unique[:end].cpu(), un.kv_start.cpu().numpy())
+        sh_host = (sh.k_shared.cpu(), sh.v_shared.cpu())
+        summ = None if w.dense else O.chunk_summaries(sh_host[0])
+        t0 = time.perf_counter()
+        reps = 0
+        while True:
+            cpu_oracle_step(w, sh_host, un_host, qh, lens_s, summ, sample)
+            reps += 1
+            if time.perf_counter() - t0 > args.cpu_seconds or reps >= 50:
+                break
+        dt = (time.perf_counter() - t0) / reps
+        cpu = {"value": n_s / dt, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+               "sample": f"first {n_s} of {w.B} requests (all heads, full context), {reps} repeats, "
+                         f"{dt * reps:.1f} s"}
+
+    n_launch = (3 if w.dense else 8) * args.steps
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step_max, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {
+            "workload": w.name, "batch": w.B, "q_heads": w.Hq, "kv_heads": w.Hkv, "head_dim": w.D,
+            "shared_tokens": w.C * w.L, "chunk_tokens": w.L, "top_k": None if w.dense else w.k,
+            "unique_tokens_mean": float(lens.mean()), "n_unique_splits": S.n_unique_splits,
+            "shared_slots": S.shared_slots, "streams": 2 if two_streams else 1,
+            "l2": ("flushed between steps" if flush is not None
+                   else f"inputs exceed L2 ({input_bytes / 2**20:.0f} MiB of K/V per step)"),
+            "per_gpu": "own request batch, own copy of the shared store" if world > 1 else "single GPU",
+        },
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": io_bytes,
+                "d2h_bytes_per_step": io_bytes, "ms_per_step": e2e_ms / args.steps},
+        "gpu_launches": n_launch,
+        "roofline": roof,
+        "cpu_baseline": cpu,
+        "stage_ms": stage_ms,
+        "stage_ms_isolated": iso,
+        "isolated": {
+            "unique_gbs": work["unique_bytes"] / (iso["unique"] * 1e-3) / 1e9,
+            "unique_frac_of_measured_hbm": work["unique_bytes"] / (iso["unique"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+            "shared_tflops": work["shared_flops"] / (iso["shared"] * 1e-3) / 1e12,
+            "shared_gbs": work["shared_bytes"] / (iso["shared"] * 1e-3) / 1e9,
+        },
+        "shared": {"tflops": shared_tflops, "frac_of_measured_sustained": (shared_tflops or 0) / peaks["bf16_tflops_sustained"],
+                   "frac_of_nominal_2250": (shared_tflops or 0) / 2250.0, "gbs": shared_gbs,
+                   "frac_of_measured_hbm": (shared_gbs or 0) / peaks["hbm_gbs"],
+                   "touched_segments": touched, "pairs": P,
+                   "amortisation_factor": P / max(1, touched)},
+        "unique": {"gbs": unique_gbs, "frac_of_measured_hbm": (unique_gbs or 0) / peaks["hbm_gbs"],
+                   "frac_of_nominal_8000": (unique_gbs or 0) / 8000.0},
+        "gemv_baseline": None if gemv_ms is None else {
+            "ms": gemv_ms, "shared_speedup": gemv_ms / shared_ms if shared_ms > 0 else None,
+            "step_speedup": (ms_per_step - shared_ms + gemv_ms) / ms_per_step if not two_streams else None},
+    }
+    print(json.dumps(line), flush=True)
+    DD.finalize()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", type=int, default=1, help="workload index 0..4 (default 1)")
+    ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--one-stream", action="store_true", help="run unique attention on the main stream")
+    ap.add_argument("--no-baseline", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-sample", type=int, default=16, help="requests in the CPU-oracle sample")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0)
+    ap.add_argument("--ref-sample", type=int, default=8, help="requests per step of --impl reference")
+    args = ap.parse_args()
+    w = W.CONFIGS[args.config]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_cuda(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -66,6 +66,12 @@ typedef struct moska_shape {
 
 typedef void* moska_stream; /* a cudaStream_t */
 
+/* Optional per-stage device timing of moska_decode_step (CUDA events recorded on the stream each
+ * stage is launched on).  Stage order of the arrays below. */
+enum { MOSKA_STAGE_ROUTE = 0, MOSKA_STAGE_GROUP, MOSKA_STAGE_SHARED, MOSKA_STAGE_UNIQUE,
+       MOSKA_STAGE_MERGE, MOSKA_N_STAGES };
+typedef struct moska_profiler moska_profiler;
+
 /* Library version, major * 100 + minor. */
 int moska_version(void);
 
@@ -175,12 +181,24 @@ int moska_gemv_baseline(const uint16_t* q, const uint16_t* k_shared, const uint1
                         const int32_t* topk_idx, float* o_part, float* lse_part,
                         float softmax_scale, const moska_shape* shape, moska_stream stream);
 
+/* Creates a profiler able to hold `max_steps` recorded steps (host object owning CUDA events). */
+int moska_profiler_create(moska_profiler** out, int32_t max_steps);
+void moska_profiler_destroy(moska_profiler* prof);
+/* Waits for the recorded events, adds up the elapsed milliseconds per stage over the steps
+ * recorded since the last read into stage_ms[MOSKA_N_STAGES] (host), stores their number in
+ * *n_steps (host) and clears the profiler. */
+int moska_profiler_read(moska_profiler* prof, float* stage_ms, int32_t* n_steps);
+
 /*
- * One whole decode step on device buffers: route -> group -> shared || unique -> merge, in that
- * order on `stream` (shared and unique attention overlap on an internal second stream when
- * `side_stream` is not NULL).  Dense mode (no routing) when summaries == NULL.
+ * One whole decode step on device buffers: route -> group -> shared || unique -> merge.  Without
+ * `side_stream` everything runs in that order on `stream`.  With it, route/group/shared run on
+ * `side_stream` while unique attention runs beside them on `stream`; both are ordered after the
+ * work already on `stream`, and the merge follows both on `stream`.  Create `side_stream` with a
+ * HIGHER priority than `stream`, so that the short routing kernels are not queued behind the
+ * CTAs of the unique-attention stream.  Dense mode (no routing) when summaries == NULL.
  * Scratch buffers topk_idx [B*Hkv*k], seg_offsets [Hkv*C+1], seg_entries [B*Hkv*k], o_part,
- * lse_part and ws are caller-owned as in the individual calls.
+ * lse_part and ws are caller-owned as in the individual calls.  `prof` may be NULL; otherwise
+ * the step's stage boundaries are recorded into it (steps beyond its capacity are not recorded).
  */
 int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t* k_shared,
                       const uint16_t* v_shared, const uint16_t* k_unique,
@@ -188,7 +206,7 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
                       int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
                       float* o_part, float* lse_part, uint16_t* out, float* lse_out,
                       float softmax_scale, const moska_shape* shape, void* ws, size_t ws_bytes,
-                      moska_stream stream, moska_stream side_stream);
+                      moska_stream stream, moska_stream side_stream, moska_profiler* prof);
 
 /*
  * moska_decode_step for a caller whose step inputs live in HOST memory: copies q_host (bf16
@@ -202,7 +220,8 @@ int moska_decode_step_host(const uint16_t* q_host, uint16_t* q_dev, const float*
                            int32_t* seg_offsets, int32_t* seg_entries, float* o_part,
                            float* lse_part, uint16_t* out_dev, uint16_t* out_host,
                            float softmax_scale, const moska_shape* shape, void* ws,
-                           size_t ws_bytes, moska_stream stream, moska_stream side_stream);
+                           size_t ws_bytes, moska_stream stream, moska_stream side_stream,
+                           moska_profiler* prof);
 
 #ifdef __cplusplus
 }

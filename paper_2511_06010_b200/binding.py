@@ -52,8 +52,11 @@ EXPORTS = {
     "moska_unique_attn": (_i, [_vp] * 7 + [_f, _sp, _vp]),
     "moska_merge": (_i, [_vp] * 5 + [_sp, _vp]),
     "moska_gemv_baseline": (_i, [_vp] * 6 + [_f, _sp, _vp]),
-    "moska_decode_step": (_i, [_vp] * 15 + [_f, _sp, _vp, _sz, _vp, _vp]),
-    "moska_decode_step_host": (_i, [_vp] * 17 + [_f, _sp, _vp, _sz, _vp, _vp]),
+    "moska_decode_step": (_i, [_vp] * 15 + [_f, _sp, _vp, _sz, _vp, _vp, _vp]),
+    "moska_decode_step_host": (_i, [_vp] * 16 + [_f, _sp, _vp, _sz, _vp, _vp, _vp]),
+    "moska_profiler_create": (_i, [ctypes.POINTER(_vp), ctypes.c_int32]),
+    "moska_profiler_destroy": (None, [_vp]),
+    "moska_profiler_read": (_i, [_vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]),
 }
 for _name, (_res, _args) in EXPORTS.items():
     _fn = getattr(_lib, _name)
@@ -158,23 +161,46 @@ def gemv_baseline(q, k_shared, v_shared, topk_idx, o_part, lse_part, softmax_sca
 
 def decode_step(q, summaries, k_shared, v_shared, k_unique, v_unique, kv_start, kv_len, topk_idx,
                 seg_offsets, seg_entries, o_part, lse_part, out, lse_out, softmax_scale, s, ws,
-                stream=None, side_stream=None) -> None:
+                stream=None, side_stream=None, prof=None) -> None:
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check(_lib.moska_decode_step(
         _ptr(q), _ptr(summaries), _ptr(k_shared), _ptr(v_shared), _ptr(k_unique), _ptr(v_unique),
         _ptr(kv_start), _ptr(kv_len), _ptr(topk_idx), _ptr(seg_offsets), _ptr(seg_entries),
         _ptr(o_part), _ptr(lse_part), _ptr(out), _ptr(lse_out), softmax_scale, ctypes.byref(s),
         _ptr(ws), ws_bytes, _stream(stream),
-        None if side_stream is None else _stream(side_stream)), "moska_decode_step")
+        None if side_stream is None else _stream(side_stream), prof), "moska_decode_step")
 
 
 def decode_step_host(q_host, q_dev, summaries, k_shared, v_shared, k_unique, v_unique, kv_start,
                      kv_len, topk_idx, seg_offsets, seg_entries, o_part, lse_part, out_dev,
-                     out_host, softmax_scale, s, ws, stream=None, side_stream=None) -> None:
+                     out_host, softmax_scale, s, ws, stream=None, side_stream=None,
+                     prof=None) -> None:
     ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
     _check(_lib.moska_decode_step_host(
         _ptr(q_host), _ptr(q_dev), _ptr(summaries), _ptr(k_shared), _ptr(v_shared),
         _ptr(k_unique), _ptr(v_unique), _ptr(kv_start), _ptr(kv_len), _ptr(topk_idx),
         _ptr(seg_offsets), _ptr(seg_entries), _ptr(o_part), _ptr(lse_part), _ptr(out_dev),
         _ptr(out_host), softmax_scale, ctypes.byref(s), _ptr(ws), ws_bytes, _stream(stream),
-        None if side_stream is None else _stream(side_stream)), "moska_decode_step_host")
+        None if side_stream is None else _stream(side_stream), prof), "moska_decode_step_host")
+
+
+STAGES = ("route", "group", "shared", "unique", "merge")
+
+
+def profiler_create(max_steps: int):
+    """-> opaque profiler handle (pass as `prof=` to decode_step)."""
+    h = _vp()
+    _check(_lib.moska_profiler_create(ctypes.byref(h), max_steps), "moska_profiler_create")
+    return h
+
+
+def profiler_destroy(prof) -> None:
+    _lib.moska_profiler_destroy(prof)
+
+
+def profiler_read(prof):
+    """-> ({stage: summed milliseconds}, number of recorded steps); clears the profiler."""
+    ms = (ctypes.c_float * len(STAGES))()
+    n = ctypes.c_int32(0)
+    _check(_lib.moska_profiler_read(prof, ms, ctypes.byref(n)), "moska_profiler_read")
+    return {name: float(ms[i]) for i, name in enumerate(STAGES)}, int(n.value)

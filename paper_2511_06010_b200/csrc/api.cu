@@ -62,6 +62,24 @@ int check_device()
 
 using namespace moska;
 
+struct moska_profiler {
+    int max_steps = 0;
+    int n_steps = 0;
+    cudaEvent_t* ev = nullptr;  // [max_steps][MOSKA_N_STAGES][2]
+    bool* used = nullptr;       // [max_steps][MOSKA_N_STAGES]
+};
+
+namespace {
+// Records the begin/end event of one stage of the step being recorded (no-op without profiler).
+inline cudaError_t prof_mark(moska_profiler* p, int stage, int which, cudaStream_t st)
+{
+    if (p == nullptr || p->n_steps >= p->max_steps) return cudaSuccess;
+    const int i = p->n_steps * MOSKA_N_STAGES + stage;
+    p->used[i] = true;
+    return cudaEventRecord(p->ev[2 * i + which], st);
+}
+}  // namespace
+
 #define MOSKA_TRY(expr)              \
     do {                             \
         int st__ = (expr);           \
@@ -229,7 +247,7 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
                       int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
                       float* o_part, float* lse_part, uint16_t* out, float* lse_out,
                       float softmax_scale, const moska_shape* shape, void* ws, size_t ws_bytes,
-                      moska_stream stream, moska_stream side_stream)
+                      moska_stream stream, moska_stream side_stream, moska_profiler* prof)
 {
     const bool dense = summaries == nullptr;
     cudaStream_t st = (cudaStream_t)stream, side = (cudaStream_t)side_stream;
@@ -239,30 +257,91 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
         MOSKA_CUDA_TRY(cudaEventCreateWithFlags(&ev_fork, cudaEventDisableTiming));
         MOSKA_CUDA_TRY(cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming));
     }
-    // Unique attention depends on nothing upstream: start it first on the side stream.
+    // The routed chain (route -> group -> shared) goes to the side stream when there is one; the
+    // caller gives that stream the higher priority, so its short kernels are not queued behind
+    // the thousands of CTAs of the unique-attention stream that runs beside it on `stream`.
+    cudaStream_t cs = side != nullptr ? side : st;
     if (side != nullptr) {
         MOSKA_CUDA_TRY(cudaEventRecord(ev_fork, st));
         MOSKA_CUDA_TRY(cudaStreamWaitEvent(side, ev_fork, 0));
-        MOSKA_TRY(moska_unique_attn(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part,
-                                    softmax_scale, shape, side));
-        MOSKA_CUDA_TRY(cudaEventRecord(ev_join, side));
     }
     if (!dense) {
-        MOSKA_TRY(moska_route(q, summaries, topk_idx, nullptr, shape, st));
-        MOSKA_TRY(moska_group_by_chunk(topk_idx, seg_offsets, seg_entries, shape, ws, ws_bytes, st));
+        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 0, cs));
+        MOSKA_TRY(moska_route(q, summaries, topk_idx, nullptr, shape, cs));
+        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 1, cs));
+        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 0, cs));
+        MOSKA_TRY(moska_group_by_chunk(topk_idx, seg_offsets, seg_entries, shape, ws, ws_bytes, cs));
+        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 1, cs));
+        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 0, cs));
         MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, topk_idx, seg_offsets, seg_entries,
-                                    o_part, lse_part, softmax_scale, shape, ws, ws_bytes, st));
+                                    o_part, lse_part, softmax_scale, shape, ws, ws_bytes, cs));
+        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, cs));
     } else {
+        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 0, cs));
         MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, nullptr, nullptr, nullptr, o_part,
-                                    lse_part, softmax_scale, shape, ws, ws_bytes, st));
+                                    lse_part, softmax_scale, shape, ws, ws_bytes, cs));
+        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, cs));
     }
-    if (side != nullptr) {
-        MOSKA_CUDA_TRY(cudaStreamWaitEvent(st, ev_join, 0));
-    } else {
-        MOSKA_TRY(moska_unique_attn(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part,
-                                    softmax_scale, shape, st));
+    if (side != nullptr) MOSKA_CUDA_TRY(cudaEventRecord(ev_join, side));
+    MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 0, st));
+    MOSKA_TRY(moska_unique_attn(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part,
+                                softmax_scale, shape, st));
+    MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 1, st));
+    if (side != nullptr) MOSKA_CUDA_TRY(cudaStreamWaitEvent(st, ev_join, 0));
+    MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_MERGE, 0, st));
+    MOSKA_TRY(moska_merge(o_part, lse_part, out, nullptr, lse_out, shape, st));
+    MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_MERGE, 1, st));
+    if (prof != nullptr && prof->n_steps < prof->max_steps) ++prof->n_steps;
+    return MOSKA_OK;
+}
+
+int moska_profiler_create(moska_profiler** out, int32_t max_steps)
+{
+    if (out == nullptr || max_steps < 1) return fail(MOSKA_ERR_INVALID_ARG, "profiler arguments");
+    moska_profiler* p = new moska_profiler();
+    p->max_steps = max_steps;
+    const int n = max_steps * MOSKA_N_STAGES;
+    p->ev = new cudaEvent_t[2 * n];
+    p->used = new bool[n]();
+    for (int i = 0; i < 2 * n; ++i) {
+        cudaError_t e = cudaEventCreate(&p->ev[i]);
+        if (e != cudaSuccess) {
+            for (int j = 0; j < i; ++j) cudaEventDestroy(p->ev[j]);
+            delete[] p->ev;
+            delete[] p->used;
+            delete p;
+            return fail(MOSKA_ERR_CUDA, "cudaEventCreate failed: %s", cudaGetErrorString(e));
+        }
     }
-    return moska_merge(o_part, lse_part, out, nullptr, lse_out, shape, st);
+    *out = p;
+    return MOSKA_OK;
+}
+
+void moska_profiler_destroy(moska_profiler* p)
+{
+    if (p == nullptr) return;
+    for (int i = 0; i < 2 * p->max_steps * MOSKA_N_STAGES; ++i) cudaEventDestroy(p->ev[i]);
+    delete[] p->ev;
+    delete[] p->used;
+    delete p;
+}
+
+int moska_profiler_read(moska_profiler* p, float* stage_ms, int32_t* n_steps)
+{
+    if (p == nullptr || stage_ms == nullptr || n_steps == nullptr)
+        return fail(MOSKA_ERR_INVALID_ARG, "profiler arguments");
+    for (int s = 0; s < MOSKA_N_STAGES; ++s) stage_ms[s] = 0.f;
+    for (int i = 0; i < p->n_steps * MOSKA_N_STAGES; ++i) {
+        if (!p->used[i]) continue;
+        MOSKA_CUDA_TRY(cudaEventSynchronize(p->ev[2 * i + 1]));
+        float ms = 0.f;
+        MOSKA_CUDA_TRY(cudaEventElapsedTime(&ms, p->ev[2 * i], p->ev[2 * i + 1]));
+        stage_ms[i % MOSKA_N_STAGES] += ms;
+        p->used[i] = false;
+    }
+    *n_steps = p->n_steps;
+    p->n_steps = 0;
+    return MOSKA_OK;
 }
 
 int moska_decode_step_host(const uint16_t* q_host, uint16_t* q_dev, const float* summaries,
@@ -272,7 +351,8 @@ int moska_decode_step_host(const uint16_t* q_host, uint16_t* q_dev, const float*
                            int32_t* seg_offsets, int32_t* seg_entries, float* o_part,
                            float* lse_part, uint16_t* out_dev, uint16_t* out_host,
                            float softmax_scale, const moska_shape* shape, void* ws,
-                           size_t ws_bytes, moska_stream stream, moska_stream side_stream)
+                           size_t ws_bytes, moska_stream stream, moska_stream side_stream,
+                           moska_profiler* prof)
 {
     MOSKA_TRY(check_shape(shape, summaries != nullptr));
     if (q_host == nullptr || q_dev == nullptr || out_dev == nullptr || out_host == nullptr)
@@ -283,7 +363,7 @@ int moska_decode_step_host(const uint16_t* q_host, uint16_t* q_dev, const float*
     MOSKA_TRY(moska_decode_step(q_dev, summaries, k_shared, v_shared, k_unique, v_unique, kv_start,
                                 kv_len, topk_idx, seg_offsets, seg_entries, o_part, lse_part,
                                 out_dev, nullptr, softmax_scale, shape, ws, ws_bytes, stream,
-                                side_stream));
+                                side_stream, prof));
     MOSKA_CUDA_TRY(cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, st));
     MOSKA_CUDA_TRY(cudaStreamSynchronize(st));
     return MOSKA_OK;

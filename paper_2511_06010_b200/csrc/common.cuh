@@ -58,7 +58,7 @@ struct WsHeader {
 static_assert(sizeof(WsHeader) == 256, "header is one 256-byte block");
 
 struct WsLayout {
-    int32_t n_blocks;         // request blocks of the counting sort
+    int32_t words;            // 32-bit words of one key's request bit set
     int32_t n_keys;           // Hkv * C
     int32_t small_entries;    // requests per small tile
     int32_t big_entries;      // requests per big tile

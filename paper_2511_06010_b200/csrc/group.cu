@@ -2,12 +2,12 @@
 // routed (request, KV head, slot) positions by key = h * C + chunk, entirely on the device, plus
 // the tile work lists that shared attention walks.
 //
-// Stability without ordered atomics: the requests are cut into `n_blocks` consecutive blocks.
-// Pass 1 counts keys per block (atomic adds only accumulate counts, whose value does not depend
-// on order).  Pass 2 turns the per-block counts of each key into per-block start ranks and the
-// key totals.  Pass 3 scans the totals.  Pass 4 lets each block walk ITS requests in ascending
-// order; within one request all keys are distinct (a request routes to k different chunks per
-// head), so its threads bump different counters and no two writers race.
+// Determinism without ordered atomics: a request routes to k DIFFERENT chunks per KV head, so a
+// segment (h, c) holds each request at most once and is fully described by a bit set over the
+// requests.  Pass 1 sets bit b of row (h, c) for every routed pair (atomicOr: the result does
+// not depend on the order).  Pass 2 counts the bits per row, pass 3 scans the counts into
+// segment offsets and tile lists, pass 4 walks every row's bits in ascending request order and
+// writes the positions, looking the slot j up in the request's (ascending) chunk list.
 #include "common.cuh"
 
 namespace moska {
@@ -17,7 +17,7 @@ WsLayout ws_layout(const moska_shape* s)
     WsLayout w{};
     const int G = s->Hq / s->Hkv;
     w.n_keys = s->Hkv * s->C;
-    w.n_blocks = s->B < 64 ? (s->B > 0 ? s->B : 1) : 64;
+    w.words = (s->B + 31) / 32 > 0 ? (s->B + 31) / 32 : 1;
     w.small_entries = kSmallTileRows / G;
     w.big_entries = kBigTileRows / G;
     w.big_min_entries = 0x7fffffff;  // no tensor-core tiles unless enabled below
@@ -27,9 +27,9 @@ WsLayout ws_layout(const moska_shape* s)
     w.max_big = P / w.big_entries + segs;
     size_t off = sizeof(WsHeader);
     w.off_hist = off;
-    off += round_up(sizeof(int32_t) * (size_t)w.n_blocks * w.n_keys, 256);
+    off += round_up(sizeof(uint32_t) * (size_t)w.words * w.n_keys, 256);
     w.off_totals = off;
-    off += round_up(sizeof(int32_t) * 3 * (size_t)w.n_keys, 256);
+    off += round_up(sizeof(int32_t) * (size_t)w.n_keys, 256);
     w.off_small = off;
     off += round_up(sizeof(TileItem) * (size_t)w.max_small, 256);
     w.off_big = off;
@@ -40,46 +40,34 @@ WsLayout ws_layout(const moska_shape* s)
 
 namespace {
 
-__device__ __forceinline__ void block_range(int B, int n_blocks, int blk, int& b0, int& b1)
+// Pass 1: one thread per routed pair p = (b*Hkv + h)*k + j.
+__global__ void __launch_bounds__(256)
+group_mark_kernel(const int32_t* __restrict__ topk_idx, uint32_t* __restrict__ bitmap,
+                  WsHeader* __restrict__ hdr, long long P, int Hkv, int C, int k, int words)
 {
-    const int per = (B + n_blocks - 1) / n_blocks;
-    b0 = min(B, blk * per);
-    b1 = min(B, b0 + per);
+    const long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= P) return;
+    const int c = topk_idx[p];
+    if (c < 0 || c >= C) {  // corrupt routing: record it, touch nothing
+        atomicMin(&hdr->status, (int)MOSKA_ERR_INVALID_ARG);
+        return;
+    }
+    const int h = (int)((p / k) % Hkv);
+    const int b = (int)(p / ((long long)k * Hkv));
+    atomicOr(&bitmap[((size_t)h * C + c) * words + (b >> 5)], 1u << (b & 31));
 }
 
+// Pass 2: requests per key.
 __global__ void __launch_bounds__(256)
-group_count_kernel(const int32_t* __restrict__ topk_idx, int32_t* __restrict__ hist,
-                   WsHeader* __restrict__ hdr, int B, int Hkv, int C, int k, int n_keys)
-{
-    int b0, b1;
-    block_range(B, gridDim.x, blockIdx.x, b0, b1);
-    int32_t* my = hist + (size_t)blockIdx.x * n_keys;
-    const int per_req = Hkv * k;
-    for (int b = b0; b < b1; ++b)
-        for (int i = threadIdx.x; i < per_req; i += blockDim.x) {
-            const int c = topk_idx[(size_t)b * per_req + i];
-            if (c < 0 || c >= C) {  // corrupt routing: record it, touch nothing
-                atomicMin(&hdr->status, (int)MOSKA_ERR_INVALID_ARG);
-                continue;
-            }
-            atomicAdd(&my[(i / k) * C + c], 1);
-        }
-}
-
-// Per key: per-block counts -> per-block start ranks (in place), total count.
-__global__ void __launch_bounds__(256)
-group_colscan_kernel(int32_t* __restrict__ hist, int32_t* __restrict__ totals, int n_blocks,
-                     int n_keys)
+group_count_kernel(const uint32_t* __restrict__ bitmap, int32_t* __restrict__ totals, int n_keys,
+                   int words)
 {
     const int key = blockIdx.x * blockDim.x + threadIdx.x;
     if (key >= n_keys) return;
-    int run = 0;
-    for (int blk = 0; blk < n_blocks; ++blk) {
-        const int t = hist[(size_t)blk * n_keys + key];
-        hist[(size_t)blk * n_keys + key] = run;
-        run += t;
-    }
-    totals[key] = run;
+    const uint32_t* row = bitmap + (size_t)key * words;
+    int n = 0;
+    for (int w = 0; w < words; ++w) n += __popc(row[w]);
+    totals[key] = n;
 }
 
 // Exclusive scans over the keys, one CTA: entries -> seg_offsets; tiles -> work lists.
@@ -172,25 +160,44 @@ group_scan_kernel(const int32_t* __restrict__ totals, int32_t* __restrict__ seg_
     }
 }
 
+// Pass 4: one warp per key walks the key's request bits in ascending order.
 __global__ void __launch_bounds__(256)
-group_scatter_kernel(const int32_t* __restrict__ topk_idx, const int32_t* __restrict__ seg_offsets,
-                     int32_t* __restrict__ hist, int32_t* __restrict__ seg_entries, int B, int Hkv,
-                     int C, int k, int n_keys)
+group_emit_kernel(const int32_t* __restrict__ topk_idx, const uint32_t* __restrict__ bitmap,
+                  const int32_t* __restrict__ seg_offsets, int32_t* __restrict__ seg_entries,
+                  int n_keys, int Hkv, int C, int k, int words)
 {
-    int b0, b1;
-    block_range(B, gridDim.x, blockIdx.x, b0, b1);
-    int32_t* my = hist + (size_t)blockIdx.x * n_keys;
-    const int per_req = Hkv * k;
-    for (int b = b0; b < b1; ++b) {
-        for (int i = threadIdx.x; i < per_req; i += blockDim.x) {
-            const int c = topk_idx[(size_t)b * per_req + i];
-            if (c < 0 || c >= C) continue;
-            const int key = (i / k) * C + c;
-            const int rank = my[key];  // distinct keys within one request: no other writer now
-            my[key] = rank + 1;
-            seg_entries[seg_offsets[key] + rank] = b * per_req + i;
+    const int key = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (key >= n_keys) return;
+    const int begin = seg_offsets[key];
+    if (seg_offsets[key + 1] == begin) return;
+    const int h = key / C, c = key % C;
+    const uint32_t* row = bitmap + (size_t)key * words;
+    int rank0 = begin;
+    for (int w0 = 0; w0 < words; w0 += 32) {
+        const int w = w0 + lane;
+        uint32_t bits = w < words ? row[w] : 0u;
+        const int cnt = __popc(bits);
+        int inc = cnt;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int t = __shfl_up_sync(0xffffffffu, inc, off);
+            if (lane >= off) inc += t;
         }
-        __syncthreads();  // the next request may hit the same keys
+        int rank = rank0 + inc - cnt;
+        while (bits) {
+            const int b = w * 32 + (__ffs(bits) - 1);
+            bits &= bits - 1;
+            // slot j of chunk c in the ascending list topk_idx[b][h][0..k)
+            const int32_t* lst = topk_idx + ((size_t)b * Hkv + h) * k;
+            int lo = 0, hi = k - 1;
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (lst[mid] < c) lo = mid + 1; else hi = mid;
+            }
+            seg_entries[rank++] = (b * Hkv + h) * k + lo;
+        }
+        rank0 += __shfl_sync(0xffffffffu, inc, 31);
     }
 }
 
@@ -202,25 +209,27 @@ int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_ent
     const WsLayout lay = ws_layout(s);
     char* base = static_cast<char*>(ws);
     WsHeader* hdr = reinterpret_cast<WsHeader*>(base);
-    int32_t* hist = reinterpret_cast<int32_t*>(base + lay.off_hist);
+    uint32_t* bitmap = reinterpret_cast<uint32_t*>(base + lay.off_hist);
     int32_t* totals = reinterpret_cast<int32_t*>(base + lay.off_totals);
     TileItem* small_items = reinterpret_cast<TileItem*>(base + lay.off_small);
     TileItem* big_items = reinterpret_cast<TileItem*>(base + lay.off_big);
-    // header and histogram must start at zero
+    const long long P = (long long)s->B * s->Hkv * s->k;
+    // header and bit sets must start at zero
     MOSKA_CUDA_TRY(cudaMemsetAsync(base, 0, lay.off_totals, st));
-    group_count_kernel<<<lay.n_blocks, 256, 0, st>>>(topk_idx, hist, hdr, s->B, s->Hkv, s->C, s->k,
-                                                     lay.n_keys);
+    if (P > 0) {
+        group_mark_kernel<<<(unsigned)((P + 255) / 256), 256, 0, st>>>(topk_idx, bitmap, hdr, P,
+                                                                       s->Hkv, s->C, s->k, lay.words);
+        MOSKA_LAUNCH_CHECK("group_mark_kernel");
+    }
+    group_count_kernel<<<(lay.n_keys + 255) / 256, 256, 0, st>>>(bitmap, totals, lay.n_keys, lay.words);
     MOSKA_LAUNCH_CHECK("group_count_kernel");
-    group_colscan_kernel<<<(lay.n_keys + 255) / 256, 256, 0, st>>>(hist, totals, lay.n_blocks,
-                                                                   lay.n_keys);
-    MOSKA_LAUNCH_CHECK("group_colscan_kernel");
     group_scan_kernel<<<1, 1024, 0, st>>>(totals, seg_offsets, hdr, small_items, big_items,
                                           lay.n_keys, lay.small_entries, lay.big_entries,
                                           lay.big_min_entries);
     MOSKA_LAUNCH_CHECK("group_scan_kernel");
-    group_scatter_kernel<<<lay.n_blocks, 256, 0, st>>>(topk_idx, seg_offsets, hist, seg_entries,
-                                                       s->B, s->Hkv, s->C, s->k, lay.n_keys);
-    MOSKA_LAUNCH_CHECK("group_scatter_kernel");
+    group_emit_kernel<<<(lay.n_keys + 7) / 8, 256, 0, st>>>(topk_idx, bitmap, seg_offsets, seg_entries,
+                                                            lay.n_keys, s->Hkv, s->C, s->k, lay.words);
+    MOSKA_LAUNCH_CHECK("group_emit_kernel");
     return MOSKA_OK;
 }
 

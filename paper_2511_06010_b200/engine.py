@@ -71,23 +71,24 @@ class MoskaLayer:
         M.merge(self.o_part, self.lse_part, self.out, self.out_f32, self.lse_out, self.shape)
 
     # -- the whole step --------------------------------------------------------------------------
-    def step(self, q, k_shared, v_shared, k_unique, v_unique, kv_start, kv_len, two_streams=False):
+    def step(self, q, k_shared, v_shared, k_unique, v_unique, kv_start, kv_len, two_streams=False,
+             prof=None):
         if two_streams and self.side_stream is None:
-            self.side_stream = torch.cuda.Stream(device=self.device)
+            self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
         M.decode_step(q, None if self.dense else self.summaries, k_shared, v_shared, k_unique,
                       v_unique, kv_start, kv_len, self.topk_idx, self.seg_offsets,
                       self.seg_entries, self.o_part, self.lse_part, self.out, self.lse_out,
                       self.scale, self.shape, self.ws, None,
-                      self.side_stream if two_streams else None)
+                      self.side_stream if two_streams else None, prof)
         return self.out
 
     def step_host(self, q_host, q_dev, out_host, k_shared, v_shared, k_unique, v_unique,
-                  kv_start, kv_len, two_streams=False):
+                  kv_start, kv_len, two_streams=False, prof=None):
         if two_streams and self.side_stream is None:
-            self.side_stream = torch.cuda.Stream(device=self.device)
+            self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
         M.decode_step_host(q_host, q_dev, None if self.dense else self.summaries, k_shared,
                            v_shared, k_unique, v_unique, kv_start, kv_len, self.topk_idx,
                            self.seg_offsets, self.seg_entries, self.o_part, self.lse_part,
                            self.out, out_host, self.scale, self.shape, self.ws, None,
-                           self.side_stream if two_streams else None)
+                           self.side_stream if two_streams else None, prof)
         return out_host
