@@ -37,7 +37,10 @@ L2_BYTES = 126e6
 
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from ncu captures of the same kernels
 # (summaries under profiles/).  Keyed by (kernel, workload name).
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {
+    # profiles/unique_attn_kernel_cfg1.md: 1.0744 GB read + 7.5 MB written
+    ("unique_attn_kernel", "cfg1_llama8b_b64"): 1.0819e9,
+}
 
 
 def measured_peaks():
