@@ -125,6 +125,34 @@ int moska_group_by_chunk(const int32_t* topk_idx, int32_t* seg_offsets, int32_t*
                          const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream);
 
 /*
+ * moska_group_by_chunk for callers that cannot allocate device memory.  (The paper has no
+ * counterpart; this is a packaging variant of the call above.)
+ *
+ * Some hosts of this library may not call cudaMalloc at the point where they need the grouping:
+ * a serving engine that gave all device memory to its own pool at start-up and has no bytes left
+ * to carve a workspace from, or a latency-critical loop in which an allocation (which can
+ * synchronise the whole device) is not acceptable.  For them the scratch of the grouping passes
+ * lives in a fixed buffer of MOSKA_NOALLOC_SCRATCH_BYTES inside the library image; every GPU
+ * that loads the library keeps that buffer until the process exits.  The call allocates and
+ * frees nothing, neither directly nor through another library.
+ *
+ *   inputs / outputs      as moska_group_by_chunk (topk_idx in; seg_offsets, seg_entries out)
+ *   limit                 shapes whose grouping scratch (moska_workspace_bytes) exceeds the
+ *                         buffer are rejected with MOSKA_ERR_WORKSPACE before anything runs
+ *   first call            the first call on each device looks up the buffer's device address
+ *                         (with that device current); make it before any stream capture
+ *   shared state          all calls on a device use the same buffer and each call first clears
+ *                         what it needs zeroed, so calls in stream order are independent; calls
+ *                         that overlap on the GPU (different streams, no ordering) race
+ *   work lists            the tile lists for moska_shared_attn stay inside the buffer and are not
+ *                         exported; pair moska_shared_attn with moska_group_by_chunk instead
+ */
+#define MOSKA_NOALLOC_SCRATCH_BYTES (8u << 20)
+int moska_group_by_chunk_noalloc(const int32_t* topk_idx, int32_t* seg_offsets,
+                                 int32_t* seg_entries, const moska_shape* shape,
+                                 moska_stream stream);
+
+/*
  * Shared KV Attention (Section III-A, Fig. 2a): for every non-empty segment (h, c) the query rows
  * of all requests routed to chunk c form the rows of one Q matrix; S = scale * Q Kc^T, row-wise
  * softmax statistics and O = softmax(S) Vc are computed as one batched tensor-core product, so

@@ -48,6 +48,7 @@ EXPORTS = {
     "moska_build_chunk_summaries": (_i, [_vp, _vp, _sp, _vp]),
     "moska_route": (_i, [_vp, _vp, _vp, _vp, _sp, _vp]),
     "moska_group_by_chunk": (_i, [_vp, _vp, _vp, _sp, _vp, _sz, _vp]),
+    "moska_group_by_chunk_noalloc": (_i, [_vp, _vp, _vp, _sp, _vp]),
     "moska_shared_attn": (_i, [_vp] * 8 + [_f, _sp, _vp, _sz, _vp]),
     "moska_unique_attn": (_i, [_vp] * 7 + [_f, _sp, _vp]),
     "moska_merge": (_i, [_vp] * 5 + [_sp, _vp]),
@@ -129,6 +130,14 @@ def group_by_chunk(topk_idx, seg_offsets, seg_entries, s, ws, stream=None) -> No
     _check(_lib.moska_group_by_chunk(_ptr(topk_idx), _ptr(seg_offsets), _ptr(seg_entries),
                                      ctypes.byref(s), _ptr(ws), ws.numel() * ws.element_size(),
                                      _stream(stream)), "moska_group_by_chunk")
+
+
+def group_by_chunk_noalloc(topk_idx, seg_offsets, seg_entries, s, stream=None) -> None:
+    """Grouping with the library's built-in scratch buffer: for callers that must not allocate
+    device memory (no workspace argument; shapes beyond the buffer raise ERR_WORKSPACE)."""
+    _check(_lib.moska_group_by_chunk_noalloc(_ptr(topk_idx), _ptr(seg_offsets), _ptr(seg_entries),
+                                             ctypes.byref(s), _stream(stream)),
+           "moska_group_by_chunk_noalloc")
 
 
 def shared_attn(q, k_shared, v_shared, topk_idx, seg_offsets, seg_entries, o_part, lse_part,

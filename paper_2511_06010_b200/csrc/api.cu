@@ -160,6 +160,17 @@ int moska_group_by_chunk(const int32_t* topk_idx, int32_t* seg_offsets, int32_t*
     return launch_group(topk_idx, seg_offsets, seg_entries, shape, ws, (cudaStream_t)stream);
 }
 
+int moska_group_by_chunk_noalloc(const int32_t* topk_idx, int32_t* seg_offsets,
+                                 int32_t* seg_entries, const moska_shape* shape,
+                                 moska_stream stream)
+{
+    MOSKA_TRY(check_shape(shape, true));
+    REQUIRE_PTR(topk_idx, 4);
+    REQUIRE_PTR(seg_offsets, 4);
+    REQUIRE_PTR(seg_entries, 4);
+    return launch_group_noalloc(topk_idx, seg_offsets, seg_entries, shape, (cudaStream_t)stream);
+}
+
 int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
                       const int32_t* topk_idx, const int32_t* seg_offsets,
                       const int32_t* seg_entries, float* o_part, float* lse_part,

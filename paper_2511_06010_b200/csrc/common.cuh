@@ -31,6 +31,12 @@ int fail(int status, const char* fmt, ...);
                                  cudaGetErrorString(err__));                              \
     } while (0)
 
+#define MOSKA_TRY_STATUS(expr)                 \
+    do {                                       \
+        int st__ = (expr);                     \
+        if (st__ != MOSKA_OK) return st__;     \
+    } while (0)
+
 // Validates the shape fields every entry point relies on; returns MOSKA_OK or a negative status.
 int check_shape(const moska_shape* s, bool needs_k);
 // MOSKA_OK if the current device is compute capability 10.x.
@@ -78,6 +84,8 @@ int launch_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, f
                  const moska_shape* s, cudaStream_t st);
 int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
                  const moska_shape* s, void* ws, cudaStream_t st);
+int launch_group_noalloc(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
+                         const moska_shape* s, cudaStream_t st);
 int launch_shared_small(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
                         const int32_t* seg_entries, float* o_part, float* lse_part, float scale,
                         const moska_shape* s, void* ws, bool dense, cudaStream_t st);

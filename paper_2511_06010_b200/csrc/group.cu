@@ -8,6 +8,8 @@
 // not depend on the order).  Pass 2 counts the bits per row, pass 3 scans the counts into
 // segment offsets and tile lists, pass 4 walks every row's bits in ascending request order and
 // writes the positions, looking the slot j up in the request's (ascending) chunk list.
+#include <mutex>
+
 #include "common.cuh"
 
 namespace moska {
@@ -231,6 +233,48 @@ int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_ent
                                                             lay.n_keys, s->Hkv, s->C, s->k, lay.words);
     MOSKA_LAUNCH_CHECK("group_emit_kernel");
     return MOSKA_OK;
+}
+
+// ---- grouping without any caller- or library-side allocation -----------------------------------
+// Scratch for moska_group_by_chunk_noalloc lives in the library image itself: every GPU that
+// loads the library reserves these bytes until the process exits.
+static __device__ __align__(256) unsigned char g_noalloc_scratch[MOSKA_NOALLOC_SCRATCH_BYTES];
+
+int launch_group_noalloc(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
+                         const moska_shape* s, cudaStream_t st)
+{
+    const WsLayout lay = ws_layout(s);
+    if (lay.total > (size_t)MOSKA_NOALLOC_SCRATCH_BYTES)
+        return fail(MOSKA_ERR_WORKSPACE,
+                    "shape needs %zu bytes of grouping scratch, the built-in buffer holds %zu "
+                    "(use moska_group_by_chunk with a caller workspace)",
+                    lay.total, (size_t)MOSKA_NOALLOC_SCRATCH_BYTES);
+    MOSKA_TRY_STATUS(check_device());
+    // `g_noalloc_scratch` names a host-side handle here, not a device address; the address on
+    // the current device is looked up once per device and kept.
+    constexpr int kMaxDevices = 64;
+    static void* dev_ptr[kMaxDevices] = {nullptr};
+    static std::mutex mtx;
+    int dev = 0;
+    MOSKA_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices)
+        return fail(MOSKA_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
+    void* scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(mtx);
+        if (dev_ptr[dev] == nullptr) {
+            void* p = nullptr;
+            const cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+            if (e != cudaSuccess || p == nullptr)
+                return fail(MOSKA_ERR_CUDA, "cudaGetSymbolAddress(noalloc scratch) failed: %s",
+                            cudaGetErrorString(e));
+            dev_ptr[dev] = p;
+        }
+        scratch = dev_ptr[dev];
+    }
+    // launch_group clears the header and the bit sets itself, so the previous call's contents
+    // never leak into this one.
+    return launch_group(topk_idx, seg_offsets, seg_entries, s, scratch, st);
 }
 
 }  // namespace moska
