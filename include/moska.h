@@ -46,7 +46,8 @@ typedef enum moska_status {
     MOSKA_ERR_INVALID_ARG = -1, /* null pointer, k > C, Hq % Hkv != 0, misaligned pointer ...   */
     MOSKA_ERR_UNSUPPORTED = -2, /* D not in {64,128}, G > 8, L % 128 != 0, device is not sm_100 */
     MOSKA_ERR_WORKSPACE   = -3, /* workspace missing or smaller than moska_workspace_bytes()    */
-    MOSKA_ERR_CUDA        = -4  /* a CUDA runtime call or kernel launch failed                  */
+    MOSKA_ERR_CUDA        = -4, /* a CUDA runtime call or kernel launch failed                  */
+    MOSKA_ERR_TIMEOUT     = -5  /* device side: a bounded wait inside a kernel ran out          */
 } moska_status;
 
 /* Problem shape of one decode step of one layer. */
@@ -77,6 +78,12 @@ int moska_version(void);
 
 /* Text of the last error raised on the calling thread ("" if none). Host pointer, never NULL. */
 const char* moska_last_error(void);
+
+/* Waits for the current device to finish, stores the sticky device-side status word in
+ * *status_host (host pointer) and clears it.  0 means no kernel of the library raised anything;
+ * MOSKA_ERR_TIMEOUT means a CTA of the tensor-core Shared KV Attention kernel gave up on one of
+ * its bounded waits (TMA or MMA completion) and its outputs are not valid. */
+int moska_device_status(int32_t* status_host);
 
 /* n_slots = shared_slots + n_unique_splits; negative status if the shape is invalid. Host only. */
 int moska_partial_slots(const moska_shape* shape);

@@ -34,7 +34,7 @@ class MoskaError(RuntimeError):
         super().__init__(f"{where}: status {status}: {last_error()}")
 
 
-OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA = 0, -1, -2, -3, -4
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
 
 _vp, _sz, _f, _i = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_float, ctypes.c_int
 _sp = ctypes.POINTER(MoskaShape)
@@ -42,6 +42,7 @@ _sp = ctypes.POINTER(MoskaShape)
 EXPORTS = {
     "moska_version": (_i, []),
     "moska_last_error": (ctypes.c_char_p, []),
+    "moska_device_status": (_i, [ctypes.POINTER(ctypes.c_int32)]),
     "moska_partial_slots": (_i, [_sp]),
     "moska_workspace_bytes": (_sz, [_sp]),
     "moska_default_unique_splits": (_i, [ctypes.c_int32] * 3),
@@ -99,6 +100,13 @@ def version() -> int:
 
 def last_error() -> str:
     return _lib.moska_last_error().decode()
+
+
+def device_status() -> int:
+    """Synchronises the device; returns (and clears) the sticky device-side status word."""
+    v = ctypes.c_int32(0)
+    _check(_lib.moska_device_status(ctypes.byref(v)), "moska_device_status")
+    return v.value
 
 
 def partial_slots(s: MoskaShape) -> int:

@@ -197,8 +197,31 @@ int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_
     } else if (shape->shared_slots > shape->C) {
         return fail(MOSKA_ERR_INVALID_ARG, "dense mode needs shared_slots <= C");
     }
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool tc = shared_tc_supported(shape);
+    if (dense) {
+        // enough rows to fill a good part of a 128-row tile: tensor cores; else 16-row tiles
+        if (tc && (long long)shape->B * (shape->Hq / shape->Hkv) >= kBigMinRows)
+            return launch_shared_tc(q, k_shared, v_shared, nullptr, o_part, lse_part, softmax_scale,
+                                    shape, ws, true, st);
+        return launch_shared_small(q, k_shared, v_shared, nullptr, o_part, lse_part, softmax_scale,
+                                   shape, ws, true, st);
+    }
+    // routed: the grouping pass split every segment into tensor-core tiles and 16-row tiles
+    if (tc)
+        MOSKA_TRY(launch_shared_tc(q, k_shared, v_shared, seg_entries, o_part, lse_part,
+                                   softmax_scale, shape, ws, false, st));
     return launch_shared_small(q, k_shared, v_shared, seg_entries, o_part, lse_part, softmax_scale,
-                               shape, ws, dense, (cudaStream_t)stream);
+                               shape, ws, false, st);
+}
+
+int moska_device_status(int32_t* status_host)
+{
+    if (status_host == nullptr) return fail(MOSKA_ERR_INVALID_ARG, "status_host is NULL");
+    int v = 0;
+    MOSKA_TRY(read_tc_status(&v));
+    *status_host = v;
+    return MOSKA_OK;
 }
 
 int moska_unique_attn(const uint16_t* q, const uint16_t* k_unique, const uint16_t* v_unique,

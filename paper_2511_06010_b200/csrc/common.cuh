@@ -75,7 +75,8 @@ struct WsLayout {
 WsLayout ws_layout(const moska_shape* s);
 
 constexpr int kSmallTileRows = 16;  // query rows of one small tile (two 8-row MMA column blocks)
-constexpr int kBigTileRows = 128;   // query rows of one tensor-core (tcgen05) tile
+constexpr int kBigTileRows = 128;   // query rows of one tensor-core (tcgen05) tile; a work item has two
+constexpr int kBigMinRows = 40;     // fewer leftover rows of a segment than this go to small tiles
 
 // ---- internal launchers (one per .cu file) -----------------------------------------------------
 int launch_summaries(const uint16_t* k_shared, float* summaries, const moska_shape* s,
@@ -89,6 +90,14 @@ int launch_group_noalloc(const int32_t* topk_idx, int32_t* seg_offsets, int32_t*
 int launch_shared_small(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
                         const int32_t* seg_entries, float* o_part, float* lse_part, float scale,
                         const moska_shape* s, void* ws, bool dense, cudaStream_t st);
+// Tensor-core (tcgen05) Shared KV Attention over the big-tile work list (routed) or over
+// (KV head, run of chunks, 256 / G requests) items (dense).
+bool shared_tc_supported(const moska_shape* s);
+int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
+                     const int32_t* seg_entries, float* o_part, float* lse_part, float scale,
+                     const moska_shape* s, void* ws, bool dense, cudaStream_t st);
+// Synchronises the device, returns the sticky status of the tensor-core kernel and clears it.
+int read_tc_status(int* out);
 int launch_unique(const uint16_t* q, const uint16_t* k_unique, const uint16_t* v_unique,
                   const int64_t* kv_start, const int32_t* kv_len, float* o_part, float* lse_part,
                   float scale, const moska_shape* s, cudaStream_t st);

@@ -21,8 +21,8 @@ WsLayout ws_layout(const moska_shape* s)
     w.n_keys = s->Hkv * s->C;
     w.words = (s->B + 31) / 32 > 0 ? (s->B + 31) / 32 : 1;
     w.small_entries = kSmallTileRows / G;
-    w.big_entries = kBigTileRows / G;
-    w.big_min_entries = 0x7fffffff;  // no tensor-core tiles unless enabled below
+    w.big_entries = 2 * (kBigTileRows / G);  // a tensor-core work item holds two 128-row tiles
+    w.big_min_entries = shared_tc_supported(s) ? (kBigMinRows + G - 1) / G : 0x7fffffff;
     const int64_t P = (int64_t)s->B * s->Hkv * s->k;
     const int64_t segs = P < w.n_keys ? P : w.n_keys;  // non-empty segments at most
     w.max_small = P / w.small_entries + segs;

@@ -56,7 +56,7 @@ def _subproblem(q, topk, sh, un, kv_len, sample):
 
 
 def run_case(w: W.Workload, sample=None, lengths=None, n_unique_splits=None, step=0,
-             check_baseline=True, two_streams=False):
+             check_baseline=True, two_streams=False, dense_slots=None):
     """All stages of one decode step of workload `w` against the oracle."""
     M, MoskaLayer = _mods()
     dev = "cuda"
@@ -66,7 +66,7 @@ def run_case(w: W.Workload, sample=None, lengths=None, n_unique_splits=None, ste
     kv_len = (un.kv_len + step).to(torch.int32)
     max_len = int(kv_len.max().item()) if w.B else 1
     layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, max_len, dense=w.dense,
-                       n_unique_splits=n_unique_splits)
+                       n_unique_splits=n_unique_splits, dense_slots=dense_slots)
     S = layer.shape
     scale = layer.scale
     sample = np.arange(w.B) if sample is None else np.asarray(sample)
@@ -163,6 +163,7 @@ def run_case(w: W.Workload, sample=None, lengths=None, n_unique_splits=None, ste
     ref_out, ref_lse = O.attend_direct(q_s, ks, vs, ku, vu, st_s, len_s, topk_s, scale)
     report["out"] = PU.check_attention(out[sample].float().cpu().numpy(), ref_out, "decode step out")
     report["lse"] = PU.check_lse(layer.lse_out[sample].cpu().numpy(), ref_lse, "decode step lse")
+    assert M.device_status() == 0, "a bounded wait of the tensor-core kernel ran out"
     return report
 
 
@@ -247,6 +248,26 @@ def test_reduced_configs_every_element():
     lens = np.random.default_rng(0).integers(100, 3000, size=20)
     run_case(W.scaled(W.CONFIGS[4], B=20, C=48, k=8, unique_len=0, unique_len_max=0), lengths=lens,
              two_streams=True)
+
+
+def test_large_segments_take_the_tensor_core_tiles():
+    """Few chunks and many requests: segments of tens to hundreds of rows, i.e. full 128-row
+    tiles, partial second tiles and small remainders, for several GQA group sizes."""
+    for Hq, Hkv, B, C, k in ((8, 2, 96, 4, 2), (8, 2, 200, 4, 2), (16, 2, 70, 3, 2),
+                             (6, 2, 90, 4, 2), (2, 2, 300, 3, 1), (4, 2, 150, 5, 3)):
+        w = W.Workload("bigseg", B=B, Hq=Hq, Hkv=Hkv, D=128, C=C, L=256, k=k, unique_len=33,
+                       seed=11 + B)
+        run_case(w, n_unique_splits=1)
+
+
+def test_dense_tensor_core_tiles_and_empty_runs():
+    """Dense mode on the tensor-core kernel: one partial tile, two tiles with a partial second
+    one, several row tiles per (head, run), and a trailing run slot without chunks."""
+    base = W.Workload("dense", B=20, Hq=8, Hkv=2, D=128, C=6, L=256, k=6, unique_len=50, seed=21)
+    run_case(base, n_unique_splits=1)
+    run_case(W.scaled(base, B=40), n_unique_splits=1, dense_slots=2)
+    run_case(W.scaled(base, B=150, C=5, k=5), n_unique_splits=1, dense_slots=4)
+    run_case(W.scaled(base, B=70, Hq=16, C=3, k=3, L=512), n_unique_splits=2, dense_slots=1)
 
 
 def _sample(w, n):
