@@ -36,18 +36,23 @@ constexpr int kKvTile = 128;                   // tokens per K/V tile
 constexpr int kTileBytes = 128 * kD * 2;       // one Q, K or V tile in shared memory
 constexpr int kHalfBytes = kTileBytes / 2;     // 64 head-dimension columns of a tile
 constexpr int kStages = 4;                     // K/V ring slots
-constexpr int kThreads = 320;                  // 8 softmax warps + TMA warp + MMA warp
-constexpr int kLoadWarp = 8, kMmaWarp = 9;
+constexpr int kThreads = 384;                  // 8 softmax warps, TMA warp, MMA warp, 2 gather warps
+constexpr int kLoadWarp = 8, kMmaWarp = 9, kGatherWarp0 = 10;
+constexpr int kSoftmaxRegs = 208, kOtherRegs = 80;  // per-thread register budgets after set-up
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.f;       // log2 units a row maximum may lag behind
+// Of every kPolyPeriod pairs of score columns, kPolyPairs take exp2 as a polynomial on the FMA pipe.
+constexpr int kPolyPeriod = 2, kPolyPairs = 0;
 
 struct __align__(1024) TcSmem {
     uint8_t q[2][kTileBytes];
     uint8_t kv[kStages][kTileBytes];
     uint64_t full[kStages], empty[kStages];
-    uint64_t q_full[2], s_full[2], p_full[2], o_full[2];
-    long long row_r[2 * kBigTileRows];  // global query row b * Hq + hq of each tile row, -1 = padding
+    uint64_t q_full[2], q_free[2], s_full[2], p_full[2], o_full[2];
+    uint64_t x_full, x_free;      // split items: statistics of slot 1 published / O_1 read
+    float stat_m[kBigTileRows];   // split items: running maximum and sum of slot 1's rows
+    float stat_l[kBigTileRows];
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -61,7 +66,7 @@ struct TcParams {
     float* lse_part;
     int* status;
     float scale;
-    int B, Hq, Hkv, C, L, k, shared_slots, n_slots, dense;
+    int B, Hq, Hkv, C, L, k, shared_slots, n_slots, dense, n_items_dense;
 };
 
 __device__ int g_tc_status = 0;  // sticky: first negative status raised by a tensor-core CTA
@@ -73,9 +78,303 @@ __device__ __forceinline__ float fast_exp2(float x)
     return y;
 }
 
-__device__ __forceinline__ void group_barrier(int id)
+// ---- packed fp32 arithmetic (two lanes per instruction) -------------------------------------------
+__device__ __forceinline__ float2 ffma2(float2 a, float2 b, float2 c)
 {
-    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(128) : "memory");
+    float2 d;
+    asm("{\n"
+        ".reg .b64 ra, rb, rc, rd;\n"
+        "mov.b64 ra, {%2, %3};\n"
+        "mov.b64 rb, {%4, %5};\n"
+        "mov.b64 rc, {%6, %7};\n"
+        "fma.rn.f32x2 rd, ra, rb, rc;\n"
+        "mov.b64 {%0, %1}, rd;\n"
+        "}\n"
+        : "=f"(d.x), "=f"(d.y)
+        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y), "f"(c.x), "f"(c.y));
+    return d;
+}
+
+__device__ __forceinline__ float2 fadd2(float2 a, float2 b)
+{
+    float2 d;
+    asm("{\n"
+        ".reg .b64 ra, rb, rd;\n"
+        "mov.b64 ra, {%2, %3};\n"
+        "mov.b64 rb, {%4, %5};\n"
+        "add.rn.f32x2 rd, ra, rb;\n"
+        "mov.b64 {%0, %1}, rd;\n"
+        "}\n"
+        : "=f"(d.x), "=f"(d.y)
+        : "f"(a.x), "f"(a.y), "f"(b.x), "f"(b.y));
+    return d;
+}
+
+__device__ __forceinline__ float fmax3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// 2^x for two values on the FMA pipe instead of the special-function unit: round x to the nearest
+// integer n with the 1.5 * 2^23 trick, 2^(x - n) by a cubic with relative error 7.6e-5 on
+// [-0.5, 0.5], then n is added into the exponent field.  x is clamped at -125 (result ~ 2^-125).
+__device__ __forceinline__ float2 exp2_poly2(float2 x)
+{
+    const float kMagic = 12582912.f;  // 1.5 * 2^23
+    x.x = fmaxf(x.x, -125.f);
+    x.y = fmaxf(x.y, -125.f);
+    const float2 t = fadd2(x, make_float2(kMagic, kMagic));
+    const float2 n = fadd2(t, make_float2(-kMagic, -kMagic));
+    const float2 f = ffma2(n, make_float2(-1.f, -1.f), x);
+    float2 q = ffma2(f, make_float2(0.05521666631102562f, 0.05521666631102562f),
+                     make_float2(0.24261489510536194f, 0.24261489510536194f));
+    q = ffma2(q, f, make_float2(0.693252682685852f, 0.693252682685852f));
+    q = ffma2(q, f, make_float2(0.9999276399612427f, 0.9999276399612427f));
+    float2 r;
+    r.x = __int_as_float(__float_as_int(q.x) + (__float_as_int(t.x) << 23));
+    r.y = __int_as_float(__float_as_int(q.y) + (__float_as_int(t.y) << 23));
+    return r;
+}
+
+// One work item.  The CTA has two "slots" (t = 0, 1), each with its own S/P and O accumulator in
+// TMEM and its own softmax warp group.  An item with more than 128 rows runs its two query tiles
+// in the two slots over all K/V tiles.  An item with at most 128 rows is SPLIT: both slots hold
+// the same query tile, slot 0 takes the even and slot 1 the odd K/V tiles, and the two partial
+// softmax states are combined at the end -- so the tensor pipe always has two independent
+// dependency chains to alternate between.
+struct Item {
+    int h;            // KV head
+    int n_kv;         // K/V tiles of 128 tokens
+    int n_e[2];       // requests in query tile 0 / 1
+    int entry_begin;  // routed: first entry of the item in seg_entries
+    int b0;           // dense: first request of the item
+    int slot_dense;   // dense: partial slot (= run of chunks)
+    int split;        // 1: both slots work on query tile 0
+    int n_it[2];      // K/V tiles handled by slot 0 / 1
+    long long kv_row0;  // first token row of the item's K/V range in the [Hkv*C*L][D] store
+};
+
+__device__ __forceinline__ Item decode_item(const TcParams& p, int item, int G, int per_tile)
+{
+    Item it;
+    if (!p.dense) {
+        const int4 raw = __ldg(reinterpret_cast<const int4*>(p.items) + item);  // TileItem
+        it.h = raw.x / p.C;
+        it.entry_begin = raw.y;
+        it.n_e[0] = min(raw.z, per_tile);
+        it.n_e[1] = min(raw.z - it.n_e[0], per_tile);
+        it.kv_row0 = (long long)raw.x * p.L;
+        it.n_kv = p.L / kKvTile;
+        it.b0 = 0;
+        it.slot_dense = 0;
+    } else {
+        const int b_tiles = (p.B + 2 * per_tile - 1) / (2 * per_tile);
+        const int bt = item % b_tiles;
+        it.slot_dense = (item / b_tiles) % p.shared_slots;
+        it.h = item / (b_tiles * p.shared_slots);
+        const int run = (p.C + p.shared_slots - 1) / p.shared_slots;
+        const int c0 = min(p.C, it.slot_dense * run), c1 = min(p.C, c0 + run);
+        it.b0 = bt * 2 * per_tile;
+        it.n_e[0] = min(per_tile, p.B - it.b0);
+        it.n_e[1] = max(0, min(per_tile, p.B - it.b0 - per_tile));
+        it.kv_row0 = ((long long)it.h * p.C + c0) * p.L;
+        it.n_kv = (c1 - c0) * (p.L / kKvTile);
+        it.entry_begin = 0;
+    }
+    it.split = (it.n_e[1] == 0 && it.n_kv >= 2) ? 1 : 0;
+    if (it.split) {
+        it.n_it[0] = (it.n_kv + 1) >> 1;
+        it.n_it[1] = it.n_kv >> 1;
+    } else {
+        it.n_it[0] = it.n_kv;
+        it.n_it[1] = it.n_e[1] > 0 ? it.n_kv : 0;
+    }
+    return it;
+}
+
+// Roles of the third warp group (after it has given registers up): TMA producer, MMA issuer and
+// the two query-gather warps.
+__device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+                                         const TcParams& p, int n_items, int G, int per_tile,
+                                         uint32_t tmem, int warp, int lane)
+{
+    volatile int* ab = &sm.abort_flag;
+
+    if (warp == kLoadWarp) {
+        // =========================== TMA producer: K_0, V_0, K_1, V_1, ... =======================
+        if (lane == 0) {
+            uint32_t ld = 0;  // loads issued so far, over all items
+            bool ok = true;
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+                const Item it = decode_item(p, item, G, per_tile);
+                for (int x = 0; x < 2 * it.n_kv; ++x, ++ld) {
+                    const uint32_t s = ld % kStages;
+                    if (ld >= kStages && !mbar_wait(&sm.empty[s], ((ld / kStages) - 1) & 1, ab)) {
+                        ok = false;
+                        break;
+                    }
+                    mbar_arrive_expect_tx(&sm.full[s], kTileBytes);
+                    const CUtensorMap* tm = (x & 1) ? &tm_v : &tm_k;
+                    const int y = (int)(it.kv_row0 + (long long)(x >> 1) * kKvTile);
+                    tma_load_2d(sm.kv[s], tm, 0, y, &sm.full[s]);
+                    tma_load_2d(sm.kv[s] + kHalfBytes, tm, 64, y, &sm.full[s]);
+                }
+            }
+            if (*ab) {
+                // giving up: let the copies still in flight land before the CTA leaves
+                volatile int never = 0;
+                for (uint32_t x = ld > kStages ? ld - kStages : 0; x < ld; ++x)
+                    mbar_wait(&sm.full[x % kStages], (x / kStages) & 1, &never);
+            }
+        }
+        __syncwarp();
+    } else if (warp >= kGatherWarp0) {
+        // =========================== query gather of tile u ======================================
+        // Copies the tile's query rows into the 128-byte-swizzled K-major operand layout as soon
+        // as the MMAs of the previous item have stopped reading the buffer.
+        const int u = warp - kGatherWarp0;
+        uint32_t uses = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+            const Item it = decode_item(p, item, G, per_tile);
+            if (it.n_kv == 0 || it.n_e[u] == 0) continue;
+            long long rr[4];  // global query row of tile rows lane, lane + 32, lane + 64, lane + 96
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+                const int i = lane + 32 * m;
+                rr[m] = -1;
+                if (i < it.n_e[u] * G) {
+                    const int e = i / G, g = i % G;
+                    int b;
+                    if (!p.dense)
+                        b = __ldg(p.seg_entries + it.entry_begin + u * per_tile + e) / (p.k * p.Hkv);
+                    else
+                        b = it.b0 + u * per_tile + e;
+                    rr[m] = (long long)b * p.Hq + it.h * G + g;
+                }
+            }
+            if (uses > 0) {
+                ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_free[u], (uses - 1) & 1, ab));
+                if (!ok) break;
+            }
+            ++uses;
+            const uint32_t q_base = smem_u32(sm.q[u]);
+#pragma unroll
+            for (int m = 0; m < 4; ++m) {
+#pragma unroll 4
+                for (int n = 0; n < 16; ++n) {
+                    const int lr = 2 * n + (lane >> 4), c = lane & 15;
+                    const long long src_row = __shfl_sync(0xffffffffu, rr[m], lr);
+                    const int row = 32 * m + lr;
+                    const uint32_t dst = q_base + (c >> 3) * kHalfBytes + row * 128 + (((c & 7) ^ (row & 7)) << 4);
+                    const uint16_t* src = src_row >= 0 ? p.q + src_row * kD + c * 8 : p.q;
+                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src),
+                                 "r"(src_row >= 0 ? 16 : 0)
+                                 : "memory");
+                }
+            }
+            asm volatile("cp.async.wait_all;" ::: "memory");
+            fence_proxy_async_smem();
+            mbar_arrive(&sm.q_full[u]);
+        }
+    } else {
+        // =========================== MMA issuer ===================================================
+        if (lane == 0) {
+            const uint32_t id_qk = idesc_bf16_f32(128, kKvTile, false);
+            const uint32_t id_pv = idesc_bf16_f32(128, kD, true);
+            // Operand descriptors differ only in their start-address field (low word, units of 16
+            // bytes): build the constant parts once and add tile offsets per instruction, so that
+            // issuing an MMA costs a handful of integer instructions.
+            const uint64_t d_kmajor = smem_desc_sw128(0, 16, 1024);          // Q and K tiles
+            const uint64_t d_nmajor = smem_desc_sw128(0, kHalfBytes, 1024);  // V tiles
+            const uint32_t hi_k = static_cast<uint32_t>(d_kmajor >> 32);
+            const uint32_t hi_n = static_cast<uint32_t>(d_nmajor >> 32);
+            const uint32_t lo_q = static_cast<uint32_t>(d_kmajor) + (smem_u32(sm.q[0]) >> 4);
+            const uint32_t lo_k = static_cast<uint32_t>(d_kmajor) + (smem_u32(sm.kv[0]) >> 4);
+            const uint32_t lo_v = static_cast<uint32_t>(d_nmajor) + (smem_u32(sm.kv[0]) >> 4);
+            auto desc = [](uint32_t hi, uint32_t lo) { return (static_cast<uint64_t>(hi) << 32) | lo; };
+            // S_t = Q_u K^T, K in ring slot s: 8 steps of 16 head-dimension columns
+            auto issue_qk = [&](int tq, int u, uint32_t s) {
+                const uint32_t a = lo_q + u * (kTileBytes >> 4), b = lo_k + s * (kTileBytes >> 4);
+#pragma unroll
+                for (int ks = 0; ks < kD / 16; ++ks) {
+                    const uint32_t off = ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
+                    mma_ss(tmem + tq * 128, desc(hi_k, a + off), desc(hi_k, b + off), id_qk, ks > 0);
+                }
+            };
+            // O_t += P_t V, V in ring slot s: 8 steps of 16 tokens
+            auto issue_pv = [&](int tq, uint32_t s, bool acc) {
+                const uint32_t b = lo_v + s * (kTileBytes >> 4);
+#pragma unroll
+                for (int ks = 0; ks < kKvTile / 16; ++ks)
+                    mma_ts(tmem + 256 + tq * 128, tmem + tq * 128 + ks * 8,
+                           desc(hi_n, b + ks * (2048 >> 4)), id_pv, acc || ks > 0);
+            };
+            uint32_t ld0 = 0;               // ring position of the item's first load
+            uint32_t qc[2] = {0, 0}, pc[2] = {0, 0};
+            int q_reads[2] = {0, 0};        // score MMAs of the item that still have to read q[u]
+            auto issue_scores = [&](const Item& it, int tq, uint32_t s) {
+                const int u = it.split ? 0 : tq;
+                issue_qk(tq, u, s);
+                tc_commit(&sm.s_full[tq]);
+                if (--q_reads[u] == 0) tc_commit(&sm.q_free[u]);  // the gather warp may refill q[u]
+            };
+            bool ok = true;
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+                const Item it = decode_item(p, item, G, per_tile);
+                // K/V tile of slot tq's x-th step, and whether that slot is the tile's last reader
+                auto tile_of = [&](int tq, int x) { return it.split ? 2 * x + tq : x; };
+                auto last_reader = [&](int tq) { return it.split || it.n_it[1] == 0 || tq == 1; };
+                auto wait_load = [&](uint32_t g) {
+                    return mbar_wait(&sm.full[g % kStages], (g / kStages) & 1, ab);
+                };
+                q_reads[0] = it.n_kv;
+                q_reads[1] = it.n_e[1] > 0 ? it.n_kv : 0;
+                for (int u = 0; u < 2 && ok; ++u) {
+                    if (it.n_kv == 0 || it.n_e[u] == 0) continue;
+                    ok = mbar_wait(&sm.q_full[u], qc[u] & 1, ab);
+                    ++qc[u];
+                }
+                // first scores of both slots
+                for (int tq = 0; tq < 2 && ok; ++tq) {
+                    if (it.n_it[tq] == 0) continue;
+                    const uint32_t g = ld0 + 2 * tile_of(tq, 0);
+                    ok = wait_load(g);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    issue_scores(it, tq, g % kStages);
+                    if (last_reader(tq)) tc_commit(&sm.empty[g % kStages]);
+                }
+                for (int x = 0; x < it.n_it[0] && ok; ++x) {
+                    for (int tq = 0; tq < 2 && ok; ++tq) {
+                        if (x >= it.n_it[tq]) continue;
+                        const uint32_t gv = ld0 + 2 * tile_of(tq, x) + 1;
+                        ok = wait_load(gv) && mbar_wait(&sm.p_full[tq], pc[tq] & 1, ab);
+                        if (!ok) break;
+                        ++pc[tq];
+                        tc_fence_after_sync();
+                        issue_pv(tq, gv % kStages, x > 0);
+                        if (last_reader(tq)) tc_commit(&sm.empty[gv % kStages]);
+                        if (x + 1 < it.n_it[tq]) {
+                            const uint32_t gk = ld0 + 2 * tile_of(tq, x + 1);
+                            ok = wait_load(gk);
+                            if (!ok) break;
+                            tc_fence_after_sync();
+                            issue_scores(it, tq, gk % kStages);
+                            if (last_reader(tq)) tc_commit(&sm.empty[gk % kStages]);
+                        } else {
+                            tc_commit(&sm.o_full[tq]);
+                        }
+                    }
+                }
+                ld0 += 2 * it.n_kv;
+            }
+        }
+        __syncwarp();
+    }
+
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -88,60 +387,8 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = p.Hq / p.Hkv;
     const int per_tile = kBigTileRows / G;  // requests per query tile
-
-    // ---- the work item of this CTA (uniform over the CTA) --------------------------------------
-    int h, slot_dense = 0, entry_begin = 0, b0 = 0, n_e[2], n_kv_tiles;
-    long long kv_row0;
-    if (!p.dense) {
-        if ((int)blockIdx.x >= p.hdr->n_big_tiles) return;
-        const TileItem it = p.items[blockIdx.x];
-        h = it.key / p.C;
-        entry_begin = it.entry_begin;
-        n_e[0] = min(it.n_entries, per_tile);
-        n_e[1] = min(it.n_entries - n_e[0], per_tile);
-        kv_row0 = (long long)it.key * p.L;
-        n_kv_tiles = p.L / kKvTile;
-    } else {
-        const int b_tiles = (p.B + 2 * per_tile - 1) / (2 * per_tile);
-        const int bt = blockIdx.x % b_tiles;
-        slot_dense = (blockIdx.x / b_tiles) % p.shared_slots;
-        h = blockIdx.x / (b_tiles * p.shared_slots);
-        const int run = (p.C + p.shared_slots - 1) / p.shared_slots;
-        const int c0 = min(p.C, slot_dense * run), c1 = min(p.C, c0 + run);
-        b0 = bt * 2 * per_tile;
-        n_e[0] = min(per_tile, p.B - b0);
-        n_e[1] = max(0, min(per_tile, p.B - b0 - per_tile));
-        kv_row0 = ((long long)h * p.C + c0) * p.L;
-        n_kv_tiles = (c1 - c0) * (p.L / kKvTile);
-    }
-    const int nq = n_e[1] > 0 ? 2 : 1;
-
-    // Row owned by a softmax thread: tile t, tile row i.
-    const int t = warp >> 2;           // only meaningful for warps 0..7
-    const int i = tid & 127;
-    long long my_r = -1;
-    int my_slot = 0;
-    if (warp < 8 && i < n_e[t] * G) {
-        const int e = i / G, g = i % G;
-        int b;
-        if (!p.dense) {
-            const int pp = p.seg_entries[entry_begin + t * per_tile + e];
-            my_slot = pp % p.k;
-            b = pp / (p.k * p.Hkv);
-        } else {
-            my_slot = slot_dense;
-            b = b0 + t * per_tile + e;
-        }
-        my_r = (long long)b * p.Hq + h * G + g;
-    }
-    if (n_kv_tiles == 0) {  // dense mode: a trailing slot without chunks
-        if (my_r >= 0) {
-            float4* o = reinterpret_cast<float4*>(p.o_part + (my_r * p.n_slots + my_slot) * kD);
-            for (int d = 0; d < kD / 4; ++d) o[d] = make_float4(0.f, 0.f, 0.f, 0.f);
-            p.lse_part[my_r * p.n_slots + my_slot] = -INFINITY;
-        }
-        return;
-    }
+    const int n_items = p.dense ? p.n_items_dense : p.hdr->n_big_tiles;
+    if ((int)blockIdx.x >= n_items) return;
 
     // ---- set-up: barriers, tensor memory --------------------------------------------------------
     if (tid == 0) {
@@ -150,11 +397,14 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             mbar_init(&sm.empty[s], 1);
         }
         for (int u = 0; u < 2; ++u) {
-            mbar_init(&sm.q_full[u], 128);
+            mbar_init(&sm.q_full[u], 32);
+            mbar_init(&sm.q_free[u], 1);
             mbar_init(&sm.s_full[u], 1);
             mbar_init(&sm.p_full[u], 128);
             mbar_init(&sm.o_full[u], 1);
         }
+        mbar_init(&sm.x_full, 128);
+        mbar_init(&sm.x_free, 128);
         sm.abort_flag = 0;
         fence_mbar_init();
     }
@@ -174,42 +424,74 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     volatile int* ab = &sm.abort_flag;
 
     if (warp < 8) {
-        // =========================== softmax group of query tile t ==============================
-        if (n_e[t] > 0) {
-            sm.row_r[tid] = my_r;
-            group_barrier(1 + t);
-            // gather the tile's query rows into the 128-byte-swizzled K-major operand layout
-            for (int idx = i; idx < kBigTileRows * 16; idx += 128) {
-                const int row = idx >> 4, c = idx & 15;
-                const long long rr = sm.row_r[t * kBigTileRows + row];
-                uint4 val = make_uint4(0u, 0u, 0u, 0u);
-                if (rr >= 0) val = __ldg(reinterpret_cast<const uint4*>(p.q + rr * kD + c * 8));
-                uint8_t* dst = sm.q[t] + (c >> 3) * kHalfBytes + row * 128 + (((c & 7) ^ (row & 7)) << 4);
-                *reinterpret_cast<uint4*>(dst) = val;
-            }
-            fence_proxy_async_smem();
-            mbar_arrive(&sm.q_full[t]);
-
-            const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
-            const uint32_t t_s = tmem + lane_sel + t * 128;        // S_t, and P_t over its columns
-            const uint32_t t_o = tmem + lane_sel + 256 + t * 128;  // O_t
-            const float sl2 = p.scale * kLog2e;
-            float m_ref = -INFINITY, l_sum = 0.f;
-            bool alive = true;
-            for (int j = 0; j < n_kv_tiles; ++j) {
-                alive = __all_sync(0xffffffffu, mbar_wait(&sm.s_full[t], j & 1, ab));
-                if (!alive) break;
-                tc_fence_after_sync();
-                // pass 1: row maximum of this tile's scores
-                float mx = -INFINITY;
-#pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(t_s + c * 32, r);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int x = 0; x < 32; ++x) mx = fmaxf(mx, __uint_as_float(r[x]));
+        // =========================== softmax group of slot t =====================================
+        asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kSoftmaxRegs));
+        const int t = warp >> 2;
+        const int i = tid & 127;  // tile row = TMEM lane
+        const uint32_t lane_sel = static_cast<uint32_t>((warp & 3) * 32) << 16;
+        const uint32_t t_s = tmem + lane_sel + t * 128;        // S_t, and P_t over its columns
+        const uint32_t t_o = tmem + lane_sel + 256 + t * 128;  // O_t
+        const uint32_t t_o_other = tmem + lane_sel + 256 + (1 - t) * 128;
+        const float sl2 = p.scale * kLog2e;
+        uint32_t sc = 0, oc[2] = {0, 0}, xc = 0;  // barrier phases completed before this item
+        bool alive = true;
+        for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
+            const Item it = decode_item(p, item, G, per_tile);
+            const int n_it = it.n_it[t];
+            const int src = it.split ? 0 : t;  // query tile whose rows sit on this group's lanes
+            const uint32_t ph_o[2] = {oc[0] & 1u, oc[1] & 1u}, ph_x = xc & 1u;
+            oc[0] += it.n_it[0] > 0;
+            oc[1] += it.n_it[1] > 0;
+            xc += it.split;
+            long long my_r = -1;
+            int my_slot = 0;
+            if (i < it.n_e[src] * G) {
+                const int e = i / G, g = i % G;
+                int b;
+                if (!p.dense) {
+                    const int pp = __ldg(p.seg_entries + it.entry_begin + src * per_tile + e);
+                    my_slot = pp % p.k;
+                    b = pp / (p.k * p.Hkv);
+                } else {
+                    my_slot = it.slot_dense;
+                    b = it.b0 + src * per_tile + e;
                 }
+                my_r = (long long)b * p.Hq + it.h * G + g;
+            }
+            if (it.n_kv == 0) {  // dense mode: a trailing run without chunks
+                if (my_r >= 0) {
+                    float4* o = reinterpret_cast<float4*>(p.o_part + (my_r * p.n_slots + my_slot) * kD);
+                    for (int d = 0; d < kD / 4; ++d) o[d] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    p.lse_part[my_r * p.n_slots + my_slot] = -INFINITY;
+                }
+                continue;
+            }
+            float m_ref = -INFINITY, l_sum = 0.f;
+            for (int j = 0; j < n_it; ++j) {
+                alive = __all_sync(0xffffffffu, mbar_wait(&sm.s_full[t], sc & 1, ab));
+                if (!alive) break;
+                ++sc;
+                tc_fence_after_sync();
+                // the row's 128 scores: four loads in flight, one wait
+                uint32_t r[4][32];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) tmem_ld32(t_s + c * 32, r[c]);
+                tmem_ld_wait();
+                // eight independent maximum chains of three-input maxima, then a tree
+                float mxs[8];
+#pragma unroll
+                for (int x = 0; x < 8; ++x)
+                    mxs[x] = fmaxf(__uint_as_float(r[0][2 * x]), __uint_as_float(r[0][2 * x + 1]));
+#pragma unroll
+                for (int x = 8; x < 16; ++x)
+                    mxs[x & 7] = fmax3(mxs[x & 7], __uint_as_float(r[0][2 * x]), __uint_as_float(r[0][2 * x + 1]));
+#pragma unroll
+                for (int c = 1; c < 4; ++c)
+#pragma unroll
+                    for (int x = 0; x < 16; ++x)
+                        mxs[x & 7] = fmax3(mxs[x & 7], __uint_as_float(r[c][2 * x]), __uint_as_float(r[c][2 * x + 1]));
+                const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
+                                       fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
                 if (j == 0) {
                     m_ref = mx;
                 } else {
@@ -219,151 +501,111 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         const float alpha = need ? fast_exp2((m_ref - mx) * sl2) : 1.f;
                         if (need) m_ref = mx;
                         l_sum *= alpha;
-#pragma unroll
+#pragma unroll 1
                         for (int c = 0; c < 4; ++c) {
-                            uint32_t r[32];
-                            tmem_ld32(t_o + c * 32, r);
+                            uint32_t o_acc[32];
+                            tmem_ld32(t_o + c * 32, o_acc);
                             tmem_ld_wait();
 #pragma unroll
                             for (int x = 0; x < 32; ++x)
-                                r[x] = __float_as_uint(__uint_as_float(r[x]) * alpha);
-                            tmem_st32(t_o + c * 32, r);
+                                o_acc[x] = __float_as_uint(__uint_as_float(o_acc[x]) * alpha);
+                            tmem_st32(t_o + c * 32, o_acc);
                         }
                     }
                 }
-                // pass 2: P = exp2((S - m_ref) * scale * log2 e) as bf16 over the columns of S
-                const float mb = m_ref * sl2;
+                // P = exp2((S - m_ref) * scale * log2 e) as bf16, written over the columns of S
+                // Every other pair of columns takes its exponential on the FMA pipe, the rest on the
+                // special-function unit, so that neither pipe alone bounds the row.
+                const float2 sl2_2 = make_float2(sl2, sl2);
+                const float2 nmb_2 = make_float2(-m_ref * sl2, -m_ref * sl2);
+                float2 ls[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};  // partial row sums
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(t_s + c * 32, r);
-                    tmem_ld_wait();
                     uint32_t pk[16];
 #pragma unroll
                     for (int x = 0; x < 16; ++x) {
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(r[2 * x]), sl2, -mb));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(r[2 * x + 1]), sl2, -mb));
-                        l_sum += p0 + p1;
-                        __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
+                        const float2 e = ffma2(make_float2(__uint_as_float(r[c][2 * x]),
+                                                           __uint_as_float(r[c][2 * x + 1])),
+                                               sl2_2, nmb_2);
+                        float2 pr;
+                        if ((x % kPolyPeriod) < kPolyPairs) {
+                            pr = exp2_poly2(e);
+                        } else {
+                            pr.x = fast_exp2(e.x);
+                            pr.y = fast_exp2(e.y);
+                        }
+                        ls[x & 1] = fadd2(ls[x & 1], pr);
+                        __nv_bfloat162 b2 = __floats2bfloat162_rn(pr.x, pr.y);
                         pk[x] = *reinterpret_cast<uint32_t*>(&b2);
                     }
                     tmem_st16(t_s + c * 16, pk);
                 }
+                l_sum += (ls[0].x + ls[0].y) + (ls[1].x + ls[1].y);
                 tmem_st_wait();
                 tc_fence_before_sync();
                 mbar_arrive(&sm.p_full[t]);
             }
-            // epilogue: normalised partial output and log-sum-exp of the row
-            if (alive) alive = __all_sync(0xffffffffu, mbar_wait(&sm.o_full[t], 0, ab));
-            if (alive) {
-                tc_fence_after_sync();
-                const float inv = 1.f / l_sum;
-                float4* o = my_r >= 0
-                    ? reinterpret_cast<float4*>(p.o_part + (my_r * p.n_slots + my_slot) * kD)
-                    : nullptr;
+            if (!alive) break;
+
+            // ---- epilogue: normalised partial output and log-sum-exp of the row -----------------
+            if (it.split && t == 1) {
+                // publish this slot's statistics; slot 0's group combines and writes
+                sm.stat_m[i] = m_ref;
+                sm.stat_l[i] = l_sum;
+                mbar_arrive(&sm.x_full);
+                alive = __all_sync(0xffffffffu, mbar_wait(&sm.x_free, ph_x, ab));
+                continue;
+            }
+            if (n_it == 0) continue;  // slot 1 of an item with a single tile and a single K/V tile
+            alive = __all_sync(0xffffffffu, mbar_wait(&sm.o_full[t], ph_o[t], ab));
+            if (!alive) break;
+            float a_mine = 1.f, a_other = 0.f, m_all = m_ref, den = l_sum;
+            if (it.split) {
+                alive = __all_sync(0xffffffffu, mbar_wait(&sm.o_full[1], ph_o[1], ab)) &&
+                        __all_sync(0xffffffffu, mbar_wait(&sm.x_full, ph_x, ab));
+                if (!alive) break;
+                const float m1 = sm.stat_m[i], l1 = sm.stat_l[i];
+                m_all = fmaxf(m_ref, m1);
+                a_mine = fast_exp2((m_ref - m_all) * sl2);
+                a_other = fast_exp2((m1 - m_all) * sl2);
+                den = a_mine * l_sum + a_other * l1;
+            }
+            tc_fence_after_sync();
+            const float inv = 1.f / den;
+            a_mine *= inv;
+            a_other *= inv;
+            float4* o = my_r >= 0
+                ? reinterpret_cast<float4*>(p.o_part + (my_r * p.n_slots + my_slot) * kD)
+                : nullptr;
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t r[32];
-                    tmem_ld32(t_o + c * 32, r);
+            for (int c = 0; c < 4; ++c) {
+                uint32_t r[32];
+                tmem_ld32(t_o + c * 32, r);
+                tmem_ld_wait();
+                float v[32];
+#pragma unroll
+                for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(r[x]) * a_mine;
+                if (it.split) {
+                    tmem_ld32(t_o_other + c * 32, r);
                     tmem_ld_wait();
-                    if (o != nullptr) {
 #pragma unroll
-                        for (int x = 0; x < 8; ++x)
-                            o[c * 8 + x] = make_float4(__uint_as_float(r[4 * x]) * inv,
-                                                       __uint_as_float(r[4 * x + 1]) * inv,
-                                                       __uint_as_float(r[4 * x + 2]) * inv,
-                                                       __uint_as_float(r[4 * x + 3]) * inv);
-                    }
+                    for (int x = 0; x < 32; ++x) v[x] = fmaf(__uint_as_float(r[x]), a_other, v[x]);
                 }
-                if (my_r >= 0)
-                    p.lse_part[my_r * p.n_slots + my_slot] = m_ref * p.scale + logf(l_sum);
+                if (o != nullptr) {
+#pragma unroll
+                    for (int x = 0; x < 8; ++x)
+                        o[c * 8 + x] = make_float4(v[4 * x], v[4 * x + 1], v[4 * x + 2], v[4 * x + 3]);
+                }
+            }
+            if (my_r >= 0) p.lse_part[my_r * p.n_slots + my_slot] = m_all * p.scale + logf(den);
+            if (it.split) {
+                tc_fence_before_sync();
+                mbar_arrive(&sm.x_free);  // O_1 and the statistics may be overwritten
             }
         }
-    } else if (warp == kLoadWarp) {
-        // =========================== TMA producer: K_0, V_0, K_1, V_1, ... =======================
-        if (lane == 0) {
-            const int n_loads = 2 * n_kv_tiles;
-            int issued = 0;
-            for (int ld = 0; ld < n_loads; ++ld) {
-                const int s = ld % kStages;
-                if (ld >= kStages && !mbar_wait(&sm.empty[s], ((ld / kStages) - 1) & 1, ab)) break;
-                mbar_arrive_expect_tx(&sm.full[s], kTileBytes);
-                const CUtensorMap* tm = (ld & 1) ? &tm_v : &tm_k;
-                const int y = (int)(kv_row0 + (long long)(ld >> 1) * kKvTile);
-                tma_load_2d(sm.kv[s], tm, 0, y, &sm.full[s]);
-                tma_load_2d(sm.kv[s] + kHalfBytes, tm, 64, y, &sm.full[s]);
-                issued = ld + 1;
-            }
-            if (*ab) {
-                // giving up: let the copies still in flight land before the CTA leaves
-                volatile int never = 0;
-                for (int ld = max(0, issued - kStages); ld < issued; ++ld)
-                    mbar_wait(&sm.full[ld % kStages], (ld / kStages) & 1, &never);
-            }
-        }
-        __syncwarp();
     } else {
-        // =========================== MMA issuer ===================================================
-        if (lane == 0) {
-            const uint32_t id_qk = idesc_bf16_f32(128, kKvTile, false);
-            const uint32_t id_pv = idesc_bf16_f32(128, kD, true);
-            const uint32_t q_addr[2] = {smem_u32(sm.q[0]), smem_u32(sm.q[1])};
-            // S_t = Q_t K^T with K in ring slot s: 8 steps of 16 head-dimension columns
-            auto issue_qk = [&](int tq, int s) {
-                const uint32_t k_addr = smem_u32(sm.kv[s]);
-#pragma unroll
-                for (int ks = 0; ks < kD / 16; ++ks) {
-                    const uint32_t off = (ks >> 2) * kHalfBytes + (ks & 3) * 32;
-                    mma_ss(tmem + tq * 128, smem_desc_sw128(q_addr[tq] + off, 16, 1024),
-                           smem_desc_sw128(k_addr + off, 16, 1024), id_qk, ks > 0);
-                }
-            };
-            // O_t += P_t V with V in ring slot s: 8 steps of 16 tokens
-            auto issue_pv = [&](int tq, int s, bool acc) {
-                const uint32_t v_addr = smem_u32(sm.kv[s]);
-#pragma unroll
-                for (int ks = 0; ks < kKvTile / 16; ++ks)
-                    mma_ts(tmem + 256 + tq * 128, tmem + tq * 128 + ks * 8,
-                           smem_desc_sw128(v_addr + ks * 2048, kHalfBytes, 1024), id_pv,
-                           acc || ks > 0);
-            };
-            bool ok = true;
-            for (int tq = 0; tq < nq && ok; ++tq) ok = mbar_wait(&sm.q_full[tq], 0, ab);
-            if (ok) ok = mbar_wait(&sm.full[0], 0, ab);  // K_0
-            if (ok) {
-                tc_fence_after_sync();
-                for (int tq = 0; tq < nq; ++tq) {
-                    issue_qk(tq, 0);
-                    tc_commit(&sm.s_full[tq]);
-                }
-                tc_commit(&sm.empty[0]);
-            }
-            for (int j = 0; j < n_kv_tiles && ok; ++j) {
-                const int ld_v = 2 * j + 1, ld_k = 2 * j + 2;
-                const int s_v = ld_v % kStages, s_k = ld_k % kStages;
-                ok = mbar_wait(&sm.full[s_v], (ld_v / kStages) & 1, ab);
-                for (int tq = 0; tq < nq && ok; ++tq) {
-                    ok = mbar_wait(&sm.p_full[tq], j & 1, ab);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    issue_pv(tq, s_v, j > 0);
-                    if (tq == nq - 1) tc_commit(&sm.empty[s_v]);
-                    if (j + 1 < n_kv_tiles) {
-                        if (tq == 0) {
-                            ok = mbar_wait(&sm.full[s_k], (ld_k / kStages) & 1, ab);
-                            if (!ok) break;
-                            tc_fence_after_sync();
-                        }
-                        issue_qk(tq, s_k);
-                        tc_commit(&sm.s_full[tq]);
-                        if (tq == nq - 1) tc_commit(&sm.empty[s_k]);
-                    } else {
-                        tc_commit(&sm.o_full[tq]);
-                    }
-                }
-            }
-        }
-        __syncwarp();
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
+        other_roles(sm, tm_k, tm_v, p, n_items, G, per_tile, tmem, warp, lane);
     }
 
     // ---- teardown -------------------------------------------------------------------------------
@@ -424,10 +666,11 @@ int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t
 {
     const int G = s->Hq / s->Hkv;
     const int per_cta = 2 * (kBigTileRows / G);
-    long long grid;
+    long long grid;  // upper bound of the number of work items
     TcParams p{};
     if (dense) {
         grid = (long long)s->Hkv * s->shared_slots * ((s->B + per_cta - 1) / per_cta);
+        p.n_items_dense = (int)grid;
     } else {
         const WsLayout lay = ws_layout(s);
         grid = lay.max_big;
@@ -436,6 +679,11 @@ int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t
     }
     if (grid == 0) return MOSKA_OK;
     if (grid > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "shared attention grid too large");
+    // persistent CTAs, one per SM, each walking the item list with the grid as its stride
+    int dev = 0, n_sms = 0;
+    MOSKA_CUDA_TRY(cudaGetDevice(&dev));
+    MOSKA_CUDA_TRY(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
+    if (grid > n_sms) grid = n_sms;
     const long long kv_rows = (long long)s->Hkv * s->C * s->L;
     if (kv_rows > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "shared store exceeds 2^31 tokens");
     CUtensorMap tm_k, tm_v;

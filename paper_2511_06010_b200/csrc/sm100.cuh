@@ -63,15 +63,20 @@ constexpr uint64_t kWaitLimitNs = 2000000000ull;
 // common teardown.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag)
 {
-    if (mbar_try_wait(bar, parity)) return true;
-    const uint64_t t0 = global_timer_ns();
-    uint32_t polls = 0;
-    while (true) {
+    // Fast path: plain polling (each try_wait already suspends the thread for a short,
+    // hardware-defined time).  The abort flag and the clock are only looked at now and then:
+    // reading the global timer is slow and must stay off the critical path.
+    uint64_t t0 = 0;
+    for (uint32_t polls = 1;; ++polls) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if ((++polls & 63u) == 0u && global_timer_ns() - t0 > kWaitLimitNs) {
-            *abort_flag = 1;
-            return false;
+        if ((polls & 1023u) == 0u) {
+            if (*abort_flag) return false;
+            const uint64_t now = global_timer_ns();
+            if (t0 == 0) t0 = now;
+            if (now - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                return false;
+            }
         }
     }
 }
