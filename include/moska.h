@@ -225,12 +225,16 @@ void moska_profiler_destroy(moska_profiler* prof);
 int moska_profiler_read(moska_profiler* prof, float* stage_ms, int32_t* n_steps);
 
 /*
- * One whole decode step on device buffers: route -> group -> shared || unique -> merge.  Without
- * `side_stream` everything runs in that order on `stream`.  With it, route/group/shared run on
- * `side_stream` while unique attention runs beside them on `stream`; both are ordered after the
- * work already on `stream`, and the merge follows both on `stream`.  Create `side_stream` with a
- * HIGHER priority than `stream`, so that the short routing kernels are not queued behind the
- * CTAs of the unique-attention stream.  Dense mode (no routing) when summaries == NULL.
+ * One whole decode step on device buffers: route -> group -> unique -> shared -> merge.  Without
+ * `side_stream` everything runs in that order on `stream`.  With it, the short routing and
+ * grouping kernels run on `side_stream` beside unique attention; both are ordered after the work
+ * already on `stream`; shared attention and the merge follow on `stream` once both are done.
+ * Create `side_stream` with a HIGHER priority than `stream`, or the routing kernels queue behind
+ * the CTAs of unique attention.  The overlap pays while the router's shared-memory footprint
+ * (4 bytes per chunk and warp) is small; with thousands of chunks the SMs switch to a large
+ * shared-memory carve-out while both run, which leaves unique attention too little L1 for its
+ * loads in flight (measured: up to 40 % slower) -- pass side_stream = NULL then.
+ * Dense mode (no routing) when summaries == NULL.
  * Scratch buffers topk_idx [B*Hkv*k], seg_offsets [Hkv*C+1], seg_entries [B*Hkv*k], o_part,
  * lse_part and ws are caller-owned as in the individual calls.  `prof` may be NULL; otherwise
  * the step's stage boundaries are recorded into it (steps beyond its capacity are not recorded).

@@ -291,37 +291,38 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
         MOSKA_CUDA_TRY(cudaEventCreateWithFlags(&ev_fork, cudaEventDisableTiming));
         MOSKA_CUDA_TRY(cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming));
     }
-    // The routed chain (route -> group -> shared) goes to the side stream when there is one; the
-    // caller gives that stream the higher priority, so its short kernels are not queued behind
-    // the thousands of CTAs of the unique-attention stream that runs beside it on `stream`.
+    // Routing and grouping are short, latency-bound kernels: with a side stream they run beside
+    // unique attention (the caller gives that stream the higher priority, so they are not queued
+    // behind the thousands of CTAs of the unique-attention grid).  The two attention kernels each
+    // fill the GPU on their own (HBM-bound unique attention, tensor- or HBM-bound shared
+    // attention), so they run one after the other on `stream`.
     cudaStream_t cs = side != nullptr ? side : st;
-    if (side != nullptr) {
-        MOSKA_CUDA_TRY(cudaEventRecord(ev_fork, st));
-        MOSKA_CUDA_TRY(cudaStreamWaitEvent(side, ev_fork, 0));
-    }
     if (!dense) {
+        if (side != nullptr) {
+            MOSKA_CUDA_TRY(cudaEventRecord(ev_fork, st));
+            MOSKA_CUDA_TRY(cudaStreamWaitEvent(side, ev_fork, 0));
+        }
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 0, cs));
         MOSKA_TRY(moska_route(q, summaries, topk_idx, nullptr, shape, cs));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 1, cs));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 0, cs));
         MOSKA_TRY(moska_group_by_chunk(topk_idx, seg_offsets, seg_entries, shape, ws, ws_bytes, cs));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 1, cs));
-        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 0, cs));
-        MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, topk_idx, seg_offsets, seg_entries,
-                                    o_part, lse_part, softmax_scale, shape, ws, ws_bytes, cs));
-        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, cs));
-    } else {
-        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 0, cs));
-        MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, nullptr, nullptr, nullptr, o_part,
-                                    lse_part, softmax_scale, shape, ws, ws_bytes, cs));
-        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, cs));
+        if (side != nullptr) MOSKA_CUDA_TRY(cudaEventRecord(ev_join, side));
     }
-    if (side != nullptr) MOSKA_CUDA_TRY(cudaEventRecord(ev_join, side));
     MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 0, st));
     MOSKA_TRY(moska_unique_attn(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part,
                                 softmax_scale, shape, st));
     MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 1, st));
-    if (side != nullptr) MOSKA_CUDA_TRY(cudaStreamWaitEvent(st, ev_join, 0));
+    if (!dense && side != nullptr) MOSKA_CUDA_TRY(cudaStreamWaitEvent(st, ev_join, 0));
+    MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 0, st));
+    if (!dense)
+        MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, topk_idx, seg_offsets, seg_entries,
+                                    o_part, lse_part, softmax_scale, shape, ws, ws_bytes, st));
+    else
+        MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, nullptr, nullptr, nullptr, o_part,
+                                    lse_part, softmax_scale, shape, ws, ws_bytes, st));
+    MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, st));
     MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_MERGE, 0, st));
     MOSKA_TRY(moska_merge(o_part, lse_part, out, nullptr, lse_out, shape, st));
     MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_MERGE, 1, st));

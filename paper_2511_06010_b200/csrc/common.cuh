@@ -76,7 +76,10 @@ WsLayout ws_layout(const moska_shape* s);
 
 constexpr int kSmallTileRows = 16;  // query rows of one small tile (two 8-row MMA column blocks)
 constexpr int kBigTileRows = 128;   // query rows of one tensor-core (tcgen05) tile; a work item has two
-constexpr int kBigMinRows = 40;     // fewer leftover rows of a segment than this go to small tiles
+#ifndef MOSKA_BIG_MIN_ROWS
+#define MOSKA_BIG_MIN_ROWS 16
+#endif
+constexpr int kBigMinRows = MOSKA_BIG_MIN_ROWS;  // fewer leftover rows of a segment than this go to small tiles
 
 // ---- internal launchers (one per .cu file) -----------------------------------------------------
 int launch_summaries(const uint16_t* k_shared, float* summaries, const moska_shape* s,

@@ -117,44 +117,49 @@ shared_small_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
     __shared__ CombineSmem<D, NT> sm;
     const int G = Hq / Hkv;
     const int per_tile = kSmallTileRows / G;  // requests per tile
-    clear_rows(rows);
-    __syncthreads();
-    int64_t tok0;
-    int n_tok;
-    if (!dense) {
-        if ((int)blockIdx.x >= hdr->n_small_tiles) return;
-        const TileItem it = items[blockIdx.x];
-        const int h = it.key / C;
-        if (threadIdx.x < it.n_entries * G) {
-            const int p = seg_entries[it.entry_begin + threadIdx.x / G];
-            const int g = threadIdx.x % G;
-            const int j = p % k, b = p / (k * Hkv);
-            const int64_t r = (int64_t)b * Hq + h * G + g;
-            rows.q[threadIdx.x] = q + r * D;
-            rows.o[threadIdx.x] = o_part + (r * n_slots + j) * D;
-            rows.lse[threadIdx.x] = lse_part + r * n_slots + j;
+    // Routed mode: the CTAs walk the device-side tile list with the grid as their stride (the
+    // host only knows an upper bound of its length).  Dense mode: one tile per CTA.
+    const int n_tiles = dense ? (int)gridDim.x : hdr->n_small_tiles;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
+        __syncthreads();  // the previous tile's row descriptors and combine buffers are done with
+        clear_rows(rows);
+        __syncthreads();
+        int64_t tok0;
+        int n_tok;
+        if (!dense) {
+            const TileItem it = items[tile];
+            const int h = it.key / C;
+            if (threadIdx.x < it.n_entries * G) {
+                const int p = seg_entries[it.entry_begin + threadIdx.x / G];
+                const int g = threadIdx.x % G;
+                const int j = p % k, b = p / (k * Hkv);
+                const int64_t r = (int64_t)b * Hq + h * G + g;
+                rows.q[threadIdx.x] = q + r * D;
+                rows.o[threadIdx.x] = o_part + (r * n_slots + j) * D;
+                rows.lse[threadIdx.x] = lse_part + r * n_slots + j;
+            }
+            tok0 = (int64_t)it.key * L;
+            n_tok = L;
+        } else {
+            const int b_tiles = (B + per_tile - 1) / per_tile;
+            const int bt = tile % b_tiles;
+            const int j = (tile / b_tiles) % shared_slots;
+            const int h = tile / (b_tiles * shared_slots);
+            const int b = bt * per_tile + threadIdx.x / G;
+            if (threadIdx.x < per_tile * G && b < B) {
+                const int64_t r = (int64_t)b * Hq + h * G + threadIdx.x % G;
+                rows.q[threadIdx.x] = q + r * D;
+                rows.o[threadIdx.x] = o_part + (r * n_slots + j) * D;
+                rows.lse[threadIdx.x] = lse_part + r * n_slots + j;
+            }
+            const int run = (C + shared_slots - 1) / shared_slots;
+            const int c0 = min(C, j * run), c1 = min(C, c0 + run);
+            tok0 = ((int64_t)h * C + c0) * L;
+            n_tok = (c1 - c0) * L;
         }
-        tok0 = (int64_t)it.key * L;
-        n_tok = L;
-    } else {
-        const int b_tiles = (B + per_tile - 1) / per_tile;
-        const int bt = blockIdx.x % b_tiles;
-        const int j = (blockIdx.x / b_tiles) % shared_slots;
-        const int h = blockIdx.x / (b_tiles * shared_slots);
-        const int b = bt * per_tile + threadIdx.x / G;
-        if (threadIdx.x < per_tile * G && b < B) {
-            const int64_t r = (int64_t)b * Hq + h * G + threadIdx.x % G;
-            rows.q[threadIdx.x] = q + r * D;
-            rows.o[threadIdx.x] = o_part + (r * n_slots + j) * D;
-            rows.lse[threadIdx.x] = lse_part + r * n_slots + j;
-        }
-        const int run = (C + shared_slots - 1) / shared_slots;
-        const int c0 = min(C, j * run), c1 = min(C, c0 + run);
-        tok0 = ((int64_t)h * C + c0) * L;
-        n_tok = (c1 - c0) * L;
+        __syncthreads();
+        attend_stream<D, NT>(rows, k_shared + tok0 * D, v_shared + tok0 * D, D, 0, n_tok, scale, sm);
     }
-    __syncthreads();
-    attend_stream<D, NT>(rows, k_shared + tok0 * D, v_shared + tok0 * D, D, 0, n_tok, scale, sm);
 }
 
 }  // namespace
@@ -213,7 +218,11 @@ int launch_shared_small(const uint16_t* q, const uint16_t* k_shared, const uint1
         grid = (long long)s->Hkv * s->shared_slots * ((s->B + per_tile - 1) / per_tile);
     } else {
         const WsLayout lay = ws_layout(s);
-        grid = lay.max_small;
+        // resident CTAs (2 per SM) a few times over; they stride through the device-side list
+        int dev = 0, n_sms = 0;
+        MOSKA_CUDA_TRY(cudaGetDevice(&dev));
+        MOSKA_CUDA_TRY(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
+        grid = lay.max_small < 8LL * n_sms ? lay.max_small : 8LL * n_sms;
         hdr = reinterpret_cast<const WsHeader*>(ws);
         items = reinterpret_cast<const TileItem*>(static_cast<const char*>(ws) + lay.off_small);
     }

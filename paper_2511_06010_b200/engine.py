@@ -42,6 +42,11 @@ class MoskaLayer:
         ws_bytes = M.workspace_bytes(self.shape)
         self.ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=dev)
         self.side_stream: Optional[torch.cuda.Stream] = None
+        # The router keeps one score per chunk in shared memory.  With many chunks that footprint
+        # makes the SMs switch to a large shared-memory carve-out while it runs beside unique
+        # attention, whose loads then have too little L1 to stay in flight (measured: up to 40 %
+        # slower).  So routing only goes to a second, high-priority stream when C is small.
+        self.overlap_routing = (not dense) and C <= 512
 
     # -- offline ---------------------------------------------------------------------------------
     def build_summaries(self, k_shared):
@@ -73,6 +78,7 @@ class MoskaLayer:
     # -- the whole step --------------------------------------------------------------------------
     def step(self, q, k_shared, v_shared, k_unique, v_unique, kv_start, kv_len, two_streams=False,
              prof=None):
+        two_streams = two_streams and self.overlap_routing
         if two_streams and self.side_stream is None:
             self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
         M.decode_step(q, None if self.dense else self.summaries, k_shared, v_shared, k_unique,
@@ -84,6 +90,7 @@ class MoskaLayer:
 
     def step_host(self, q_host, q_dev, out_host, k_shared, v_shared, k_unique, v_unique,
                   kv_start, kv_len, two_streams=False, prof=None):
+        two_streams = two_streams and self.overlap_routing
         if two_streams and self.side_stream is None:
             self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
         M.decode_step_host(q_host, q_dev, None if self.dense else self.summaries, k_shared,
