@@ -238,6 +238,7 @@ def test_run_twice_bitwise_identical():
         outs.append((layer.out.clone(), layer.seg_entries.clone(), layer.o_part.clone()))
     for a, b in zip(outs[0], outs[1]):
         assert torch.equal(a, b)
+    assert M.device_status() == 0
 
 
 def test_reduced_configs_every_element():
