@@ -113,10 +113,13 @@ int moska_build_chunk_summaries(const uint16_t* k_shared, float* summaries,
  *   summaries   float [Hkv][C][D]
  *   topk_idx    int32 [B][Hkv][k]   out, chunk indices in ASCENDING order
  *   topk_score  float [B][Hkv][k]   out, score of topk_idx[...] (same order); may be NULL
- * One warp scores and selects for one (b, h).  No workspace.
+ * Up to 256 chunks one warp scores and selects for one (b, h) out of shared memory and `ws` may
+ * be NULL; beyond that the scores are computed as a tiled fp32 product into `ws` (which must
+ * then hold moska_workspace_bytes(); the grouping call may reuse the same workspace afterwards)
+ * and selected by one warp per (b, h).
  */
 int moska_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
-                const moska_shape* shape, moska_stream stream);
+                const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream);
 
 /*
  * Query aggregation (Section III-A: the N concurrent queries that hit the same shared chunk are

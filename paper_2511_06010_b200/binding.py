@@ -47,7 +47,7 @@ EXPORTS = {
     "moska_workspace_bytes": (_sz, [_sp]),
     "moska_default_unique_splits": (_i, [ctypes.c_int32] * 3),
     "moska_build_chunk_summaries": (_i, [_vp, _vp, _sp, _vp]),
-    "moska_route": (_i, [_vp, _vp, _vp, _vp, _sp, _vp]),
+    "moska_route": (_i, [_vp, _vp, _vp, _vp, _sp, _vp, _sz, _vp]),
     "moska_group_by_chunk": (_i, [_vp, _vp, _vp, _sp, _vp, _sz, _vp]),
     "moska_group_by_chunk_noalloc": (_i, [_vp, _vp, _vp, _sp, _vp]),
     "moska_shared_attn": (_i, [_vp] * 8 + [_f, _sp, _vp, _sz, _vp]),
@@ -129,9 +129,11 @@ def build_chunk_summaries(k_shared, summaries, s, stream=None) -> None:
                                             _stream(stream)), "moska_build_chunk_summaries")
 
 
-def route(q, summaries, topk_idx, topk_score, s, stream=None) -> None:
+def route(q, summaries, topk_idx, topk_score, s, ws=None, stream=None) -> None:
     _check(_lib.moska_route(_ptr(q), _ptr(summaries), _ptr(topk_idx), _ptr(topk_score),
-                            ctypes.byref(s), _stream(stream)), "moska_route")
+                            ctypes.byref(s), _ptr(ws),
+                            0 if ws is None else ws.numel() * ws.element_size(),
+                            _stream(stream)), "moska_route")
 
 
 def group_by_chunk(topk_idx, seg_offsets, seg_entries, s, ws, stream=None) -> None:

@@ -136,14 +136,18 @@ int moska_build_chunk_summaries(const uint16_t* k_shared, float* summaries,
 }
 
 int moska_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
-                const moska_shape* shape, moska_stream stream)
+                const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream)
 {
     MOSKA_TRY(check_shape(shape, true));
     MOSKA_TRY(check_device());
     REQUIRE_PTR(q, 16);
     REQUIRE_PTR(summaries, 16);
     REQUIRE_PTR(topk_idx, 4);
-    return launch_route(q, summaries, topk_idx, topk_score, shape, (cudaStream_t)stream);
+    if (shape->C > kRouteSmallC &&
+        (ws == nullptr || !aligned(ws, 256) || ws_bytes < ws_layout(shape).total))
+        return fail(MOSKA_ERR_WORKSPACE, "workspace missing, misaligned or smaller than %zu bytes",
+                    ws_layout(shape).total);
+    return launch_route(q, summaries, topk_idx, topk_score, shape, ws, (cudaStream_t)stream);
 }
 
 int moska_group_by_chunk(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
@@ -303,7 +307,7 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
             MOSKA_CUDA_TRY(cudaStreamWaitEvent(side, ev_fork, 0));
         }
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 0, cs));
-        MOSKA_TRY(moska_route(q, summaries, topk_idx, nullptr, shape, cs));
+        MOSKA_TRY(moska_route(q, summaries, topk_idx, nullptr, shape, ws, ws_bytes, cs));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 1, cs));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 0, cs));
         MOSKA_TRY(moska_group_by_chunk(topk_idx, seg_offsets, seg_entries, shape, ws, ws_bytes, cs));

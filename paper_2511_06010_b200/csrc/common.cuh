@@ -70,10 +70,14 @@ struct WsLayout {
     int32_t big_entries;      // requests per big tile
     int32_t big_min_entries;  // a remainder of at least this many requests still forms a big tile
     int64_t max_small, max_big;
-    size_t off_hist, off_totals, off_small, off_big, total;
+    size_t off_hist, off_totals, off_small, off_big;
+    size_t group_total;  // end of what the grouping passes and shared attention use
+    size_t off_scores;   // router: fp32 scores [B * Hkv][C] (only when C > kRouteSmallC)
+    size_t total;
 };
 WsLayout ws_layout(const moska_shape* s);
 
+constexpr int kRouteSmallC = 256;   // up to this many chunks the router keeps its scores in shared memory
 constexpr int kSmallTileRows = 16;  // query rows of one small tile (two 8-row MMA column blocks)
 constexpr int kBigTileRows = 128;   // query rows of one tensor-core (tcgen05) tile; a work item has two
 #ifndef MOSKA_BIG_MIN_ROWS
@@ -85,7 +89,7 @@ constexpr int kBigMinRows = MOSKA_BIG_MIN_ROWS;  // fewer leftover rows of a seg
 int launch_summaries(const uint16_t* k_shared, float* summaries, const moska_shape* s,
                      cudaStream_t st);
 int launch_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
-                 const moska_shape* s, cudaStream_t st);
+                 const moska_shape* s, void* ws, cudaStream_t st);
 int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
                  const moska_shape* s, void* ws, cudaStream_t st);
 int launch_group_noalloc(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,

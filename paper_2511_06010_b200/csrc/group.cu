@@ -36,6 +36,9 @@ WsLayout ws_layout(const moska_shape* s)
     off += round_up(sizeof(TileItem) * (size_t)w.max_small, 256);
     w.off_big = off;
     off += round_up(sizeof(TileItem) * (size_t)w.max_big, 256);
+    w.group_total = off;
+    w.off_scores = off;
+    if (s->C > kRouteSmallC) off += round_up(sizeof(float) * (size_t)s->B * s->Hkv * s->C, 256);
     w.total = off;
     return w;
 }
@@ -244,11 +247,11 @@ int launch_group_noalloc(const int32_t* topk_idx, int32_t* seg_offsets, int32_t*
                          const moska_shape* s, cudaStream_t st)
 {
     const WsLayout lay = ws_layout(s);
-    if (lay.total > (size_t)MOSKA_NOALLOC_SCRATCH_BYTES)
+    if (lay.group_total > (size_t)MOSKA_NOALLOC_SCRATCH_BYTES)
         return fail(MOSKA_ERR_WORKSPACE,
                     "shape needs %zu bytes of grouping scratch, the built-in buffer holds %zu "
                     "(use moska_group_by_chunk with a caller workspace)",
-                    lay.total, (size_t)MOSKA_NOALLOC_SCRATCH_BYTES);
+                    lay.group_total, (size_t)MOSKA_NOALLOC_SCRATCH_BYTES);
     MOSKA_TRY_STATUS(check_device());
     // `g_noalloc_scratch` names a host-side handle here, not a device address; the address on
     // the current device is looked up once per device and kept.

@@ -42,11 +42,12 @@ class MoskaLayer:
         ws_bytes = M.workspace_bytes(self.shape)
         self.ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=dev)
         self.side_stream: Optional[torch.cuda.Stream] = None
-        # The router keeps one score per chunk in shared memory.  With many chunks that footprint
-        # makes the SMs switch to a large shared-memory carve-out while it runs beside unique
-        # attention, whose loads then have too little L1 to stay in flight (measured: up to 40 %
-        # slower).  So routing only goes to a second, high-priority stream when C is small.
-        self.overlap_routing = (not dense) and C <= 512
+        # Routing and grouping can run on a second, high-priority stream beside unique attention.
+        # That only pays for the small-C router: the tiled router's CTAs (51 KB of shared memory
+        # each) make the SMs switch to a large shared-memory carve-out while they are resident,
+        # which leaves unique attention too little L1 for its loads in flight (measured: up to
+        # 40 % slower), more than the overlap saves.
+        self.overlap_routing = (not dense) and C <= 256
 
     # -- offline ---------------------------------------------------------------------------------
     def build_summaries(self, k_shared):
@@ -55,7 +56,7 @@ class MoskaLayer:
 
     # -- the individual stages (used by the per-stage parity tests and per-kernel timing) --------
     def route(self, q):
-        M.route(q, self.summaries, self.topk_idx, self.topk_score, self.shape)
+        M.route(q, self.summaries, self.topk_idx, self.topk_score, self.shape, self.ws)
 
     def group(self):
         M.group_by_chunk(self.topk_idx, self.seg_offsets, self.seg_entries, self.shape, self.ws)

@@ -223,6 +223,30 @@ def test_exact_ties_route_to_lower_chunk():
                           np.tile(np.arange(3, dtype=np.int32), (8, 2, 1)))
 
 
+def test_router_many_chunks_ties_and_ragged_tiles():
+    """The tiled router (C > 256): C and B that are no multiples of its tile sizes, duplicated
+    chunks (bit-identical scores: the lower index must win) and all-zero queries."""
+    M, MoskaLayer = _mods()
+    for B, Hq, Hkv, D, C, k in ((37, 8, 2, 128, 300, 5), (70, 4, 2, 64, 515, 33), (5, 8, 1, 128, 257, 64)):
+        w = W.Workload("route", B=B, Hq=Hq, Hkv=Hkv, D=D, C=C, L=128, k=k, unique_len=16, seed=31 + B)
+        sh = W.make_shared_store(w, "cuda")
+        sh.k_shared[:, C - 3] = sh.k_shared[:, 7]      # duplicates far apart and in the last tile
+        sh.k_shared[:, 100] = sh.k_shared[:, 7]
+        q = W.make_queries(w, sh, 0, "cuda")
+        layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, 16)
+        layer.build_summaries(sh.k_shared)
+        layer.route(q)
+        summ = O.chunk_summaries(sh.k_shared.cpu())
+        ref_idx, _, ref_all = O.route(q.cpu(), summ, w.k, return_all=True)
+        gpu_idx = layer.topk_idx.cpu().numpy()
+        assert PU.check_routing(gpu_idx, ref_idx, ref_all) == 0
+        picked = np.take_along_axis(ref_all, gpu_idx.astype(np.int64), axis=-1)
+        np.testing.assert_allclose(layer.topk_score.cpu().numpy(), picked, rtol=1e-4, atol=1e-3)
+        layer.route(torch.zeros_like(q))
+        assert np.array_equal(layer.topk_idx.cpu().numpy(),
+                              np.tile(np.arange(k, dtype=np.int32), (B, Hkv, 1)))
+
+
 def test_run_twice_bitwise_identical():
     M, MoskaLayer = _mods()
     w = W.scaled(W.CONFIGS[1], B=16, C=32, unique_len=700)
