@@ -59,18 +59,20 @@ struct WsHeader {
     int32_t n_small_tiles;  // items in the small-tile list
     int32_t n_big_tiles;    // items in the big-tile list
     int32_t status;         // 0, or a negative code set by a device-side range check
-    int32_t pad[61];
+    int32_t n_tiny_tiles;   // items in the 8-row tile list
+    int32_t pad[60];
 };
 static_assert(sizeof(WsHeader) == 256, "header is one 256-byte block");
 
 struct WsLayout {
     int32_t words;            // 32-bit words of one key's request bit set
     int32_t n_keys;           // Hkv * C
-    int32_t small_entries;    // requests per small tile
+    int32_t small_entries;    // requests per small (16-row) tile
+    int32_t tiny_entries;     // requests per 8-row tile
     int32_t big_entries;      // requests per big tile
     int32_t big_min_entries;  // a remainder of at least this many requests still forms a big tile
     int64_t max_small, max_big;
-    size_t off_hist, off_totals, off_small, off_big;
+    size_t off_hist, off_totals, off_small, off_big, off_tiny;
     size_t group_total;  // end of what the grouping passes and shared attention use
     size_t off_scores;   // router: fp32 scores [B * Hkv][C] (only when C > kRouteSmallC)
     size_t total;

@@ -21,6 +21,7 @@ WsLayout ws_layout(const moska_shape* s)
     w.n_keys = s->Hkv * s->C;
     w.words = (s->B + 31) / 32 > 0 ? (s->B + 31) / 32 : 1;
     w.small_entries = kSmallTileRows / G;
+    w.tiny_entries = 8 / G;  // requests whose rows fit one 8-row MMA column block (0: no such tiles)
     w.big_entries = 2 * (kBigTileRows / G);  // a tensor-core work item holds two 128-row tiles
     w.big_min_entries = shared_tc_supported(s) ? (kBigMinRows + G - 1) / G : 0x7fffffff;
     const int64_t P = (int64_t)s->B * s->Hkv * s->k;
@@ -36,6 +37,8 @@ WsLayout ws_layout(const moska_shape* s)
     off += round_up(sizeof(TileItem) * (size_t)w.max_small, 256);
     w.off_big = off;
     off += round_up(sizeof(TileItem) * (size_t)w.max_big, 256);
+    w.off_tiny = off;
+    off += round_up(sizeof(TileItem) * (size_t)segs, 256);  // at most one 8-row tile per segment
     w.group_total = off;
     w.off_scores = off;
     if (s->C > kRouteSmallC) off += round_up(sizeof(float) * (size_t)s->B * s->Hkv * s->C, 256);
@@ -76,21 +79,29 @@ group_count_kernel(const uint32_t* __restrict__ bitmap, int32_t* __restrict__ to
 }
 
 // Exclusive scans over the keys, one CTA: entries -> seg_offsets; tiles -> work lists.
+// A segment's requests go, in order, to tensor-core items (whole multiples of big_entries, and a
+// remainder of at least big_min_entries), then to 16-row tiles, and a last piece of at most
+// tiny_entries requests (8 rows) to the 8-row tile list.
 __global__ void __launch_bounds__(1024)
 group_scan_kernel(const int32_t* __restrict__ totals, int32_t* __restrict__ seg_offsets,
                   WsHeader* __restrict__ hdr, TileItem* __restrict__ small_items,
-                  TileItem* __restrict__ big_items, int n_keys, int small_entries,
-                  int big_entries, int big_min_entries)
+                  TileItem* __restrict__ tiny_items, TileItem* __restrict__ big_items, int n_keys,
+                  int small_entries, int tiny_entries, int big_entries, int big_min_entries)
 {
-    __shared__ int3 warp_sum[32];
-    __shared__ int3 carry;
+    __shared__ int4 warp_sum[32];
+    __shared__ int4 carry;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (threadIdx.x == 0) carry = make_int3(0, 0, 0);
+    auto add = [](int4 a, int4 b) { return make_int4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); };
+    auto sub = [](int4 a, int4 b) { return make_int4(a.x - b.x, a.y - b.y, a.z - b.z, a.w - b.w); };
+    auto shfl_up = [](int4 a, int off) {
+        return make_int4(__shfl_up_sync(0xffffffffu, a.x, off), __shfl_up_sync(0xffffffffu, a.y, off),
+                         __shfl_up_sync(0xffffffffu, a.z, off), __shfl_up_sync(0xffffffffu, a.w, off));
+    };
+    if (threadIdx.x == 0) carry = make_int4(0, 0, 0, 0);
     __syncthreads();
     for (int base = 0; base < n_keys; base += blockDim.x) {
         const int key = base + threadIdx.x;
         const int n = key < n_keys ? totals[key] : 0;
-        // tensor-core tiles take whole multiples of big_entries, and a large enough remainder
         int n_big = n / big_entries;
         int rem = n - n_big * big_entries;
         if (rem >= big_min_entries) {
@@ -101,67 +112,58 @@ group_scan_kernel(const int32_t* __restrict__ totals, int32_t* __restrict__ seg_
             n_big = 0;
             rem = n;
         }
-        const int n_small = (rem + small_entries - 1) / small_entries;
-        int3 v = make_int3(n, n_small, n_big);
-        int3 inc = v;
+        int n_small = rem / small_entries;
+        const int last = rem - n_small * small_entries;  // requests of the last, partial tile
+        int n_tiny = 0;
+        if (last > 0) {
+            if (last <= tiny_entries) n_tiny = 1; else ++n_small;
+        }
+        // x: entries, y: 16-row tiles, z: tensor-core items, w: 8-row tiles
+        const int4 v = make_int4(n, n_small, n_big, n_tiny);
+        int4 inc = v;
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
-            const int a = __shfl_up_sync(0xffffffffu, inc.x, off);
-            const int b = __shfl_up_sync(0xffffffffu, inc.y, off);
-            const int c = __shfl_up_sync(0xffffffffu, inc.z, off);
-            if (lane >= off) {
-                inc.x += a;
-                inc.y += b;
-                inc.z += c;
-            }
+            const int4 t = shfl_up(inc, off);
+            if (lane >= off) inc = add(inc, t);
         }
         if (lane == 31) warp_sum[warp] = inc;
         __syncthreads();
         if (warp == 0) {
-            int3 w = warp_sum[lane];
-            int3 winc = w;
+            const int4 w = warp_sum[lane];
+            int4 winc = w;
 #pragma unroll
             for (int off = 1; off < 32; off <<= 1) {
-                const int a = __shfl_up_sync(0xffffffffu, winc.x, off);
-                const int b = __shfl_up_sync(0xffffffffu, winc.y, off);
-                const int c = __shfl_up_sync(0xffffffffu, winc.z, off);
-                if (lane >= off) {
-                    winc.x += a;
-                    winc.y += b;
-                    winc.z += c;
-                }
+                const int4 t = shfl_up(winc, off);
+                if (lane >= off) winc = add(winc, t);
             }
-            warp_sum[lane] = make_int3(winc.x - w.x, winc.y - w.y, winc.z - w.z);  // exclusive
+            warp_sum[lane] = sub(winc, w);  // exclusive
         }
         __syncthreads();
-        const int3 wbase = warp_sum[warp];
-        const int3 cr = carry;
-        const int ex_n = cr.x + wbase.x + inc.x - v.x;
-        const int ex_s = cr.y + wbase.y + inc.y - v.y;
-        const int ex_b = cr.z + wbase.z + inc.z - v.z;
+        const int4 ex = add(add(carry, warp_sum[warp]), sub(inc, v));
         if (key < n_keys) {
-            seg_offsets[key] = ex_n;
-            int e = ex_n;
+            seg_offsets[key] = ex.x;
+            int e = ex.x;
             for (int t = 0; t < n_big; ++t) {
-                const int cnt = min(big_entries, ex_n + n - e);
-                big_items[ex_b + t] = TileItem{key, e, cnt, 0};
+                const int cnt = min(big_entries, ex.x + n - e);
+                big_items[ex.z + t] = TileItem{key, e, cnt, 0};
                 e += cnt;
             }
             for (int t = 0; t < n_small; ++t) {
-                const int cnt = min(small_entries, ex_n + n - e);
-                small_items[ex_s + t] = TileItem{key, e, cnt, 0};
+                const int cnt = min(small_entries, ex.x + n - e);
+                small_items[ex.y + t] = TileItem{key, e, cnt, 0};
                 e += cnt;
             }
+            if (n_tiny) tiny_items[ex.w] = TileItem{key, e, ex.x + n - e, 0};
         }
         __syncthreads();
-        if (threadIdx.x == blockDim.x - 1)
-            carry = make_int3(ex_n + v.x, ex_s + v.y, ex_b + v.z);
+        if (threadIdx.x == blockDim.x - 1) carry = add(ex, v);
         __syncthreads();
     }
     if (threadIdx.x == 0) {
         seg_offsets[n_keys] = carry.x;
         hdr->n_small_tiles = carry.y;
         hdr->n_big_tiles = carry.z;
+        hdr->n_tiny_tiles = carry.w;
     }
 }
 
@@ -218,6 +220,7 @@ int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_ent
     int32_t* totals = reinterpret_cast<int32_t*>(base + lay.off_totals);
     TileItem* small_items = reinterpret_cast<TileItem*>(base + lay.off_small);
     TileItem* big_items = reinterpret_cast<TileItem*>(base + lay.off_big);
+    TileItem* tiny_items = reinterpret_cast<TileItem*>(base + lay.off_tiny);
     const long long P = (long long)s->B * s->Hkv * s->k;
     // header and bit sets must start at zero
     MOSKA_CUDA_TRY(cudaMemsetAsync(base, 0, lay.off_totals, st));
@@ -228,9 +231,9 @@ int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_ent
     }
     group_count_kernel<<<(lay.n_keys + 255) / 256, 256, 0, st>>>(bitmap, totals, lay.n_keys, lay.words);
     MOSKA_LAUNCH_CHECK("group_count_kernel");
-    group_scan_kernel<<<1, 1024, 0, st>>>(totals, seg_offsets, hdr, small_items, big_items,
-                                          lay.n_keys, lay.small_entries, lay.big_entries,
-                                          lay.big_min_entries);
+    group_scan_kernel<<<1, 1024, 0, st>>>(totals, seg_offsets, hdr, small_items, tiny_items, big_items,
+                                          lay.n_keys, lay.small_entries, lay.tiny_entries,
+                                          lay.big_entries, lay.big_min_entries);
     MOSKA_LAUNCH_CHECK("group_scan_kernel");
     group_emit_kernel<<<(lay.n_keys + 7) / 8, 256, 0, st>>>(topk_idx, bitmap, seg_offsets, seg_entries,
                                                             lay.n_keys, s->Hkv, s->C, s->k, lay.words);

@@ -1,5 +1,7 @@
 // Kernels built on the streaming decode-attention block: Unique KV Attention, the unbatched
 // per-request GEMV baseline over shared chunks, and Shared KV Attention for small query tiles.
+#include <cstddef>
+
 #include "common.cuh"
 #include "stream_attn.cuh"
 
@@ -104,22 +106,23 @@ gemv_baseline_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict_
 // Routed mode: one CTA per work item = up to 16/G requests of one (KV head, chunk) segment; the
 // chunk's K/V is streamed once for all of them.  Dense mode: one CTA per (KV head, run of chunks,
 // group of 16/G requests).
-template <int D>
-__global__ void __launch_bounds__(kThreads, 2)
+template <int D, int NT>
+__global__ void __launch_bounds__(kThreads, NT == 1 ? 3 : 2)
 shared_small_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_shared,
                     const uint16_t* __restrict__ v_shared, const int32_t* __restrict__ seg_entries,
                     const WsHeader* __restrict__ hdr, const TileItem* __restrict__ items,
                     float* __restrict__ o_part, float* __restrict__ lse_part, float scale, int B,
-                    int Hq, int Hkv, int C, int L, int k, int shared_slots, int n_slots, int dense)
+                    int Hq, int Hkv, int C, int L, int k, int shared_slots, int n_slots, int dense,
+                    int n_tiles_offset)
 {
-    constexpr int NT = kSmallTileRows / 8;
     __shared__ TileRows<NT> rows;
     __shared__ CombineSmem<D, NT> sm;
     const int G = Hq / Hkv;
-    const int per_tile = kSmallTileRows / G;  // requests per tile
+    const int per_tile = NT * 8 / G;  // requests per tile
     // Routed mode: the CTAs walk the device-side tile list with the grid as their stride (the
     // host only knows an upper bound of its length).  Dense mode: one tile per CTA.
-    const int n_tiles = dense ? (int)gridDim.x : hdr->n_small_tiles;
+    // which header word counts this list: the 16-row (NT = 2) or the 8-row (NT = 1) tiles
+    const int n_tiles = dense ? (int)gridDim.x : reinterpret_cast<const int32_t*>(hdr)[n_tiles_offset];
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x) {
         __syncthreads();  // the previous tile's row descriptors and combine buffers are done with
         clear_rows(rows);
@@ -213,6 +216,7 @@ int launch_shared_small(const uint16_t* q, const uint16_t* k_shared, const uint1
     long long grid;
     const WsHeader* hdr = nullptr;
     const TileItem* items = nullptr;
+    const TileItem* tiny_items = nullptr;
     if (dense) {
         const int per_tile = kSmallTileRows / G;
         grid = (long long)s->Hkv * s->shared_slots * ((s->B + per_tile - 1) / per_tile);
@@ -225,17 +229,25 @@ int launch_shared_small(const uint16_t* q, const uint16_t* k_shared, const uint1
         grid = lay.max_small < 8LL * n_sms ? lay.max_small : 8LL * n_sms;
         hdr = reinterpret_cast<const WsHeader*>(ws);
         items = reinterpret_cast<const TileItem*>(static_cast<const char*>(ws) + lay.off_small);
+        if (lay.tiny_entries > 0)
+            tiny_items = reinterpret_cast<const TileItem*>(static_cast<const char*>(ws) + lay.off_tiny);
     }
     if (grid == 0) return MOSKA_OK;
     if (grid > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "shared attention grid too large");
-    if (s->D == 128)
-        shared_small_kernel<128><<<(unsigned)grid, kThreads, 0, st>>>(
-            q, k_shared, v_shared, seg_entries, hdr, items, o_part, lse_part, scale, s->B, s->Hq,
-            s->Hkv, s->C, s->L, s->k, s->shared_slots, n_slots, dense ? 1 : 0);
-    else
-        shared_small_kernel<64><<<(unsigned)grid, kThreads, 0, st>>>(
-            q, k_shared, v_shared, seg_entries, hdr, items, o_part, lse_part, scale, s->B, s->Hq,
-            s->Hkv, s->C, s->L, s->k, s->shared_slots, n_slots, dense ? 1 : 0);
+    constexpr int kSmallWord = offsetof(WsHeader, n_small_tiles) / 4;
+    constexpr int kTinyWord = offsetof(WsHeader, n_tiny_tiles) / 4;
+#define MOSKA_LAUNCH_SMALL(DD, NN, ITEMS, WORD)                                                        \
+    shared_small_kernel<DD, NN><<<(unsigned)grid, kThreads, 0, st>>>(                                  \
+        q, k_shared, v_shared, seg_entries, hdr, ITEMS, o_part, lse_part, scale, s->B, s->Hq, s->Hkv,  \
+        s->C, s->L, s->k, s->shared_slots, n_slots, dense ? 1 : 0, WORD)
+    if (s->D == 128) MOSKA_LAUNCH_SMALL(128, 2, items, kSmallWord);
+    else MOSKA_LAUNCH_SMALL(64, 2, items, kSmallWord);
+    if (!dense && tiny_items != nullptr) {
+        MOSKA_LAUNCH_CHECK("shared_small_kernel");
+        if (s->D == 128) MOSKA_LAUNCH_SMALL(128, 1, tiny_items, kTinyWord);
+        else MOSKA_LAUNCH_SMALL(64, 1, tiny_items, kTinyWord);
+    }
+#undef MOSKA_LAUNCH_SMALL
     MOSKA_LAUNCH_CHECK("shared_small_kernel");
     return MOSKA_OK;
 }
