@@ -56,7 +56,10 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock, power and throttle reasons of one GPU while the timed region runs.
+
+    Reads through NVML in a thread every 5 ms (read-only queries); falls back to an `nvidia-smi`
+    loop when the NVML binding is missing."""
 
     Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
          "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -64,47 +67,91 @@ class ClockSampler:
 
     def __init__(self, index: int):
         self.index = index
-        self.rows = []
+        self.rows = []          # (sm_mhz, set of reason names)
+        self.sm_max = None
         self.proc = None
+        self.thread = None
+        self.stop_flag = False
+        self.source = None
+
+    def _nvml_loop(self, nv, handle):
+        names = {
+            "hw_slowdown": nv.nvmlClocksEventReasonHwSlowdown
+            if hasattr(nv, "nvmlClocksEventReasonHwSlowdown") else nv.nvmlClocksThrottleReasonHwSlowdown,
+            "hw_thermal_slowdown": nv.nvmlClocksEventReasonHwThermalSlowdown
+            if hasattr(nv, "nvmlClocksEventReasonHwThermalSlowdown") else nv.nvmlClocksThrottleReasonHwThermalSlowdown,
+            "sw_thermal_slowdown": nv.nvmlClocksEventReasonSwThermalSlowdown
+            if hasattr(nv, "nvmlClocksEventReasonSwThermalSlowdown") else nv.nvmlClocksThrottleReasonSwThermalSlowdown,
+            "sw_power_cap": nv.nvmlClocksEventReasonSwPowerCap
+            if hasattr(nv, "nvmlClocksEventReasonSwPowerCap") else nv.nvmlClocksThrottleReasonSwPowerCap,
+        }
+        get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+            nv.nvmlDeviceGetCurrentClocksThrottleReasons
+        while not self.stop_flag:
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(handle, nv.NVML_CLOCK_SM)
+                bits = get_reasons(handle)
+                self.rows.append((float(mhz), {n for n, b in names.items() if bits & b}))
+            except Exception:
+                pass
+            time.sleep(0.005)
 
     def start(self):
         try:
+            import pynvml as nv
+
+            nv.nvmlInit()
+            # NVML enumerates physical GPUs; honour CUDA_VISIBLE_DEVICES when it lists indices
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+            ids = [v for v in vis.split(",") if v.strip().isdigit()]
+            phys = int(ids[self.index]) if self.index < len(ids) else self.index
+            handle = nv.nvmlDeviceGetHandleByIndex(phys)
+            self.sm_max = float(nv.nvmlDeviceGetMaxClockInfo(handle, nv.NVML_CLOCK_SM))
+            self.source = "nvml"
+            self.thread = threading.Thread(target=self._nvml_loop, args=(nv, handle), daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.source = None
+        try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
-            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.source = "nvidia-smi"
+            self.thread = threading.Thread(target=self._read_smi, daemon=True)
             self.thread.start()
         except Exception:
             self.proc = None
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.rows.append([x.strip() for x in line.split(",")])
-
-    def stop(self):
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.15)
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=2)
-        except Exception:
-            self.proc.kill()
-        sm, smax, reasons = [], [], set()
+    def _read_smi(self):
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for r in self.rows:
+        for line in self.proc.stdout:
+            r = [x.strip() for x in line.split(",")]
             try:
-                sm.append(float(r[0]))
-                smax.append(float(r[1]))
+                self.sm_max = float(r[1])
+                self.rows.append((float(r[0]),
+                                  {n for n, v in zip(names, r[3:7]) if v.lower().startswith("active")}))
             except Exception:
                 continue
-            for n, v in zip(names, r[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": statistics.median(sm) if sm else None,
-                "sm_max_mhz": max(smax) if smax else None, "samples": len(sm),
-                "reasons": sorted(reasons)}
+
+    def stop(self):
+        if self.source is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no clock source available"]}
+        if self.source == "nvml":
+            self.stop_flag = True
+            self.thread.join(timeout=1)
+        else:
+            time.sleep(0.05)
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                self.proc.kill()
+        sm = [r[0] for r in self.rows]
+        reasons = set().union(*[r[1] for r in self.rows]) if self.rows else set()
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": self.sm_max,
+                "samples": len(sm), "source": self.source, "reasons": sorted(reasons)}
 
 
 def algorithmic_work(w: W.Workload, lens: np.ndarray, n_unique_splits: int, shared_slots: int,
@@ -377,8 +424,10 @@ def run_cuda(args, w):
                "sample": f"first {n_s} of {w.B} requests (all heads, full context), {reps} repeats, "
                          f"{dt * reps:.1f} s"}
 
-    # kernels of one step: route, 4 grouping passes, unique, shared (tensor-core + small tiles), merge
-    n_launch = (3 if w.dense else (9 if w.D == 128 else 8)) * args.steps
+    # kernels of one step: route (scoring + selection beyond 256 chunks), 4 grouping passes, unique,
+    # shared (tensor-core items, 16-row tiles, 8-row tiles), merge
+    n_launch = 3 if w.dense else (1 + (w.C > 256)) + 4 + 1 + (3 if w.D == 128 else 2) + 1
+    n_launch *= args.steps
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": ms_per_step_max, "higher_is_better": True,
