@@ -417,7 +417,7 @@ def run_cuda(args, w):
         while True:
             cpu_oracle_step(w, sh_host, un_host, qh, lens_s, summ, sample)
             reps += 1
-            if time.perf_counter() - t0 > args.cpu_seconds or reps >= 50:
+            if time.perf_counter() - t0 > args.cpu_seconds or reps >= 500:
                 break
         dt = (time.perf_counter() - t0) / reps
         cpu = {"value": n_s / dt, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",

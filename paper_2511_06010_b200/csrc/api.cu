@@ -312,7 +312,14 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 0, cs));
         MOSKA_TRY(moska_group_by_chunk(topk_idx, seg_offsets, seg_entries, shape, ws, ws_bytes, cs));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 1, cs));
-        if (side != nullptr) MOSKA_CUDA_TRY(cudaEventRecord(ev_join, side));
+        if (side != nullptr) {
+            // the streaming (16- and 8-row) tiles of shared attention are HBM-bound like unique
+            // attention and small in shared memory: they run beside it; only the tensor-core
+            // items wait for the main stream
+            MOSKA_TRY(launch_shared_small(q, k_shared, v_shared, seg_entries, o_part, lse_part,
+                                          softmax_scale, shape, ws, false, side));
+            MOSKA_CUDA_TRY(cudaEventRecord(ev_join, side));
+        }
     }
     MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 0, st));
     MOSKA_TRY(moska_unique_attn(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part,
@@ -320,7 +327,11 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
     MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 1, st));
     if (!dense && side != nullptr) MOSKA_CUDA_TRY(cudaStreamWaitEvent(st, ev_join, 0));
     MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 0, st));
-    if (!dense)
+    if (!dense && side != nullptr) {
+        if (shared_tc_supported(shape))
+            MOSKA_TRY(launch_shared_tc(q, k_shared, v_shared, seg_entries, o_part, lse_part,
+                                       softmax_scale, shape, ws, false, st));
+    } else if (!dense)
         MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, topk_idx, seg_offsets, seg_entries,
                                     o_part, lse_part, softmax_scale, shape, ws, ws_bytes, st));
     else
