@@ -187,7 +187,7 @@ int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_
     REQUIRE_PTR(q, 16);
     REQUIRE_PTR(k_shared, 128);
     REQUIRE_PTR(v_shared, 128);
-    REQUIRE_PTR(o_part, 16);
+    REQUIRE_PTR(o_part, 32);
     REQUIRE_PTR(lse_part, 4);
     if (!dense) {
         REQUIRE_PTR(topk_idx, 4);

@@ -110,6 +110,14 @@ __device__ __forceinline__ float2 fadd2(float2 a, float2 b)
     return d;
 }
 
+// One 32-byte store (sm_100): p must be 32-byte aligned.
+__device__ __forceinline__ void st_global_v8(float* p, const float* v)
+{
+    asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "f"(v[0]),
+                 "f"(v[1]), "f"(v[2]), "f"(v[3]), "f"(v[4]), "f"(v[5]), "f"(v[6]), "f"(v[7])
+                 : "memory");
+}
+
 __device__ __forceinline__ float fmax3(float a, float b, float c)
 {
     float d;
@@ -577,24 +585,40 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             float4* o = my_r >= 0
                 ? reinterpret_cast<float4*>(p.o_part + (my_r * p.n_slots + my_slot) * kD)
                 : nullptr;
+            // the whole accumulator row: four loads in flight, one wait (two rounds when a second
+            // accumulator has to be folded in)
+            {
+                uint32_t r[4][32];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t r[32];
-                tmem_ld32(t_o + c * 32, r);
+                for (int c = 0; c < 4; ++c) tmem_ld32(t_o + c * 32, r[c]);
                 tmem_ld_wait();
-                float v[32];
 #pragma unroll
-                for (int x = 0; x < 32; ++x) v[x] = __uint_as_float(r[x]) * a_mine;
+                for (int c = 0; c < 4; ++c)
+#pragma unroll
+                    for (int x = 0; x < 32; ++x) r[c][x] = __float_as_uint(__uint_as_float(r[c][x]) * a_mine);
                 if (it.split) {
-                    tmem_ld32(t_o_other + c * 32, r);
-                    tmem_ld_wait();
 #pragma unroll
-                    for (int x = 0; x < 32; ++x) v[x] = fmaf(__uint_as_float(r[x]), a_other, v[x]);
+                    for (int hv = 0; hv < 2; ++hv) {
+                        uint32_t r2[2][32];
+                        tmem_ld32(t_o_other + hv * 64, r2[0]);
+                        tmem_ld32(t_o_other + hv * 64 + 32, r2[1]);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int c = 0; c < 2; ++c)
+#pragma unroll
+                            for (int x = 0; x < 32; ++x)
+                                r[2 * hv + c][x] = __float_as_uint(
+                                    fmaf(__uint_as_float(r2[c][x]), a_other, __uint_as_float(r[2 * hv + c][x])));
+                    }
                 }
                 if (o != nullptr) {
+                    // 32-byte stores: every instruction writes whole sectors of the row
 #pragma unroll
-                    for (int x = 0; x < 8; ++x)
-                        o[c * 8 + x] = make_float4(v[4 * x], v[4 * x + 1], v[4 * x + 2], v[4 * x + 3]);
+                    for (int c = 0; c < 4; ++c)
+#pragma unroll
+                        for (int x = 0; x < 4; ++x)
+                            st_global_v8(reinterpret_cast<float*>(o) + c * 32 + x * 8,
+                                         reinterpret_cast<const float*>(&r[c][8 * x]));
                 }
             }
             if (my_r >= 0) p.lse_part[my_r * p.n_slots + my_slot] = m_all * p.scale + logf(den);
