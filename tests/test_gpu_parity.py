@@ -322,3 +322,27 @@ def test_full_cfg4_sampled_steps():
     for step in (0, w.steps - 1):
         run_case(w, sample=_sample(w, 3), check_baseline=False, step=step, two_streams=True)
         torch.cuda.empty_cache()
+
+
+def test_several_query_tokens_per_request_by_batch_expansion():
+    """Speculative decoding / chunked prefill: t query tokens of one request are t batch rows that
+    share the request's unique KV (token i sees the first len + i tokens of it).  The library
+    needs nothing special for it: `kv_start` may alias.  Checked against the oracle row by row."""
+    M, MoskaLayer = _mods()
+    base, t = 6, 4
+    w = W.Workload("multi", B=base * t, Hq=8, Hkv=2, D=128, C=8, L=256, k=2, unique_len=0, seed=41)
+    sh = W.make_shared_store(w, "cuda")
+    lens0 = np.array([40, 1, 130, 77, 300, 15], dtype=np.int64)
+    un = W.make_unique_store(W.scaled(w, B=base, steps=t), "cuda", lens0)
+    q = W.make_queries(w, sh, 0, "cuda")
+    kv_start = un.kv_start.repeat_interleave(t)
+    kv_len = (un.kv_len.repeat_interleave(t) + torch.arange(t, device="cuda").repeat(base)).to(torch.int32)
+    layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, int(kv_len.max().item()), n_unique_splits=2)
+    layer.build_summaries(sh.k_shared)
+    out = layer.step(q, sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, kv_start, kv_len)
+    torch.cuda.synchronize()
+    ref, _ = O.attend_direct(q.cpu(), sh.k_shared.cpu(), sh.v_shared.cpu(), un.k_unique.cpu(),
+                             un.v_unique.cpu(), kv_start.cpu().numpy(), kv_len.cpu().numpy(),
+                             layer.topk_idx.cpu().numpy(), layer.scale)
+    PU.check_attention(out.float().cpu().numpy(), ref, "several query tokens per request")
+    assert M.device_status() == 0
