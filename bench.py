@@ -424,9 +424,9 @@ def run_cuda(args, w):
                "sample": f"first {n_s} of {w.B} requests (all heads, full context), {reps} repeats, "
                          f"{dt * reps:.1f} s"}
 
-    # kernels of one step: route (scoring + selection beyond 256 chunks), 4 grouping passes, unique,
+    # kernels of one step: route (scoring + selection beyond 256 chunks), 2-3 grouping passes, unique,
     # shared (tensor-core items, 16-row tiles, 8-row tiles), merge
-    n_launch = 3 if w.dense else (1 + (w.C > 256)) + 4 + 1 + (3 if w.D == 128 else 2) + 1
+    n_launch = 3 if w.dense else (1 + (w.C > 256)) + (3 if w.B > 64 else 2) + 1 + (3 if w.D == 128 else 2) + 1
     n_launch *= args.steps
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

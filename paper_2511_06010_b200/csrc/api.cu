@@ -135,23 +135,27 @@ int moska_build_chunk_summaries(const uint16_t* k_shared, float* summaries,
     return launch_summaries(k_shared, summaries, shape, (cudaStream_t)stream);
 }
 
-int moska_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
-                const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream)
+namespace {
+// Validation + launch of the router; mark_groups also runs the grouping's first pass in it.
+int route_impl(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
+               const moska_shape* shape, void* ws, size_t ws_bytes, bool mark_groups,
+               cudaStream_t stream)
 {
     MOSKA_TRY(check_shape(shape, true));
     MOSKA_TRY(check_device());
     REQUIRE_PTR(q, 16);
     REQUIRE_PTR(summaries, 16);
     REQUIRE_PTR(topk_idx, 4);
-    if (shape->C > kRouteSmallC &&
+    if ((shape->C > kRouteSmallC || mark_groups) &&
         (ws == nullptr || !aligned(ws, 256) || ws_bytes < ws_layout(shape).total))
         return fail(MOSKA_ERR_WORKSPACE, "workspace missing, misaligned or smaller than %zu bytes",
                     ws_layout(shape).total);
-    return launch_route(q, summaries, topk_idx, topk_score, shape, ws, (cudaStream_t)stream);
+    return launch_route(q, summaries, topk_idx, topk_score, shape, ws, mark_groups, stream);
 }
 
-int moska_group_by_chunk(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
-                         const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream)
+int group_impl(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
+               const moska_shape* shape, void* ws, size_t ws_bytes, bool premarked,
+               cudaStream_t stream)
 {
     MOSKA_TRY(check_shape(shape, true));
     MOSKA_TRY(check_device());
@@ -161,7 +165,22 @@ int moska_group_by_chunk(const int32_t* topk_idx, int32_t* seg_offsets, int32_t*
     if (ws == nullptr || !aligned(ws, 256) || ws_bytes < ws_layout(shape).total)
         return fail(MOSKA_ERR_WORKSPACE, "workspace missing, misaligned or smaller than %zu bytes",
                     ws_layout(shape).total);
-    return launch_group(topk_idx, seg_offsets, seg_entries, shape, ws, (cudaStream_t)stream);
+    return launch_group(topk_idx, seg_offsets, seg_entries, shape, ws, premarked, stream);
+}
+}  // namespace
+
+int moska_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
+                const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream)
+{
+    return route_impl(q, summaries, topk_idx, topk_score, shape, ws, ws_bytes, false,
+                      (cudaStream_t)stream);
+}
+
+int moska_group_by_chunk(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
+                         const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream)
+{
+    return group_impl(topk_idx, seg_offsets, seg_entries, shape, ws, ws_bytes, false,
+                      (cudaStream_t)stream);
 }
 
 int moska_group_by_chunk_noalloc(const int32_t* topk_idx, int32_t* seg_offsets,
@@ -307,10 +326,11 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
             MOSKA_CUDA_TRY(cudaStreamWaitEvent(side, ev_fork, 0));
         }
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 0, cs));
-        MOSKA_TRY(moska_route(q, summaries, topk_idx, nullptr, shape, ws, ws_bytes, cs));
+        // the router also sets the grouping's request bits while it writes its picks
+        MOSKA_TRY(route_impl(q, summaries, topk_idx, nullptr, shape, ws, ws_bytes, true, cs));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 1, cs));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 0, cs));
-        MOSKA_TRY(moska_group_by_chunk(topk_idx, seg_offsets, seg_entries, shape, ws, ws_bytes, cs));
+        MOSKA_TRY(group_impl(topk_idx, seg_offsets, seg_entries, shape, ws, ws_bytes, true, cs));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 1, cs));
         if (side != nullptr) {
             // the streaming (16- and 8-row) tiles of shared attention are HBM-bound like unique

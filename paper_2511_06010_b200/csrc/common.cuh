@@ -91,9 +91,9 @@ constexpr int kBigMinRows = MOSKA_BIG_MIN_ROWS;  // fewer leftover rows of a seg
 int launch_summaries(const uint16_t* k_shared, float* summaries, const moska_shape* s,
                      cudaStream_t st);
 int launch_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
-                 const moska_shape* s, void* ws, cudaStream_t st);
+                 const moska_shape* s, void* ws, bool mark_groups, cudaStream_t st);
 int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
-                 const moska_shape* s, void* ws, cudaStream_t st);
+                 const moska_shape* s, void* ws, bool premarked, cudaStream_t st);
 int launch_group_noalloc(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
                          const moska_shape* s, cudaStream_t st);
 int launch_shared_small(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,

@@ -5,9 +5,10 @@
 // Determinism without ordered atomics: a request routes to k DIFFERENT chunks per KV head, so a
 // segment (h, c) holds each request at most once and is fully described by a bit set over the
 // requests.  Pass 1 sets bit b of row (h, c) for every routed pair (atomicOr: the result does
-// not depend on the order).  Pass 2 counts the bits per row, pass 3 scans the counts into
-// segment offsets and tile lists, pass 4 walks every row's bits in ascending request order and
-// writes the positions, looking the slot j up in the request's (ascending) chunk list.
+// not depend on the order; inside moska_decode_step the router does it while it writes its
+// picks).  Pass 2 counts the bits per row and scans the counts into segment offsets and tile
+// lists, pass 3 walks every row's bits in ascending request order and writes the positions,
+// looking the slot j up in the request's (ascending) chunk list.
 #include <mutex>
 
 #include "common.cuh"
@@ -65,7 +66,7 @@ group_mark_kernel(const int32_t* __restrict__ topk_idx, uint32_t* __restrict__ b
     atomicOr(&bitmap[((size_t)h * C + c) * words + (b >> 5)], 1u << (b & 31));
 }
 
-// Pass 2: requests per key.
+// Requests per key, for shapes whose bit sets are too wide to be counted inside the scan.
 __global__ void __launch_bounds__(256)
 group_count_kernel(const uint32_t* __restrict__ bitmap, int32_t* __restrict__ totals, int n_keys,
                    int words)
@@ -83,7 +84,8 @@ group_count_kernel(const uint32_t* __restrict__ bitmap, int32_t* __restrict__ to
 // remainder of at least big_min_entries), then to 16-row tiles, and a last piece of at most
 // tiny_entries requests (8 rows) to the 8-row tile list.
 __global__ void __launch_bounds__(1024)
-group_scan_kernel(const int32_t* __restrict__ totals, int32_t* __restrict__ seg_offsets,
+group_scan_kernel(const uint32_t* __restrict__ bitmap, int words, const int32_t* __restrict__ totals,
+                  int32_t* __restrict__ seg_offsets,
                   WsHeader* __restrict__ hdr, TileItem* __restrict__ small_items,
                   TileItem* __restrict__ tiny_items, TileItem* __restrict__ big_items, int n_keys,
                   int small_entries, int tiny_entries, int big_entries, int big_min_entries)
@@ -101,7 +103,12 @@ group_scan_kernel(const int32_t* __restrict__ totals, int32_t* __restrict__ seg_
     __syncthreads();
     for (int base = 0; base < n_keys; base += blockDim.x) {
         const int key = base + threadIdx.x;
-        const int n = key < n_keys ? totals[key] : 0;
+        int n = 0;  // requests of this key: counted beforehand, or the population count of its bits
+        if (key < n_keys) {
+            if (totals != nullptr) n = totals[key];
+            else
+                for (int w = 0; w < words; ++w) n += __popc(bitmap[(size_t)key * words + w]);
+        }
         int n_big = n / big_entries;
         int rem = n - n_big * big_entries;
         if (rem >= big_min_entries) {
@@ -211,27 +218,31 @@ group_emit_kernel(const int32_t* __restrict__ topk_idx, const uint32_t* __restri
 }  // namespace
 
 int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
-                 const moska_shape* s, void* ws, cudaStream_t st)
+                 const moska_shape* s, void* ws, bool premarked, cudaStream_t st)
 {
     const WsLayout lay = ws_layout(s);
     char* base = static_cast<char*>(ws);
     WsHeader* hdr = reinterpret_cast<WsHeader*>(base);
     uint32_t* bitmap = reinterpret_cast<uint32_t*>(base + lay.off_hist);
-    int32_t* totals = reinterpret_cast<int32_t*>(base + lay.off_totals);
     TileItem* small_items = reinterpret_cast<TileItem*>(base + lay.off_small);
     TileItem* big_items = reinterpret_cast<TileItem*>(base + lay.off_big);
     TileItem* tiny_items = reinterpret_cast<TileItem*>(base + lay.off_tiny);
     const long long P = (long long)s->B * s->Hkv * s->k;
-    // header and bit sets must start at zero
-    MOSKA_CUDA_TRY(cudaMemsetAsync(base, 0, lay.off_totals, st));
-    if (P > 0) {
+    // header and bit sets must start at zero; the router has done both passes already when the
+    // two calls run back to back inside moska_decode_step
+    if (!premarked) MOSKA_CUDA_TRY(cudaMemsetAsync(base, 0, lay.off_totals, st));
+    if (!premarked && P > 0) {
         group_mark_kernel<<<(unsigned)((P + 255) / 256), 256, 0, st>>>(topk_idx, bitmap, hdr, P,
                                                                        s->Hkv, s->C, s->k, lay.words);
         MOSKA_LAUNCH_CHECK("group_mark_kernel");
     }
-    group_count_kernel<<<(lay.n_keys + 255) / 256, 256, 0, st>>>(bitmap, totals, lay.n_keys, lay.words);
-    MOSKA_LAUNCH_CHECK("group_count_kernel");
-    group_scan_kernel<<<1, 1024, 0, st>>>(totals, seg_offsets, hdr, small_items, tiny_items, big_items,
+    int32_t* totals = nullptr;
+    if (lay.words > 2) {  // wide bit sets: count them with a whole grid, not with the scan's one CTA
+        totals = reinterpret_cast<int32_t*>(base + lay.off_totals);
+        group_count_kernel<<<(lay.n_keys + 255) / 256, 256, 0, st>>>(bitmap, totals, lay.n_keys, lay.words);
+        MOSKA_LAUNCH_CHECK("group_count_kernel");
+    }
+    group_scan_kernel<<<1, 1024, 0, st>>>(bitmap, lay.words, totals, seg_offsets, hdr, small_items, tiny_items, big_items,
                                           lay.n_keys, lay.small_entries, lay.tiny_entries,
                                           lay.big_entries, lay.big_min_entries);
     MOSKA_LAUNCH_CHECK("group_scan_kernel");
@@ -280,7 +291,7 @@ int launch_group_noalloc(const int32_t* topk_idx, int32_t* seg_offsets, int32_t*
     }
     // launch_group clears the header and the bit sets itself, so the previous call's contents
     // never leak into this one.
-    return launch_group(topk_idx, seg_offsets, seg_entries, s, scratch, st);
+    return launch_group(topk_idx, seg_offsets, seg_entries, s, scratch, false, st);
 }
 
 }  // namespace moska

@@ -24,7 +24,7 @@ template <int D>
 __global__ void __launch_bounds__(256)
 route_kernel(const uint16_t* __restrict__ q, const float* __restrict__ summaries,
              int32_t* __restrict__ topk_idx, float* __restrict__ topk_score, int B, int Hq,
-             int Hkv, int C, int k)
+             int Hkv, int C, int k, uint32_t* __restrict__ mark, int mark_words)
 {
     constexpr int PITCH = D + 4;  // floats; 16-byte aligned rows, conflict-free float4 reads
     extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -122,6 +122,8 @@ route_kernel(const uint16_t* __restrict__ q, const float* __restrict__ summaries
             const int c = wd * 32 + lane;
             topk_idx[out_base + pos] = c;
             if (topk_score) topk_score[out_base + pos] = sc[c];
+            // first pass of the grouping, done here when the caller runs both back to back
+            if (mark) atomicOr(&mark[((size_t)h * C + c) * mark_words + (b >> 5)], 1u << (b & 31));
         }
         written += __popc(bits);
     }
@@ -231,7 +233,8 @@ __device__ __forceinline__ uint32_t sortable(float s)
 
 __global__ void __launch_bounds__(256)
 route_select_kernel(const float* __restrict__ scores, int32_t* __restrict__ topk_idx,
-                    float* __restrict__ topk_score, long long rows, int C, int k)
+                    float* __restrict__ topk_score, long long rows, int C, int k, int Hkv,
+                    uint32_t* __restrict__ mark, int mark_words)
 {
     __shared__ int hist[8][256];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -300,6 +303,10 @@ route_select_kernel(const float* __restrict__ scores, int32_t* __restrict__ topk
             const int pos = written + __popc(take_bits & ((1u << lane) - 1u));
             topk_idx[out_base + pos] = c;
             if (topk_score) topk_score[out_base + pos] = s;
+            if (mark) {
+                const int b = (int)(row / Hkv), h = (int)(row % Hkv);
+                atomicOr(&mark[((size_t)h * C + c) * mark_words + (b >> 5)], 1u << (b & 31));
+            }
         }
         written += __popc(take_bits);
         ties_seen += __popc(eq_bits);
@@ -316,8 +323,18 @@ size_t route_smem_bytes(int D, int C, int n_warps)
 }  // namespace
 
 int launch_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
-                 const moska_shape* s, void* ws, cudaStream_t st)
+                 const moska_shape* s, void* ws, bool mark_groups, cudaStream_t st)
 {
+    // mark_groups: also do the first grouping pass (set bit b of row (h, chunk) for every routed
+    // pair) into the workspace, which is cleared here; launch_group is then told to skip it
+    uint32_t* mark = nullptr;
+    int mark_words = 0;
+    if (mark_groups) {
+        const WsLayout lay = ws_layout(s);
+        MOSKA_CUDA_TRY(cudaMemsetAsync(ws, 0, lay.off_totals, st));
+        mark = reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + lay.off_hist);
+        mark_words = lay.words;
+    }
     if ((long long)s->B * s->Hkv == 0) return MOSKA_OK;
     // many chunks: tiled product into the workspace + selection; else one warp per request with
     // the scores in shared memory
@@ -348,8 +365,8 @@ int launch_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, f
         }
         MOSKA_LAUNCH_CHECK("route_score_kernel");
         const long long rows = (long long)s->B * s->Hkv;
-        route_select_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(scores, topk_idx, topk_score, rows,
-                                                                        s->C, s->k);
+        route_select_kernel<<<(unsigned)((rows + 7) / 8), 256, 0, st>>>(
+            scores, topk_idx, topk_score, rows, s->C, s->k, s->Hkv, mark, mark_words);
         MOSKA_LAUNCH_CHECK("route_select_kernel");
         return MOSKA_OK;
     }
@@ -363,12 +380,12 @@ int launch_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, f
         MOSKA_CUDA_TRY(cudaFuncSetAttribute(route_kernel<128>,
                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         route_kernel<128><<<(unsigned)grid, n_warps * 32, smem, st>>>(
-            q, summaries, topk_idx, topk_score, s->B, s->Hq, s->Hkv, s->C, s->k);
+            q, summaries, topk_idx, topk_score, s->B, s->Hq, s->Hkv, s->C, s->k, mark, mark_words);
     } else {
         MOSKA_CUDA_TRY(cudaFuncSetAttribute(route_kernel<64>,
                                             cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         route_kernel<64><<<(unsigned)grid, n_warps * 32, smem, st>>>(
-            q, summaries, topk_idx, topk_score, s->B, s->Hq, s->Hkv, s->C, s->k);
+            q, summaries, topk_idx, topk_score, s->B, s->Hq, s->Hkv, s->C, s->k, mark, mark_words);
     }
     MOSKA_LAUNCH_CHECK("route_kernel");
     return MOSKA_OK;
