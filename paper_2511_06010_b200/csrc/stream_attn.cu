@@ -65,6 +65,38 @@ unique_attn_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ 
     attend_stream<D, 1>(rows, kb, vb, stride, t0, t1, scale, sm);
 }
 
+// ---- Unique KV Attention with K/V staged through shared memory (D = 128) -------------------------
+__global__ void __launch_bounds__(kThreads, 2)
+unique_staged_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_unique,
+                     const uint16_t* __restrict__ v_unique, const int64_t* __restrict__ kv_start,
+                     const int32_t* __restrict__ kv_len, float* __restrict__ o_part,
+                     float* __restrict__ lse_part, float scale, int Hq, int Hkv, int n_splits,
+                     int slot0, int n_slots)
+{
+    constexpr int D = 128;
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ TileRows<1> rows;
+    const int G = Hq / Hkv;
+    const int h = blockIdx.x % Hkv;
+    const int s = (blockIdx.x / Hkv) % n_splits;
+    const int b = blockIdx.x / (Hkv * n_splits);
+    clear_rows(rows);
+    __syncthreads();
+    if (threadIdx.x < G) {
+        const int64_t r = (int64_t)b * Hq + h * G + threadIdx.x;
+        rows.q[threadIdx.x] = q + r * D;
+        rows.o[threadIdx.x] = o_part + (r * n_slots + slot0 + s) * D;
+        rows.lse[threadIdx.x] = lse_part + r * n_slots + slot0 + s;
+    }
+    __syncthreads();
+    int t0, t1;
+    split_range(kv_len[b], n_splits, s, t0, t1);
+    const int64_t stride = (int64_t)Hkv * D;
+    const uint16_t* kb = k_unique + kv_start[b] * stride + (int64_t)h * D;
+    const uint16_t* vb = v_unique + kv_start[b] * stride + (int64_t)h * D;
+    attend_stream_staged(rows, kb, vb, stride, t0, t1, scale, ring);
+}
+
 // ---- per-request GEMV baseline over shared chunks: one CTA per (request, KV head, slot) ---------
 template <int D>
 __global__ void __launch_bounds__(kThreads, 3)
@@ -175,6 +207,17 @@ int launch_unique(const uint16_t* q, const uint16_t* k_unique, const uint16_t* v
     const long long grid = (long long)s->B * s->Hkv * s->n_unique_splits;
     if (grid == 0) return MOSKA_OK;
     if (grid > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "unique attention grid too large");
+    if (s->D == 128) {
+        constexpr int kRing = kWarps * kStagedWarpBytes;
+        static_assert(kRing >= (int)sizeof(CombineSmem<128, 1>), "the combine step reuses the ring");
+        MOSKA_CUDA_TRY(cudaFuncSetAttribute(unique_staged_kernel,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kRing));
+        unique_staged_kernel<<<(unsigned)grid, kThreads, kRing, st>>>(
+            q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part, scale, s->Hq, s->Hkv,
+            s->n_unique_splits, s->shared_slots, n_slots);
+        MOSKA_LAUNCH_CHECK("unique_staged_kernel");
+        return MOSKA_OK;
+    }
     if (s->D == 128)
         unique_attn_kernel<128><<<(unsigned)grid, kThreads, 0, st>>>(
             q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part, scale, s->Hq, s->Hkv,

@@ -291,5 +291,213 @@ __device__ __forceinline__ void attend_stream(const TileRows<NT>& rows, const ui
     }
 }
 
+// ---- the same block with K/V staged through shared memory ---------------------------------------
+// attend_stream keeps the next tile's K/V in registers while it is in flight: the bytes a SM has
+// in flight are bounded by its register file, and the 64-byte pieces of a K row that one load
+// instruction fetches rely on L1 to be merged into whole lines.  Here a warp copies whole token
+// rows (256 contiguous bytes per 16 lanes, cp.async.cg: L2 -> shared memory, no L1) into its own
+// ring of tiles, kStagedDepth tiles ahead, and builds the MMA fragments from shared memory.
+// The 16-byte chunks of token row t are stored at chunk ^ (t & 7), and the head dimension is
+// assigned to the fragment registers such that every 16-byte shared load of a quarter warp hits
+// eight different chunk positions (K: lane c owns chunks 2c, 2c+1 of each 128-byte half row;
+// V: lane group g owns chunk g of each half row) -- no bank conflicts, no ldmatrix.
+// Twice the bytes in flight per SM, fewer registers, and no dependence on the L1 / shared-memory
+// carve-out: the kernel keeps its bandwidth when CTAs with large shared memory share the SM.
+constexpr int kStagedDepth = 3;                                  // tiles in flight per warp
+constexpr int kStagedTileBytes = 2 * kTileTokens * 256;          // K and V of one 16-token tile, D = 128
+constexpr int kStagedWarpBytes = kStagedDepth * kStagedTileBytes;
+
+__device__ __forceinline__ void cp_async16(uint32_t smem_dst, const void* src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_dst), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait()
+{
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ uint4 lds16(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "r"(addr));
+    return v;
+}
+
+// D = 128, one 8-row column block (NT = 1), the kWarps warps of the CTA take interleaved tiles.
+// `ring` is the CTA's staging memory (kWarps * kStagedWarpBytes bytes, 128-byte aligned); the
+// final combination of the warps reuses it.
+__device__ __forceinline__ void attend_stream_staged(const TileRows<1>& rows, const uint16_t* k_base,
+                                                     const uint16_t* v_base, int64_t tok_stride,
+                                                     int t_begin, int t_end, float scale,
+                                                     unsigned char* ring)
+{
+    constexpr int D = 128, KU = 4, VL = 2, MT = 8;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, c = lane & 3;
+    const float sl2 = scale * kLog2e;
+    // 16-byte chunk of a token row that lane c consumes as its u-th K piece
+    auto k_chunk = [&](int u) { return 2 * c + (u & 1) + 8 * (u >> 1); };
+
+    uint4 qf[KU];  // Q as the B operand, in the same head-dimension order as the K pieces
+    {
+        const uint16_t* qp = rows.q[g];
+#pragma unroll
+        for (int u = 0; u < KU; ++u) qf[u] = qp ? ldg16(qp + 8 * k_chunk(u)) : make_uint4(0, 0, 0, 0);
+    }
+    float oacc[MT][4];
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) oacc[mt][0] = oacc[mt][1] = oacc[mt][2] = oacc[mt][3] = 0.f;
+
+    const int n_tok = t_end - t_begin;
+    const int n_tiles = (n_tok + kTileTokens - 1) / kTileTokens;
+    const int last_tok = t_end - 1;
+    const int my_tiles = n_tiles > warp ? (n_tiles - warp + kWarps - 1) / kWarps : 0;
+    const uint32_t ring_base = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + warp * kStagedWarpBytes;
+    // chunk `ch` of token row `t` (0..15) of the K (kv = 0) or V (kv = 1) tile in ring stage s
+    auto slot = [&](int s, int kv, int t, int ch) {
+        return ring_base + s * kStagedTileBytes + kv * (kTileTokens * 256) + t * 256 + ((ch ^ (t & 7)) << 4);
+    };
+    // cooperative copy of the i-th tile of this warp: 16 lanes per token row, two rows per instruction
+    auto issue = [&](int i) {
+        const int s = i % kStagedDepth;
+        const int t0 = t_begin + (warp + i * kWarps) * kTileTokens;
+        const int ch = lane & 15;
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int t = 2 * it + (lane >> 4);
+            const int64_t off = (int64_t)min(t0 + t, last_tok) * tok_stride + 8 * ch;
+            cp_async16(slot(s, 0, t, ch), k_base + off);
+            cp_async16(slot(s, 1, t, ch), v_base + off);
+        }
+    };
+#pragma unroll
+    for (int i = 0; i < kStagedDepth; ++i) {
+        if (i < my_tiles) issue(i);
+        cp_async_commit();  // one group per ring stage, empty ones included
+    }
+
+    for (int i = 0; i < my_tiles; ++i) {
+        const int s = i % kStagedDepth;
+        const int t0 = t_begin + (warp + i * kWarps) * kTileTokens;
+        cp_async_wait<kStagedDepth - 1>();  // this lane's copies of tile i have landed ...
+        __syncwarp();                       // ... and so have the other lanes'
+        uint4 kA[KU], kB[KU];               // K rows of tokens g and g+8
+#pragma unroll
+        for (int u = 0; u < KU; ++u) {
+            kA[u] = lds16(slot(s, 0, g, k_chunk(u)));
+            kB[u] = lds16(slot(s, 0, g + 8, k_chunk(u)));
+        }
+        float sc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int u = 0; u < KU; ++u) {
+            mma_bf16_16816(sc, kA[u].x, kB[u].x, kA[u].y, kB[u].y, qf[u].x, qf[u].y);
+            mma_bf16_16816(sc, kA[u].z, kB[u].z, kA[u].w, kB[u].w, qf[u].z, qf[u].w);
+        }
+        const bool va = (t0 + g) <= last_tok, vb = (t0 + 8 + g) <= last_tok;
+        if (!va) sc[0] = sc[1] = -INFINITY;
+        if (!vb) sc[2] = sc[3] = -INFINITY;
+        float mx0 = fmaxf(sc[0], sc[2]), mx1 = fmaxf(sc[1], sc[3]);
+#pragma unroll
+        for (int off = 4; off < 32; off <<= 1) {
+            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+        }
+        const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
+        const bool grew = (mn0 > m_run[0]) | (mn1 > m_run[1]);
+        const float al0 = fast_exp2((m_run[0] - mn0) * sl2), al1 = fast_exp2((m_run[1] - mn1) * sl2);
+        m_run[0] = mn0;
+        m_run[1] = mn1;
+        const float ms0 = mn0 * sl2, ms1 = mn1 * sl2;
+        const float p0 = fast_exp2(fmaf(sc[0], sl2, -ms0)), p1 = fast_exp2(fmaf(sc[1], sl2, -ms1));
+        const float p2 = fast_exp2(fmaf(sc[2], sl2, -ms0)), p3 = fast_exp2(fmaf(sc[3], sl2, -ms1));
+        l_run[0] = fmaf(l_run[0], al0, p0 + p2);
+        l_run[1] = fmaf(l_run[1], al1, p1 + p3);
+        const uint32_t pb0 = movmatrix_trans(pack_bf16(p0, p1));
+        const uint32_t pb1 = movmatrix_trans(pack_bf16(p2, p3));
+        if (__any_sync(0xffffffffu, grew)) {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                oacc[mt][0] *= al0;
+                oacc[mt][1] *= al1;
+                oacc[mt][2] *= al0;
+                oacc[mt][3] *= al1;
+            }
+        }
+        uint4 vr[4][VL];  // V rows of tokens 2c, 2c+1, 2c+8, 2c+9: chunk g of each half row
+#pragma unroll
+        for (int r = 0; r < 4; ++r)
+#pragma unroll
+            for (int j = 0; j < VL; ++j)
+                vr[r][j] = lds16(slot(s, 1, 2 * c + (r & 1) + 8 * (r >> 1), g + 8 * j));
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            const int e0 = mt, e1 = MT + mt;
+            const uint32_t sel0 = (e0 & 1) ? 0x7632u : 0x5410u;
+            const uint32_t sel1 = (e1 & 1) ? 0x7632u : 0x5410u;
+            auto word = [&](int r, int e) -> uint32_t {
+                const uint4& x = vr[r][e >> 3];
+                const int w = (e & 7) >> 1;
+                return w == 0 ? x.x : (w == 1 ? x.y : (w == 2 ? x.z : x.w));
+            };
+            const uint32_t a0 = __byte_perm(word(0, e0), word(1, e0), sel0);
+            const uint32_t a1 = __byte_perm(word(0, e1), word(1, e1), sel1);
+            const uint32_t a2 = __byte_perm(word(2, e0), word(3, e0), sel0);
+            const uint32_t a3 = __byte_perm(word(2, e1), word(3, e1), sel1);
+            mma_bf16_16816(oacc[mt], a0, a1, a2, a3, pb0, pb1);
+        }
+        __syncwarp();  // every lane has read the stage into registers: refill it
+        if (i + kStagedDepth < my_tiles) issue(i + kStagedDepth);
+        cp_async_commit();
+    }
+    cp_async_wait<0>();
+
+    // ---- combine the warps through the (now idle) staging memory
+#pragma unroll
+    for (int off = 4; off < 32; off <<= 1) {
+        l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], off);
+        l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], off);
+    }
+    __syncthreads();  // every warp has left its ring
+    CombineSmem<D, 1>& sm = *reinterpret_cast<CombineSmem<D, 1>*>(ring);
+    if (g == 0) {
+        sm.m[warp][2 * c] = m_run[0];
+        sm.m[warp][2 * c + 1] = m_run[1];
+        sm.l[warp][2 * c] = l_run[0];
+        sm.l[warp][2 * c + 1] = l_run[1];
+    }
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+        const int d0 = v_dim_of(g, mt), d1 = v_dim_of(g, MT + mt);
+        sm.o[warp][2 * c][d0] = oacc[mt][0];
+        sm.o[warp][2 * c + 1][d0] = oacc[mt][1];
+        sm.o[warp][2 * c][d1] = oacc[mt][2];
+        sm.o[warp][2 * c + 1][d1] = oacc[mt][3];
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < 8 * D; i += kThreads) {
+        const int r = i / D, d = i % D;
+        float* orow = rows.o[r];
+        if (orow == nullptr) continue;
+        float M = sm.m[0][r];
+#pragma unroll
+        for (int w = 1; w < kWarps; ++w) M = fmaxf(M, sm.m[w][r]);
+        float num = 0.f, den = 0.f;
+        if (M != -INFINITY) {
+#pragma unroll
+            for (int w = 0; w < kWarps; ++w) {
+                const float a = fast_exp2((sm.m[w][r] - M) * sl2);
+                num = fmaf(a, sm.o[w][r][d], num);
+                den = fmaf(a, sm.l[w][r], den);
+            }
+        }
+        orow[d] = den > 0.f ? num / den : 0.f;
+        if (d == 0) rows.lse[r][0] = den > 0.f ? M * scale + logf(den) : -INFINITY;
+    }
+}
+
 }  // namespace stream
 }  // namespace moska

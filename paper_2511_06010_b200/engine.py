@@ -42,12 +42,10 @@ class MoskaLayer:
         ws_bytes = M.workspace_bytes(self.shape)
         self.ws = torch.empty(max(ws_bytes, 256), dtype=torch.uint8, device=dev)
         self.side_stream: Optional[torch.cuda.Stream] = None
-        # Routing and grouping can run on a second, high-priority stream beside unique attention.
-        # That only pays for the small-C router: the tiled router's CTAs (51 KB of shared memory
-        # each) make the SMs switch to a large shared-memory carve-out while they are resident,
-        # which leaves unique attention too little L1 for its loads in flight (measured: up to
-        # 40 % slower), more than the overlap saves.
-        self.overlap_routing = (not dense) and C <= 256
+        # Routing, grouping and the streaming shared-attention tiles run on a second, high-priority
+        # stream beside unique attention (which stages K/V through shared memory and therefore
+        # keeps its bandwidth whatever shares the SM with it).
+        self.overlap_routing = not dense
 
     # -- offline ---------------------------------------------------------------------------------
     def build_summaries(self, k_shared):
