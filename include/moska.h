@@ -63,6 +63,10 @@ typedef struct moska_shape {
                              /* in dense mode (no routing) the C chunks are cut into this many   */
                              /* runs of ceil(C / shared_slots) consecutive chunks                */
     int32_t n_unique_splits; /* partial slots written by unique attention (split-K), >= 1        */
+    int64_t unique_tokens;   /* optional hint: the private tokens of all requests together, if   */
+                             /* the host knows them, else 0.  Only moska_decode_step reads it,   */
+                             /* to divide the SMs between shared and unique attention; results   */
+                             /* never depend on it                                               */
 } moska_shape;
 
 typedef void* moska_stream; /* a cudaStream_t */
@@ -228,15 +232,14 @@ void moska_profiler_destroy(moska_profiler* prof);
 int moska_profiler_read(moska_profiler* prof, float* stage_ms, int32_t* n_steps);
 
 /*
- * One whole decode step on device buffers: route -> group -> unique -> shared -> merge.  Without
- * `side_stream` everything runs in that order on `stream`.  With it, the short routing and
- * grouping kernels run on `side_stream` beside unique attention; both are ordered after the work
- * already on `stream`; shared attention and the merge follow on `stream` once both are done.
- * Create `side_stream` with a HIGHER priority than `stream`, or the routing kernels queue behind
- * the CTAs of unique attention.  The overlap pays while the router's shared-memory footprint
- * (4 bytes per chunk and warp) is small; with thousands of chunks the SMs switch to a large
- * shared-memory carve-out while both run, which leaves unique attention too little L1 for its
- * loads in flight (measured: up to 40 % slower) -- pass side_stream = NULL then.
+ * One whole decode step on device buffers.  Without `side_stream` everything runs on `stream`
+ * in the order route, group, unique, shared, merge.  With it, unique attention is enqueued first
+ * on `stream`; route, group and shared attention follow on `side_stream` (both ordered after the
+ * work already on `stream`), and the merge waits for both.  `side_stream` must have a HIGHER
+ * priority than `stream`: its CTAs then take SMs over as unique-attention CTAs retire.  The
+ * persistent tensor-core kernel of shared attention is given only a share of the SMs (derived
+ * from the two kernels' estimated work, see shape->unique_tokens), so the HBM-bound unique
+ * attention keeps running on the others: the two resource profiles overlap on one GPU.
  * Dense mode (no routing) when summaries == NULL.
  * Scratch buffers topk_idx [B*Hkv*k], seg_offsets [Hkv*C+1], seg_entries [B*Hkv*k], o_part,
  * lse_part and ws are caller-owned as in the individual calls.  `prof` may be NULL; otherwise

@@ -25,7 +25,8 @@ _lib = ctypes.CDLL(LIB_PATH)
 
 class MoskaShape(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
-                ("B", "Hq", "Hkv", "D", "C", "L", "k", "shared_slots", "n_unique_splits")]
+                ("B", "Hq", "Hkv", "D", "C", "L", "k", "shared_slots", "n_unique_splits")] + \
+               [("unique_tokens", ctypes.c_int64)]
 
 
 class MoskaError(RuntimeError):
@@ -68,7 +69,7 @@ for _name, (_res, _args) in EXPORTS.items():
 
 def shape(B, Hq, Hkv, D, C, L, k, shared_slots=None, n_unique_splits=1) -> MoskaShape:
     return MoskaShape(B, Hq, Hkv, D, C, L, k, k if shared_slots is None else shared_slots,
-                      n_unique_splits)
+                      n_unique_splits, 0)
 
 
 def _ptr(t) -> Optional[int]:

@@ -136,6 +136,31 @@ int moska_build_chunk_summaries(const uint16_t* k_shared, float* summaries,
 }
 
 namespace {
+// SMs the persistent tensor-core kernel gets when it runs beside unique attention: both kernels'
+// work is estimated (tensor-core items from the shape, unique attention from the token hint at
+// 7 TB/s) and the SMs are divided so that neither waits for the other.  Unique attention reaches
+// most of the HBM bandwidth from about 96 SMs; if it is the longer job the tensor-core kernel
+// hides entirely on the remaining ones.
+int tc_sm_share(const moska_shape* s, bool dense)
+{
+    int dev = 0, n_sms = 148;
+    if (cudaGetDevice(&dev) == cudaSuccess)
+        cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev);
+    const double a = shared_tc_cost_sm_ms(s, dense);  // SM * ms
+    int x;
+    if (s->unique_tokens <= 0) {
+        x = dense ? (n_sms * 4) / 5 : (n_sms * 35) / 100;  // no hint: tensor-heavy / HBM-heavy guess
+    } else {
+        const double b = (double)s->unique_tokens * s->Hkv * 4.0 * s->D / 7.0e9;  // ms
+        const int hbm_sms = (n_sms * 65) / 100;
+        if (a <= b * (n_sms - hbm_sms)) x = n_sms - hbm_sms;
+        else x = (int)(a * n_sms / (a + b * 0.4 * n_sms));
+    }
+    if (x < 16) x = 16;
+    if (x > n_sms) x = n_sms;
+    return x;
+}
+
 // Validation + launch of the router; mark_groups also runs the grouping's first pass in it.
 int route_impl(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
                const moska_shape* shape, void* ws, size_t ws_bytes, bool mark_groups,
@@ -226,14 +251,14 @@ int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_
         // enough rows to fill a good part of a 128-row tile: tensor cores; else 16-row tiles
         if (tc && (long long)shape->B * (shape->Hq / shape->Hkv) >= kBigMinRows)
             return launch_shared_tc(q, k_shared, v_shared, nullptr, o_part, lse_part, softmax_scale,
-                                    shape, ws, true, st);
+                                    shape, ws, true, 0, st);
         return launch_shared_small(q, k_shared, v_shared, nullptr, o_part, lse_part, softmax_scale,
                                    shape, ws, true, st);
     }
     // routed: the grouping pass split every segment into tensor-core tiles and 16-row tiles
     if (tc)
         MOSKA_TRY(launch_shared_tc(q, k_shared, v_shared, seg_entries, o_part, lse_part,
-                                   softmax_scale, shape, ws, false, st));
+                                   softmax_scale, shape, ws, false, 0, st));
     return launch_shared_small(q, k_shared, v_shared, seg_entries, o_part, lse_part, softmax_scale,
                                shape, ws, false, st);
 }
@@ -308,56 +333,87 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
 {
     const bool dense = summaries == nullptr;
     cudaStream_t st = (cudaStream_t)stream, side = (cudaStream_t)side_stream;
-    // Fork/join events for the optional second stream, created once per host thread.
-    static thread_local cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
-    if (side != nullptr && ev_fork == nullptr) {
-        MOSKA_CUDA_TRY(cudaEventCreateWithFlags(&ev_fork, cudaEventDisableTiming));
-        MOSKA_CUDA_TRY(cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming));
-    }
-    // Routing and grouping are short, latency-bound kernels: with a side stream they run beside
-    // unique attention (the caller gives that stream the higher priority, so they are not queued
-    // behind the thousands of CTAs of the unique-attention grid).  The two attention kernels each
-    // fill the GPU on their own (HBM-bound unique attention, tensor- or HBM-bound shared
-    // attention), so they run one after the other on `stream`.
-    cudaStream_t cs = side != nullptr ? side : st;
-    if (!dense) {
-        if (side != nullptr) {
-            MOSKA_CUDA_TRY(cudaEventRecord(ev_fork, st));
-            MOSKA_CUDA_TRY(cudaStreamWaitEvent(side, ev_fork, 0));
+    if (side == nullptr) {
+        // one stream: route, group, unique, shared, merge
+        if (!dense) {
+            MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 0, st));
+            // the router also sets the grouping's request bits while it writes its picks
+            MOSKA_TRY(route_impl(q, summaries, topk_idx, nullptr, shape, ws, ws_bytes, true, st));
+            MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 1, st));
+            MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 0, st));
+            MOSKA_TRY(group_impl(topk_idx, seg_offsets, seg_entries, shape, ws, ws_bytes, true, st));
+            MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 1, st));
         }
-        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 0, cs));
-        // the router also sets the grouping's request bits while it writes its picks
-        MOSKA_TRY(route_impl(q, summaries, topk_idx, nullptr, shape, ws, ws_bytes, true, cs));
-        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 1, cs));
-        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 0, cs));
-        MOSKA_TRY(group_impl(topk_idx, seg_offsets, seg_entries, shape, ws, ws_bytes, true, cs));
-        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 1, cs));
-        if (side != nullptr) {
-            // the streaming (16- and 8-row) tiles of shared attention are HBM-bound like unique
-            // attention and small in shared memory: they run beside it; only the tensor-core
-            // items wait for the main stream
-            MOSKA_TRY(launch_shared_small(q, k_shared, v_shared, seg_entries, o_part, lse_part,
-                                          softmax_scale, shape, ws, false, side));
-            MOSKA_CUDA_TRY(cudaEventRecord(ev_join, side));
-        }
-    }
-    MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 0, st));
-    MOSKA_TRY(moska_unique_attn(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part,
-                                softmax_scale, shape, st));
-    MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 1, st));
-    if (!dense && side != nullptr) MOSKA_CUDA_TRY(cudaStreamWaitEvent(st, ev_join, 0));
-    MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 0, st));
-    if (!dense && side != nullptr) {
-        if (shared_tc_supported(shape))
-            MOSKA_TRY(launch_shared_tc(q, k_shared, v_shared, seg_entries, o_part, lse_part,
-                                       softmax_scale, shape, ws, false, st));
-    } else if (!dense)
-        MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, topk_idx, seg_offsets, seg_entries,
+        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 0, st));
+        MOSKA_TRY(moska_unique_attn(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part,
+                                    softmax_scale, shape, st));
+        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 1, st));
+        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 0, st));
+        MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, dense ? nullptr : topk_idx,
+                                    dense ? nullptr : seg_offsets, dense ? nullptr : seg_entries,
                                     o_part, lse_part, softmax_scale, shape, ws, ws_bytes, st));
-    else
-        MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, nullptr, nullptr, nullptr, o_part,
-                                    lse_part, softmax_scale, shape, ws, ws_bytes, st));
-    MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, st));
+        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, st));
+    } else {
+        // Two streams.  Unique attention (HBM-bound, thousands of short-lived CTAs) is enqueued
+        // first on `stream`; everything else follows on the higher-priority side stream and takes
+        // SMs over as unique-attention CTAs retire: the short routing and grouping kernels, the
+        // streaming shared-attention tiles, and the persistent tensor-core kernel, which gets
+        // only a share of the SMs so that unique attention keeps the others and HBM stays busy
+        // while the tensor pipe works -- the single-GPU form of the paper's split into Shared-KV
+        // and Unique-KV nodes (Section III-C).
+        static thread_local cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+        if (ev_fork == nullptr) {
+            MOSKA_CUDA_TRY(cudaEventCreateWithFlags(&ev_fork, cudaEventDisableTiming));
+            MOSKA_CUDA_TRY(cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming));
+        }
+        MOSKA_TRY(check_shape(shape, !dense));
+        REQUIRE_PTR(k_shared, 128);
+        REQUIRE_PTR(v_shared, 128);
+        REQUIRE_PTR(o_part, 32);
+        REQUIRE_PTR(lse_part, 4);
+        if (dense && shape->shared_slots > shape->C)
+            return fail(MOSKA_ERR_INVALID_ARG, "dense mode needs shared_slots <= C");
+        if (!dense && shape->shared_slots != shape->k)
+            return fail(MOSKA_ERR_INVALID_ARG, "routed mode needs shared_slots == k");
+        MOSKA_CUDA_TRY(cudaEventRecord(ev_fork, st));
+        MOSKA_CUDA_TRY(cudaStreamWaitEvent(side, ev_fork, 0));
+        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 0, st));
+        MOSKA_TRY(moska_unique_attn(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part,
+                                    softmax_scale, shape, st));
+        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 1, st));
+        if (!dense) {
+            MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 0, side));
+            MOSKA_TRY(route_impl(q, summaries, topk_idx, nullptr, shape, ws, ws_bytes, true, side));
+            MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 1, side));
+            MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 0, side));
+            MOSKA_TRY(group_impl(topk_idx, seg_offsets, seg_entries, shape, ws, ws_bytes, true, side));
+            MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 1, side));
+        }
+        MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 0, side));
+        const bool tc = shared_tc_supported(shape) &&
+                        (!dense || (long long)shape->B * (shape->Hq / shape->Hkv) >= kBigMinRows);
+        // Sharing the SMs pays when unique attention runs long enough for the tensor-core kernel
+        // to start beside it (the routing chain in front of it takes a few hundred microseconds
+        // under contention); for a short unique attention the tensor-core items run after it, on
+        // all SMs.
+        const double unique_ms = (double)shape->unique_tokens * shape->Hkv * 4.0 * shape->D / 7.0e9;
+        const bool beside = tc && (dense || unique_ms >= 0.6);
+        if (tc && beside)
+            MOSKA_TRY(launch_shared_tc(q, k_shared, v_shared, dense ? nullptr : seg_entries, o_part,
+                                       lse_part, softmax_scale, shape, ws, dense,
+                                       tc_sm_share(shape, dense), side));
+        if (!dense || !tc)
+            MOSKA_TRY(launch_shared_small(q, k_shared, v_shared, dense ? nullptr : seg_entries, o_part,
+                                          lse_part, softmax_scale, shape, ws, dense, side));
+        if (beside || !tc) MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, side));
+        MOSKA_CUDA_TRY(cudaEventRecord(ev_join, side));
+        MOSKA_CUDA_TRY(cudaStreamWaitEvent(st, ev_join, 0));
+        if (tc && !beside) {
+            MOSKA_TRY(launch_shared_tc(q, k_shared, v_shared, seg_entries, o_part, lse_part,
+                                       softmax_scale, shape, ws, false, 0, st));
+            MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, st));
+        }
+    }
     MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_MERGE, 0, st));
     MOSKA_TRY(moska_merge(o_part, lse_part, out, nullptr, lse_out, shape, st));
     MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_MERGE, 1, st));

@@ -104,7 +104,9 @@ int launch_shared_small(const uint16_t* q, const uint16_t* k_shared, const uint1
 bool shared_tc_supported(const moska_shape* s);
 int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
                      const int32_t* seg_entries, float* o_part, float* lse_part, float scale,
-                     const moska_shape* s, void* ws, bool dense, cudaStream_t st);
+                     const moska_shape* s, void* ws, bool dense, int max_ctas, cudaStream_t st);
+// Estimated SM-milliseconds of the tensor-core kernel for this shape (host, pure).
+double shared_tc_cost_sm_ms(const moska_shape* s, bool dense);
 // Synchronises the device, returns the sticky status of the tensor-core kernel and clears it.
 int read_tc_status(int* out);
 int launch_unique(const uint16_t* q, const uint16_t* k_unique, const uint16_t* v_unique,

@@ -686,7 +686,7 @@ bool shared_tc_supported(const moska_shape* s) { return s->D == kD && s->L % kKv
 
 int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
                      const int32_t* seg_entries, float* o_part, float* lse_part, float scale,
-                     const moska_shape* s, void* ws, bool dense, cudaStream_t st)
+                     const moska_shape* s, void* ws, bool dense, int max_ctas, cudaStream_t st)
 {
     const int G = s->Hq / s->Hkv;
     const int per_cta = 2 * (kBigTileRows / G);
@@ -708,6 +708,7 @@ int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t
     MOSKA_CUDA_TRY(cudaGetDevice(&dev));
     MOSKA_CUDA_TRY(cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, dev));
     if (grid > n_sms) grid = n_sms;
+    if (max_ctas > 0 && grid > max_ctas) grid = max_ctas;  // the caller keeps the other SMs for another kernel
     const long long kv_rows = (long long)s->Hkv * s->C * s->L;
     if (kv_rows > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "shared store exceeds 2^31 tokens");
     CUtensorMap tm_k, tm_v;
@@ -735,6 +736,28 @@ int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t
     shared_tc_kernel<<<(unsigned)grid, kThreads, smem, st>>>(tm_k, tm_v, p);
     MOSKA_LAUNCH_CHECK("shared_tc_kernel");
     return MOSKA_OK;
+}
+
+// Measured on B200: an item costs about 6 us of fill, drain and epilogue plus 2.2 us per K/V
+// tile with two query tiles (1.1 us with one, split between the two slots).
+double shared_tc_cost_sm_ms(const moska_shape* s, bool dense)
+{
+    const int G = s->Hq / s->Hkv;
+    const int per_cta = 2 * (kBigTileRows / G);
+    double items, n_kv;
+    bool two_tiles;
+    if (dense) {
+        items = (double)s->Hkv * s->shared_slots * ((s->B + per_cta - 1) / per_cta);
+        n_kv = (double)((s->C + s->shared_slots - 1) / s->shared_slots) * (s->L / kKvTile);
+        two_tiles = s->B * G > kBigTileRows;
+    } else {
+        const double P = (double)s->B * s->Hkv * s->k;
+        const double segs = P < (double)s->Hkv * s->C ? P : (double)s->Hkv * s->C;
+        items = 0.75 * (P / per_cta + segs);
+        n_kv = s->L / kKvTile;
+        two_tiles = P / segs > kBigTileRows / G;
+    }
+    return items * (6.0 + (two_tiles ? 2.2 : 1.1) * n_kv) * 1e-3;
 }
 
 int read_tc_status(int* out)

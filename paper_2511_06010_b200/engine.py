@@ -45,7 +45,7 @@ class MoskaLayer:
         # Routing, grouping and the streaming shared-attention tiles run on a second, high-priority
         # stream beside unique attention (which stages K/V through shared memory and therefore
         # keeps its bandwidth whatever shares the SM with it).
-        self.overlap_routing = not dense
+        self.overlap_routing = True
 
     # -- offline ---------------------------------------------------------------------------------
     def build_summaries(self, k_shared):
@@ -76,7 +76,8 @@ class MoskaLayer:
 
     # -- the whole step --------------------------------------------------------------------------
     def step(self, q, k_shared, v_shared, k_unique, v_unique, kv_start, kv_len, two_streams=False,
-             prof=None):
+             prof=None, unique_tokens=0):
+        self.shape.unique_tokens = int(unique_tokens)
         two_streams = two_streams and self.overlap_routing
         if two_streams and self.side_stream is None:
             self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
@@ -88,7 +89,8 @@ class MoskaLayer:
         return self.out
 
     def step_host(self, q_host, q_dev, out_host, k_shared, v_shared, k_unique, v_unique,
-                  kv_start, kv_len, two_streams=False, prof=None):
+                  kv_start, kv_len, two_streams=False, prof=None, unique_tokens=0):
+        self.shape.unique_tokens = int(unique_tokens)
         two_streams = two_streams and self.overlap_routing
         if two_streams and self.side_stream is None:
             self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
