@@ -1,6 +1,7 @@
 // Kernels built on the streaming decode-attention block: Unique KV Attention, the unbatched
 // per-request GEMV baseline over shared chunks, and Shared KV Attention for small query tiles.
 #include <cstddef>
+#include <type_traits>
 
 #include "common.cuh"
 #include "stream_attn.cuh"
@@ -94,19 +95,21 @@ unique_staged_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict_
     const int64_t stride = (int64_t)Hkv * D;
     const uint16_t* kb = k_unique + kv_start[b] * stride + (int64_t)h * D;
     const uint16_t* vb = v_unique + kv_start[b] * stride + (int64_t)h * D;
-    attend_stream_staged(rows, kb, vb, stride, t0, t1, scale, ring);
+    attend_stream_staged<1>(rows, kb, vb, stride, t0, t1, scale, ring);
 }
 
 // ---- per-request GEMV baseline over shared chunks: one CTA per (request, KV head, slot) ---------
 template <int D>
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, D == 128 ? 2 : 3)
 gemv_baseline_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_shared,
                      const uint16_t* __restrict__ v_shared, const int32_t* __restrict__ topk_idx,
                      float* __restrict__ o_part, float* __restrict__ lse_part, float scale,
                      int Hq, int Hkv, int C, int L, int k, int shared_slots, int n_slots)
 {
+    // same streaming block as unique attention: staged through shared memory for D = 128
+    extern __shared__ __align__(128) unsigned char ring[];
     __shared__ TileRows<1> rows;
-    __shared__ CombineSmem<D, 1> sm;
+    __shared__ typename std::conditional<D == 128, int, CombineSmem<D, 1>>::type sm;
     const int G = Hq / Hkv;
     const int j = blockIdx.x % shared_slots;
     const int h = (blockIdx.x / shared_slots) % Hkv;
@@ -131,7 +134,10 @@ gemv_baseline_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict_
         tok0 = ((int64_t)h * C + c0) * L;
         n_tok = (c1 - c0) * L;
     }
-    attend_stream<D, 1>(rows, k_shared + tok0 * D, v_shared + tok0 * D, D, 0, n_tok, scale, sm);
+    if constexpr (D == 128)
+        attend_stream_staged<1>(rows, k_shared + tok0 * D, v_shared + tok0 * D, D, 0, n_tok, scale, ring);
+    else
+        attend_stream<D, 1>(rows, k_shared + tok0 * D, v_shared + tok0 * D, D, 0, n_tok, scale, sm);
 }
 
 // ---- Shared KV Attention, small tiles (Section III-A) ------------------------------------------
@@ -139,7 +145,7 @@ gemv_baseline_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict_
 // chunk's K/V is streamed once for all of them.  Dense mode: one CTA per (KV head, run of chunks,
 // group of 16/G requests).
 template <int D, int NT>
-__global__ void __launch_bounds__(kThreads, NT == 1 ? 3 : 2)
+__global__ void __launch_bounds__(kThreads, (NT == 1 && D != 128) ? 3 : 2)
 shared_small_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_shared,
                     const uint16_t* __restrict__ v_shared, const int32_t* __restrict__ seg_entries,
                     const WsHeader* __restrict__ hdr, const TileItem* __restrict__ items,
@@ -147,8 +153,11 @@ shared_small_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
                     int Hq, int Hkv, int C, int L, int k, int shared_slots, int n_slots, int dense,
                     int n_tiles_offset)
 {
+    // D = 128: K/V staged through a shared-memory ring (the combine step reuses it); D = 64: the
+    // register path with its own combine buffers
+    extern __shared__ __align__(128) unsigned char ring[];
     __shared__ TileRows<NT> rows;
-    __shared__ CombineSmem<D, NT> sm;
+    __shared__ typename std::conditional<D == 128, int, CombineSmem<D, NT>>::type sm;
     const int G = Hq / Hkv;
     const int per_tile = NT * 8 / G;  // requests per tile
     // Routed mode: the CTAs walk the device-side tile list with the grid as their stride (the
@@ -193,7 +202,10 @@ shared_small_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__
             n_tok = (c1 - c0) * L;
         }
         __syncthreads();
-        attend_stream<D, NT>(rows, k_shared + tok0 * D, v_shared + tok0 * D, D, 0, n_tok, scale, sm);
+        if constexpr (D == 128)
+            attend_stream_staged<NT>(rows, k_shared + tok0 * D, v_shared + tok0 * D, D, 0, n_tok, scale, ring);
+        else
+            attend_stream<D, NT>(rows, k_shared + tok0 * D, v_shared + tok0 * D, D, 0, n_tok, scale, sm);
     }
 }
 
@@ -209,7 +221,6 @@ int launch_unique(const uint16_t* q, const uint16_t* k_unique, const uint16_t* v
     if (grid > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "unique attention grid too large");
     if (s->D == 128) {
         constexpr int kRing = kWarps * kStagedWarpBytes;
-        static_assert(kRing >= (int)sizeof(CombineSmem<128, 1>), "the combine step reuses the ring");
         MOSKA_CUDA_TRY(cudaFuncSetAttribute(unique_staged_kernel,
                                             cudaFuncAttributeMaxDynamicSharedMemorySize, kRing));
         unique_staged_kernel<<<(unsigned)grid, kThreads, kRing, st>>>(
@@ -238,11 +249,14 @@ int launch_gemv_baseline(const uint16_t* q, const uint16_t* k_shared, const uint
     const long long grid = (long long)s->B * s->Hkv * s->shared_slots;
     if (grid == 0) return MOSKA_OK;
     if (grid > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "baseline grid too large");
-    if (s->D == 128)
-        gemv_baseline_kernel<128><<<(unsigned)grid, kThreads, 0, st>>>(
+    if (s->D == 128) {
+        constexpr int kRing = kWarps * kStagedWarpBytes;
+        MOSKA_CUDA_TRY(cudaFuncSetAttribute(gemv_baseline_kernel<128>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kRing));
+        gemv_baseline_kernel<128><<<(unsigned)grid, kThreads, kRing, st>>>(
             q, k_shared, v_shared, topk_idx, o_part, lse_part, scale, s->Hq, s->Hkv, s->C, s->L,
             s->k, s->shared_slots, n_slots);
-    else
+    } else
         gemv_baseline_kernel<64><<<(unsigned)grid, kThreads, 0, st>>>(
             q, k_shared, v_shared, topk_idx, o_part, lse_part, scale, s->Hq, s->Hkv, s->C, s->L,
             s->k, s->shared_slots, n_slots);
@@ -279,16 +293,28 @@ int launch_shared_small(const uint16_t* q, const uint16_t* k_shared, const uint1
     if (grid > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "shared attention grid too large");
     constexpr int kSmallWord = offsetof(WsHeader, n_small_tiles) / 4;
     constexpr int kTinyWord = offsetof(WsHeader, n_tiny_tiles) / 4;
+    constexpr int kRing = kWarps * kStagedWarpBytes;
 #define MOSKA_LAUNCH_SMALL(DD, NN, ITEMS, WORD)                                                        \
-    shared_small_kernel<DD, NN><<<(unsigned)grid, kThreads, 0, st>>>(                                  \
-        q, k_shared, v_shared, seg_entries, hdr, ITEMS, o_part, lse_part, scale, s->B, s->Hq, s->Hkv,  \
-        s->C, s->L, s->k, s->shared_slots, n_slots, dense ? 1 : 0, WORD)
-    if (s->D == 128) MOSKA_LAUNCH_SMALL(128, 2, items, kSmallWord);
-    else MOSKA_LAUNCH_SMALL(64, 2, items, kSmallWord);
+    do {                                                                                               \
+        if (DD == 128)                                                                                 \
+            MOSKA_CUDA_TRY(cudaFuncSetAttribute(shared_small_kernel<DD, NN>,                           \
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, kRing));  \
+        shared_small_kernel<DD, NN><<<(unsigned)grid, kThreads, DD == 128 ? kRing : 0, st>>>(          \
+            q, k_shared, v_shared, seg_entries, hdr, ITEMS, o_part, lse_part, scale, s->B, s->Hq,      \
+            s->Hkv, s->C, s->L, s->k, s->shared_slots, n_slots, dense ? 1 : 0, WORD);                  \
+    } while (0)
+    if (s->D == 128) {
+        MOSKA_LAUNCH_SMALL(128, 2, items, kSmallWord);
+    } else {
+        MOSKA_LAUNCH_SMALL(64, 2, items, kSmallWord);
+    }
     if (!dense && tiny_items != nullptr) {
         MOSKA_LAUNCH_CHECK("shared_small_kernel");
-        if (s->D == 128) MOSKA_LAUNCH_SMALL(128, 1, tiny_items, kTinyWord);
-        else MOSKA_LAUNCH_SMALL(64, 1, tiny_items, kTinyWord);
+        if (s->D == 128) {
+            MOSKA_LAUNCH_SMALL(128, 1, tiny_items, kTinyWord);
+        } else {
+            MOSKA_LAUNCH_SMALL(64, 1, tiny_items, kTinyWord);
+        }
     }
 #undef MOSKA_LAUNCH_SMALL
     MOSKA_LAUNCH_CHECK("shared_small_kernel");

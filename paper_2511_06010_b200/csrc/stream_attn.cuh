@@ -326,31 +326,39 @@ __device__ __forceinline__ uint4 lds16(uint32_t addr)
     return v;
 }
 
-// D = 128, one 8-row column block (NT = 1), the kWarps warps of the CTA take interleaved tiles.
+// D = 128, NT column blocks of 8 query rows, the kWarps warps of the CTA take interleaved tiles.
 // `ring` is the CTA's staging memory (kWarps * kStagedWarpBytes bytes, 128-byte aligned); the
-// final combination of the warps reuses it.
-__device__ __forceinline__ void attend_stream_staged(const TileRows<1>& rows, const uint16_t* k_base,
+// final combination of the warps reuses it.  All threads of the CTA must call this.
+template <int NT>
+__device__ __forceinline__ void attend_stream_staged(const TileRows<NT>& rows, const uint16_t* k_base,
                                                      const uint16_t* v_base, int64_t tok_stride,
                                                      int t_begin, int t_end, float scale,
                                                      unsigned char* ring)
 {
     constexpr int D = 128, KU = 4, VL = 2, MT = 8;
+    static_assert(sizeof(CombineSmem<D, NT>) <= kWarps * kStagedWarpBytes, "the combine step reuses the ring");
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, c = lane & 3;
     const float sl2 = scale * kLog2e;
     // 16-byte chunk of a token row that lane c consumes as its u-th K piece
     auto k_chunk = [&](int u) { return 2 * c + (u & 1) + 8 * (u >> 1); };
 
-    uint4 qf[KU];  // Q as the B operand, in the same head-dimension order as the K pieces
-    {
-        const uint16_t* qp = rows.q[g];
+    uint4 qf[NT][KU];  // Q as the B operand, in the same head-dimension order as the K pieces
 #pragma unroll
-        for (int u = 0; u < KU; ++u) qf[u] = qp ? ldg16(qp + 8 * k_chunk(u)) : make_uint4(0, 0, 0, 0);
+    for (int n = 0; n < NT; ++n) {
+        const uint16_t* qp = rows.q[n * 8 + g];
+#pragma unroll
+        for (int u = 0; u < KU; ++u) qf[n][u] = qp ? ldg16(qp + 8 * k_chunk(u)) : make_uint4(0, 0, 0, 0);
     }
-    float oacc[MT][4];
-    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    float oacc[NT][MT][4];
+    float m_run[NT][2], l_run[NT][2];
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt) oacc[mt][0] = oacc[mt][1] = oacc[mt][2] = oacc[mt][3] = 0.f;
+    for (int n = 0; n < NT; ++n) {
+        m_run[n][0] = m_run[n][1] = -INFINITY;
+        l_run[n][0] = l_run[n][1] = 0.f;
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) oacc[n][mt][0] = oacc[n][mt][1] = oacc[n][mt][2] = oacc[n][mt][3] = 0.f;
+    }
 
     const int n_tok = t_end - t_begin;
     const int n_tiles = (n_tok + kTileTokens - 1) / kTileTokens;
@@ -391,41 +399,55 @@ __device__ __forceinline__ void attend_stream_staged(const TileRows<1>& rows, co
             kA[u] = lds16(slot(s, 0, g, k_chunk(u)));
             kB[u] = lds16(slot(s, 0, g + 8, k_chunk(u)));
         }
-        float sc[4] = {0.f, 0.f, 0.f, 0.f};
+        float sc[NT][4];
+#pragma unroll
+        for (int n = 0; n < NT; ++n) sc[n][0] = sc[n][1] = sc[n][2] = sc[n][3] = 0.f;
 #pragma unroll
         for (int u = 0; u < KU; ++u) {
-            mma_bf16_16816(sc, kA[u].x, kB[u].x, kA[u].y, kB[u].y, qf[u].x, qf[u].y);
-            mma_bf16_16816(sc, kA[u].z, kB[u].z, kA[u].w, kB[u].w, qf[u].z, qf[u].w);
+#pragma unroll
+            for (int n = 0; n < NT; ++n) {
+                mma_bf16_16816(sc[n], kA[u].x, kB[u].x, kA[u].y, kB[u].y, qf[n][u].x, qf[n][u].y);
+                mma_bf16_16816(sc[n], kA[u].z, kB[u].z, kA[u].w, kB[u].w, qf[n][u].z, qf[n][u].w);
+            }
         }
         const bool va = (t0 + g) <= last_tok, vb = (t0 + 8 + g) <= last_tok;
-        if (!va) sc[0] = sc[1] = -INFINITY;
-        if (!vb) sc[2] = sc[3] = -INFINITY;
-        float mx0 = fmaxf(sc[0], sc[2]), mx1 = fmaxf(sc[1], sc[3]);
+        uint32_t pb0[NT], pb1[NT];
+        bool grew = false;
+        float alpha[NT][2];
 #pragma unroll
-        for (int off = 4; off < 32; off <<= 1) {
-            mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
-            mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+        for (int n = 0; n < NT; ++n) {
+            if (!va) sc[n][0] = sc[n][1] = -INFINITY;
+            if (!vb) sc[n][2] = sc[n][3] = -INFINITY;
+            float mx0 = fmaxf(sc[n][0], sc[n][2]), mx1 = fmaxf(sc[n][1], sc[n][3]);
+#pragma unroll
+            for (int off = 4; off < 32; off <<= 1) {
+                mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, off));
+                mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, off));
+            }
+            const float mn0 = fmaxf(m_run[n][0], mx0), mn1 = fmaxf(m_run[n][1], mx1);
+            grew |= (mn0 > m_run[n][0]) | (mn1 > m_run[n][1]);
+            alpha[n][0] = fast_exp2((m_run[n][0] - mn0) * sl2);
+            alpha[n][1] = fast_exp2((m_run[n][1] - mn1) * sl2);
+            m_run[n][0] = mn0;
+            m_run[n][1] = mn1;
+            const float ms0 = mn0 * sl2, ms1 = mn1 * sl2;
+            const float p0 = fast_exp2(fmaf(sc[n][0], sl2, -ms0)), p1 = fast_exp2(fmaf(sc[n][1], sl2, -ms1));
+            const float p2 = fast_exp2(fmaf(sc[n][2], sl2, -ms0)), p3 = fast_exp2(fmaf(sc[n][3], sl2, -ms1));
+            l_run[n][0] = fmaf(l_run[n][0], alpha[n][0], p0 + p2);
+            l_run[n][1] = fmaf(l_run[n][1], alpha[n][1], p1 + p3);
+            pb0[n] = movmatrix_trans(pack_bf16(p0, p1));
+            pb1[n] = movmatrix_trans(pack_bf16(p2, p3));
         }
-        const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
-        const bool grew = (mn0 > m_run[0]) | (mn1 > m_run[1]);
-        const float al0 = fast_exp2((m_run[0] - mn0) * sl2), al1 = fast_exp2((m_run[1] - mn1) * sl2);
-        m_run[0] = mn0;
-        m_run[1] = mn1;
-        const float ms0 = mn0 * sl2, ms1 = mn1 * sl2;
-        const float p0 = fast_exp2(fmaf(sc[0], sl2, -ms0)), p1 = fast_exp2(fmaf(sc[1], sl2, -ms1));
-        const float p2 = fast_exp2(fmaf(sc[2], sl2, -ms0)), p3 = fast_exp2(fmaf(sc[3], sl2, -ms1));
-        l_run[0] = fmaf(l_run[0], al0, p0 + p2);
-        l_run[1] = fmaf(l_run[1], al1, p1 + p3);
-        const uint32_t pb0 = movmatrix_trans(pack_bf16(p0, p1));
-        const uint32_t pb1 = movmatrix_trans(pack_bf16(p2, p3));
         if (__any_sync(0xffffffffu, grew)) {
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt) {
-                oacc[mt][0] *= al0;
-                oacc[mt][1] *= al1;
-                oacc[mt][2] *= al0;
-                oacc[mt][3] *= al1;
-            }
+            for (int n = 0; n < NT; ++n)
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    oacc[n][mt][0] *= alpha[n][0];
+                    oacc[n][mt][1] *= alpha[n][1];
+                    oacc[n][mt][2] *= alpha[n][0];
+                    oacc[n][mt][3] *= alpha[n][1];
+                }
         }
         uint4 vr[4][VL];  // V rows of tokens 2c, 2c+1, 2c+8, 2c+9: chunk g of each half row
 #pragma unroll
@@ -447,7 +469,8 @@ __device__ __forceinline__ void attend_stream_staged(const TileRows<1>& rows, co
             const uint32_t a1 = __byte_perm(word(0, e1), word(1, e1), sel1);
             const uint32_t a2 = __byte_perm(word(2, e0), word(3, e0), sel0);
             const uint32_t a3 = __byte_perm(word(2, e1), word(3, e1), sel1);
-            mma_bf16_16816(oacc[mt], a0, a1, a2, a3, pb0, pb1);
+#pragma unroll
+            for (int n = 0; n < NT; ++n) mma_bf16_16816(oacc[n][mt], a0, a1, a2, a3, pb0[n], pb1[n]);
         }
         __syncwarp();  // every lane has read the stage into registers: refill it
         if (i + kStagedDepth < my_tiles) issue(i + kStagedDepth);
@@ -457,28 +480,33 @@ __device__ __forceinline__ void attend_stream_staged(const TileRows<1>& rows, co
 
     // ---- combine the warps through the (now idle) staging memory
 #pragma unroll
-    for (int off = 4; off < 32; off <<= 1) {
-        l_run[0] += __shfl_xor_sync(0xffffffffu, l_run[0], off);
-        l_run[1] += __shfl_xor_sync(0xffffffffu, l_run[1], off);
-    }
-    __syncthreads();  // every warp has left its ring
-    CombineSmem<D, 1>& sm = *reinterpret_cast<CombineSmem<D, 1>*>(ring);
-    if (g == 0) {
-        sm.m[warp][2 * c] = m_run[0];
-        sm.m[warp][2 * c + 1] = m_run[1];
-        sm.l[warp][2 * c] = l_run[0];
-        sm.l[warp][2 * c + 1] = l_run[1];
-    }
+    for (int n = 0; n < NT; ++n)
 #pragma unroll
-    for (int mt = 0; mt < MT; ++mt) {
-        const int d0 = v_dim_of(g, mt), d1 = v_dim_of(g, MT + mt);
-        sm.o[warp][2 * c][d0] = oacc[mt][0];
-        sm.o[warp][2 * c + 1][d0] = oacc[mt][1];
-        sm.o[warp][2 * c][d1] = oacc[mt][2];
-        sm.o[warp][2 * c + 1][d1] = oacc[mt][3];
+        for (int off = 4; off < 32; off <<= 1) {
+            l_run[n][0] += __shfl_xor_sync(0xffffffffu, l_run[n][0], off);
+            l_run[n][1] += __shfl_xor_sync(0xffffffffu, l_run[n][1], off);
+        }
+    __syncthreads();  // every warp has left its ring
+    CombineSmem<D, NT>& sm = *reinterpret_cast<CombineSmem<D, NT>*>(ring);
+#pragma unroll
+    for (int n = 0; n < NT; ++n) {
+        if (g == 0) {
+            sm.m[warp][n * 8 + 2 * c] = m_run[n][0];
+            sm.m[warp][n * 8 + 2 * c + 1] = m_run[n][1];
+            sm.l[warp][n * 8 + 2 * c] = l_run[n][0];
+            sm.l[warp][n * 8 + 2 * c + 1] = l_run[n][1];
+        }
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            const int d0 = v_dim_of(g, mt), d1 = v_dim_of(g, MT + mt);
+            sm.o[warp][n * 8 + 2 * c][d0] = oacc[n][mt][0];
+            sm.o[warp][n * 8 + 2 * c + 1][d0] = oacc[n][mt][1];
+            sm.o[warp][n * 8 + 2 * c][d1] = oacc[n][mt][2];
+            sm.o[warp][n * 8 + 2 * c + 1][d1] = oacc[n][mt][3];
+        }
     }
     __syncthreads();
-    for (int i = threadIdx.x; i < 8 * D; i += kThreads) {
+    for (int i = threadIdx.x; i < NT * 8 * D; i += kThreads) {
         const int r = i / D, d = i % D;
         float* orow = rows.o[r];
         if (orow == nullptr) continue;
@@ -497,6 +525,7 @@ __device__ __forceinline__ void attend_stream_staged(const TileRows<1>& rows, co
         orow[d] = den > 0.f ? num / den : 0.f;
         if (d == 0) rows.lse[r][0] = den > 0.f ? M * scale + logf(den) : -INFINITY;
     }
+    __syncthreads();  // the ring may be refilled by a following call
 }
 
 }  // namespace stream
