@@ -261,7 +261,8 @@ def run_cuda(args, w):
     qs = [W.make_queries(wr, sh, s, dev) for s in range(n_q)]
     kv_lens = [(un.kv_len + s).to(torch.int32) for s in range(n_q)]
     max_len = int(lens0.max()) + w.steps
-    layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, max_len, dense=w.dense)
+    layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, max_len, dense=w.dense,
+                       n_unique_splits=args.unique_splits)
     S = layer.shape
     if not w.dense:
         layer.build_summaries(sh.k_shared)
@@ -498,6 +499,7 @@ def main():
     ap.add_argument("--config", type=int, default=1, help="workload index 0..4 (default 1)")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--one-stream", action="store_true", help="run unique attention on the main stream")
+    ap.add_argument("--unique-splits", type=int, default=None, help="override the split-K count of unique attention")
     ap.add_argument("--no-baseline", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample", type=int, default=16, help="requests in the CPU-oracle sample")
