@@ -56,7 +56,7 @@ def _subproblem(q, topk, sh, un, kv_len, sample):
 
 
 def run_case(w: W.Workload, sample=None, lengths=None, n_unique_splits=None, step=0,
-             check_baseline=True, two_streams=False, dense_slots=None):
+             check_baseline=True, two_streams=False, dense_slots=None, unique_tokens=0):
     """All stages of one decode step of workload `w` against the oracle."""
     M, MoskaLayer = _mods()
     dev = "cuda"
@@ -158,7 +158,7 @@ def run_case(w: W.Workload, sample=None, lengths=None, n_unique_splits=None, ste
     # ---- the whole step through moska_decode_step vs the definition (one softmax over the union)
     layer.out.zero_()
     out = layer.step(q, sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, un.kv_start, kv_len,
-                     two_streams=two_streams)
+                     two_streams=two_streams, unique_tokens=unique_tokens)
     torch.cuda.synchronize()
     ref_out, ref_lse = O.attend_direct(q_s, ks, vs, ku, vu, st_s, len_s, topk_s, scale)
     report["out"] = PU.check_attention(out[sample].float().cpu().numpy(), ref_out, "decode step out")
@@ -322,6 +322,18 @@ def test_full_cfg4_sampled_steps():
     for step in (0, w.steps - 1):
         run_case(w, sample=_sample(w, 3), check_baseline=False, step=step, two_streams=True)
         torch.cuda.empty_cache()
+
+
+def test_two_stream_step_with_sm_sharing():
+    """The two-stream schedule of the whole step: unique attention on the main stream, routing,
+    grouping and shared attention on the side stream, the tensor-core kernel on a share of the SMs
+    (forced by a large token-count hint), routed and dense; results must not depend on any of it."""
+    w = W.Workload("share", B=150, Hq=8, Hkv=2, D=128, C=4, L=512, k=2, unique_len=700, seed=51)
+    for hint in (0, 10**9, 3 * 10**6):
+        run_case(w, two_streams=True, unique_tokens=hint, check_baseline=False)
+    wd = W.Workload("share_dense", B=90, Hq=8, Hkv=2, D=128, C=6, L=256, k=6, unique_len=300, seed=52)
+    for hint in (0, 10**9):
+        run_case(wd, two_streams=True, unique_tokens=hint, dense_slots=3, check_baseline=False)
 
 
 def test_several_query_tokens_per_request_by_batch_expansion():
