@@ -358,3 +358,36 @@ def test_several_query_tokens_per_request_by_batch_expansion():
                              layer.topk_idx.cpu().numpy(), layer.scale)
     PU.check_attention(out.float().cpu().numpy(), ref, "several query tokens per request")
     assert M.device_status() == 0
+
+
+def test_decode_step_can_be_captured_in_a_cuda_graph():
+    """Nothing in the step reads device results back on the host, so the whole two-stream step
+    (fork and join included) is one CUDA graph; replaying it gives the eager result bit for bit."""
+    M, MoskaLayer = _mods()
+    w = W.scaled(W.CONFIGS[1], B=32, C=16, k=4, unique_len=600)
+    sh = W.make_shared_store(w, "cuda")
+    un = W.make_unique_store(w, "cuda")
+    q = W.make_queries(w, sh, 0, "cuda")
+    layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, 600)
+    layer.build_summaries(sh.k_shared)
+
+    def step():
+        layer.step(q, sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, un.kv_start, un.kv_len,
+                   two_streams=True, unique_tokens=10**9)
+
+    step()   # also creates the side stream and the library's per-thread events outside the capture
+    torch.cuda.synchronize()
+    eager = layer.out.clone()
+    graph = torch.cuda.CUDAGraph()
+    cap = torch.cuda.Stream()
+    cap.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(cap):
+        with torch.cuda.graph(graph, stream=cap):
+            step()
+    torch.cuda.synchronize()
+    for _ in range(2):
+        layer.out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(layer.out, eager)
+    assert M.device_status() == 0
