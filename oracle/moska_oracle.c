@@ -286,3 +286,66 @@ void oracle_merge(const double* o_part, const double* lse_part, double* out, dou
         lse[r] = M + log(W);
     }
 }
+
+/* ------------------------------------------------------------------------------------------------
+ * FP8 (E4M3) private KV, the storage precision the paper's evaluation assumes (Section IV).
+ *
+ * Value of an OCP FP8 E4M3 code (1 sign bit, 4 exponent bits with bias 7, 3 mantissa bits; no
+ * infinities; S.1111.111 is NaN; exponent field 0 holds the subnormals m/8 * 2^-6), written out
+ * from the format's definition.
+ */
+double oracle_e4m3_value(uint8_t code)
+{
+    const int sign = code >> 7, e = (code >> 3) & 15, m = code & 7;
+    double v;
+    if (e == 15 && m == 7) return NAN;
+    if (e == 0) v = ldexp((double)m / 8.0, -6);
+    else v = ldexp(1.0 + (double)m / 8.0, e - 7);
+    return sign ? -v : v;
+}
+
+/*
+ * Unique KV Attention over an FP8 store (Section III-A with the KV precision of Section IV): token
+ * t of KV head h has key  k_scale[t][h] * e4m3(k8[t][h][:])  and value  v_scale[t][h] *
+ * e4m3(v8[t][h][:]); each query row attends with one softmax to its request's tokens.
+ *   q bf16 [B][Hq][D]; k8, v8 uint8 [T][Hkv][D]; k_scale, v_scale float [T][Hkv];
+ *   kv_start int64 [B], kv_len int32 [B]  ->  out [B][Hq][D], lse [B][Hq]
+ */
+void oracle_attend_unique_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v8,
+                              const float* k_scale, const float* v_scale, const int64_t* kv_start,
+                              const int32_t* kv_len, double* out, double* lse, double scale, int B,
+                              int Hq, int Hkv, int D)
+{
+    const int G = Hq / Hkv;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long r = 0; r < (long)B * Hq; ++r) {
+        const int b = (int)(r / Hq), hq = (int)(r % Hq), h = hq / G;
+        const long n = kv_len[b];
+        double* o = out + r * D;
+        for (int d = 0; d < D; ++d) o[d] = 0.0;
+        if (n == 0) {
+            lse[r] = -INFINITY;
+            continue;
+        }
+        double* s = (double*)malloc(sizeof(double) * n);
+        double m = -INFINITY;
+        for (long t = 0; t < n; ++t) {
+            const long row = ((long)kv_start[b] + t) * Hkv + h;
+            double acc = 0.0;
+            for (int d = 0; d < D; ++d)
+                acc += bf16_to_double(q[r * D + d]) * ((double)k_scale[row] * oracle_e4m3_value(k8[row * D + d]));
+            s[t] = scale * acc;
+            if (s[t] > m) m = s[t];
+        }
+        double z = 0.0;
+        for (long t = 0; t < n; ++t) z += exp(s[t] - m);
+        lse[r] = m + log(z);
+        for (long t = 0; t < n; ++t) {
+            const long row = ((long)kv_start[b] + t) * Hkv + h;
+            const double p = exp(s[t] - lse[r]);
+            for (int d = 0; d < D; ++d)
+                o[d] += p * ((double)v_scale[row] * oracle_e4m3_value(v8[row * D + d]));
+        }
+        free(s);
+    }
+}

@@ -146,3 +146,35 @@ def merge(o_part, lse_part):
     lse = np.empty((rows,), dtype=np.float64)
     _load().oracle_merge(_p(o), _p(l), _p(out), _p(lse), ctypes.c_long(rows), n_slots, D)
     return out.reshape(*lead, D), lse.reshape(lead)
+
+
+def e4m3_values() -> np.ndarray:
+    """The 256 values of the FP8 E4M3 format as the oracle decodes them (NaN for the two NaN codes)."""
+    lib = _load()
+    lib.oracle_e4m3_value.restype = ctypes.c_double
+    lib.oracle_e4m3_value.argtypes = [ctypes.c_uint8]
+    return np.array([lib.oracle_e4m3_value(c) for c in range(256)], dtype=np.float64)
+
+
+def attend_unique_fp8(q, k8, v8, k_scale, v_scale, kv_start, kv_len, scale: float):
+    """Attention of every query row over its request's FP8 private KV -> (out, lse) in f64."""
+    B, Hq, D = q.shape
+    Hkv = k8.shape[1]
+
+    def _u8(t):
+        if isinstance(t, torch.Tensor):
+            t = t.detach().cpu().numpy()
+        return np.ascontiguousarray(t, dtype=np.uint8)
+
+    def _f32(t):
+        if isinstance(t, torch.Tensor):
+            t = t.detach().cpu().numpy()
+        return np.ascontiguousarray(t, dtype=np.float32)
+
+    out = np.empty((B, Hq, D), dtype=np.float64)
+    lse = np.empty((B, Hq), dtype=np.float64)
+    qb, kk, vv, ks, vs = _bits(q), _u8(k8), _u8(v8), _f32(k_scale), _f32(v_scale)
+    st, ln = _i64(kv_start), _i32(kv_len)
+    _load().oracle_attend_unique_fp8(_p(qb), _p(kk), _p(vv), _p(ks), _p(vs), _p(st), _p(ln), _p(out),
+                                     _p(lse), ctypes.c_double(scale), B, Hq, Hkv, D)
+    return out, lse

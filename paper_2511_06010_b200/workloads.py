@@ -158,3 +158,27 @@ def make_queries(w: Workload, shared: SharedStore, step: int = 0, device="cpu") 
     head_of = torch.arange(w.Hq, device=device) // w.G
     centre = shared.mu[head_of[None, :], tgt[:, None], :]          # [B][Hq][D]
     return (centre + 0.5 * noise).to(torch.bfloat16).contiguous()
+
+
+@dataclasses.dataclass
+class UniqueStoreFp8:
+    k8: torch.Tensor        # uint8 [T_total][Hkv][D]  FP8 E4M3 codes of the keys
+    v8: torch.Tensor        # uint8 [T_total][Hkv][D]  FP8 E4M3 codes of the values
+    k_scale: torch.Tensor   # fp32  [T_total][Hkv]     key = k_scale * e4m3(k8)
+    v_scale: torch.Tensor   # fp32  [T_total][Hkv]
+
+
+def quantize_unique_store_fp8(un: UniqueStore) -> UniqueStoreFp8:
+    """Storage-format conversion of a private KV store to FP8 E4M3 with one scale per (token, KV
+    head): scale = max|x| / 448 (the largest E4M3 value), codes by torch's round-to-nearest cast.
+    Input preparation only: the FP8 store is what both the CUDA path and the oracle are given."""
+    def q8(x):
+        x = x.float()
+        amax = x.abs().amax(dim=-1)
+        scale = torch.where(amax > 0, amax / 448.0, torch.ones_like(amax))
+        codes = (x / scale[..., None]).to(torch.float8_e4m3fn).view(torch.uint8)
+        return codes.contiguous(), scale.contiguous()
+
+    k8, ks = q8(un.k_unique)
+    v8, vs = q8(un.v_unique)
+    return UniqueStoreFp8(k8, v8, ks, vs)
