@@ -257,6 +257,14 @@ def run_cuda(args, w):
         raise SystemExit(f"workload {w.name} needs {need/1e9:.1f} GB, only {free/1e9:.1f} GB free")
     sh = W.make_shared_store(wr, dev)
     un = W.make_unique_store(wr, dev)
+    fp8 = args.unique_kv == "fp8"
+    f8 = None
+    if fp8:
+        # the private store in FP8 E4M3 with per-token scales; the bf16 copy is not kept
+        if w.D != 128:
+            raise SystemExit("--unique-kv fp8 needs head dimension 128")
+        f8 = W.quantize_unique_store_fp8(un, release=True)
+        torch.cuda.empty_cache()
     n_q = max(1, w.steps)
     qs = [W.make_queries(wr, sh, s, dev) for s in range(n_q)]
     kv_lens = [(un.kv_len + s).to(torch.int32) for s in range(n_q)]
@@ -269,7 +277,7 @@ def run_cuda(args, w):
     torch.cuda.synchronize()
 
     two_streams = (not args.one_stream) and layer.overlap_routing
-    input_bytes = (sh.k_shared.numel() + un.k_unique.numel()) * 4
+    input_bytes = sh.k_shared.numel() * 4 + (f8.k8.numel() * 2 if fp8 else un.k_unique.numel() * 4)
     flush_buf = None
     if input_bytes < 2 * L2_BYTES:
         flush_buf = torch.empty(int(3 * L2_BYTES), dtype=torch.uint8, device=dev)
@@ -280,8 +288,32 @@ def run_cuda(args, w):
 
     def step(i, prof=None):
         s = i % n_q
-        layer.step(qs[s], sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, un.kv_start,
-                   kv_lens[s], two_streams=two_streams, prof=prof, unique_tokens=tokens[s])
+        if fp8:
+            layer.step_fp8kv(qs[s], sh.k_shared, sh.v_shared, f8, un.kv_start, kv_lens[s],
+                             two_streams=two_streams, prof=prof, unique_tokens=tokens[s])
+        else:
+            layer.step(qs[s], sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, un.kv_start,
+                       kv_lens[s], two_streams=two_streams, prof=prof, unique_tokens=tokens[s])
+
+    def step_host(i):
+        s = i % n_q
+        if fp8:
+            # no host-buffer entry point for the FP8 store: the same copies around the device call
+            q_dev.copy_(q_host[s], non_blocking=True)
+            out = layer.step_fp8kv(q_dev, sh.k_shared, sh.v_shared, f8, un.kv_start, kv_lens[s],
+                                   two_streams=two_streams, unique_tokens=tokens[s])
+            out_host.copy_(out, non_blocking=True)
+            torch.cuda.current_stream().synchronize()
+        else:
+            layer.step_host(q_host[s], q_dev, out_host, sh.k_shared, sh.v_shared, un.k_unique,
+                            un.v_unique, un.kv_start, kv_lens[s], two_streams=two_streams,
+                            unique_tokens=tokens[s])
+
+    def unique_alone():
+        if fp8:
+            layer.unique_fp8(qs[0], f8, un.kv_start, kv_lens[0])
+        else:
+            layer.unique(qs[0], un.k_unique, un.v_unique, un.kv_start, kv_lens[0])
 
     for i in range(max(3, args.warmup)):
         step(i)
@@ -325,9 +357,7 @@ def run_cuda(args, w):
     out_host = torch.empty(w.B, w.Hq, w.D, dtype=torch.bfloat16).pin_memory()
     q_dev = torch.empty_like(qs[0])
     for i in range(3):
-        layer.step_host(q_host[i % n_q], q_dev, out_host, sh.k_shared, sh.v_shared, un.k_unique,
-                        un.v_unique, un.kv_start, kv_lens[i % n_q], two_streams=two_streams,
-                        unique_tokens=tokens[i % n_q])
+        step_host(i)
     DD.barrier()
     torch.cuda.synchronize()
     t0 = time.perf_counter()
@@ -336,9 +366,7 @@ def run_cuda(args, w):
     for i in range(args.steps):
         if flush is not None:
             flush()
-        layer.step_host(q_host[i % n_q], q_dev, out_host, sh.k_shared, sh.v_shared, un.k_unique,
-                        un.v_unique, un.kv_start, kv_lens[i % n_q], two_streams=two_streams,
-                        unique_tokens=tokens[i % n_q])
+        step_host(i)
     e1.record()
     torch.cuda.synchronize()
     e2e_ms = e0.elapsed_time(e1)
@@ -358,6 +386,8 @@ def run_cuda(args, w):
         off = layer.seg_offsets.cpu().numpy()
         touched, P = int((np.diff(off) > 0).sum()), w.B * w.Hkv * w.k
     work = algorithmic_work(w, lens, S.n_unique_splits, S.shared_slots, touched)
+    if fp8:  # one byte per element and two fp32 scales per (token, KV head) instead of bf16 K and V
+        work["unique_bytes"] -= int(lens.sum()) * w.Hkv * (2 * w.D - 8)
     iters = max(3, min(args.steps, 10))
     gemv_ms = None
     if not args.no_baseline:
@@ -376,7 +406,7 @@ def run_cuda(args, w):
             if not w.dense:
                 layer.route(qs[0])
                 layer.group()
-            layer.unique(qs[0], un.k_unique, un.v_unique, un.kv_start, kv_lens[0])
+            unique_alone()
             layer.merge()
         # shared attention is the only stage that differs: time the other stages once, add the baseline
         gemv_step_ms = time_events(baseline_step, iters, flush) + gemv_ms
@@ -387,8 +417,7 @@ def run_cuda(args, w):
         iso["route"] = time_events(lambda: layer.route(qs[0]), iters, flush)
         iso["group"] = time_events(lambda: layer.group(), iters, flush)
     iso["shared"] = time_events(lambda: layer.shared(qs[0], sh.k_shared, sh.v_shared), iters, flush)
-    iso["unique"] = time_events(lambda: layer.unique(qs[0], un.k_unique, un.v_unique, un.kv_start,
-                                                     kv_lens[0]), iters, flush)
+    iso["unique"] = time_events(unique_alone, iters, flush)
     iso["merge"] = time_events(lambda: layer.merge(), iters, flush)
     shared_ms, unique_ms = stage_ms["shared"], stage_ms["unique"]
     shared_tflops = work["shared_flops"] / (shared_ms * 1e-3) / 1e12 if shared_ms > 0 else None
@@ -399,7 +428,7 @@ def run_cuda(args, w):
     t_flops = work["shared_flops"] / (peaks["bf16_tflops_sustained"] * 1e12)
     t_bytes = work["shared_bytes"] / (peaks["hbm_gbs"] * 1e9)
     if unique_ms >= shared_ms:
-        kernel = "unique_staged_kernel" if w.D == 128 else "unique_attn_kernel"
+        kernel = "unique_fp8_kernel" if fp8 else ("unique_staged_kernel" if w.D == 128 else "unique_attn_kernel")
         roof = dict(bound="hbm", achieved=unique_gbs, peak=peaks["hbm_gbs"], unit="GB/s")
     elif t_flops > t_bytes:
         kernel = "shared_tc_kernel"
@@ -416,7 +445,7 @@ def run_cuda(args, w):
 
     # ---- CPU baseline: the oracle as it stands on the host cores, bounded sample (N = 1 only)
     cpu = None
-    if world == 1 and not args.no_cpu_baseline:
+    if world == 1 and not args.no_cpu_baseline and not fp8:
         from oracle import oracle as O
 
         O.build()
@@ -453,6 +482,7 @@ def run_cuda(args, w):
             "shared_tokens": w.C * w.L, "chunk_tokens": w.L, "top_k": None if w.dense else w.k,
             "unique_tokens_mean": float(lens.mean()), "n_unique_splits": S.n_unique_splits,
             "shared_slots": S.shared_slots, "streams": 2 if two_streams else 1,
+            "unique_kv": "fp8_e4m3 + fp32 scale per (token, kv head)" if fp8 else "bf16",
             "l2": ("flushed between steps" if flush is not None
                    else f"inputs exceed L2 ({input_bytes / 2**20:.0f} MiB of K/V per step)"),
             "per_gpu": "own request batch, own copy of the shared store" if world > 1 else "single GPU",
@@ -500,6 +530,8 @@ def main():
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--one-stream", action="store_true", help="run unique attention on the main stream")
     ap.add_argument("--unique-splits", type=int, default=None, help="override the split-K count of unique attention")
+    ap.add_argument("--unique-kv", default="bf16", choices=["bf16", "fp8"],
+                    help="storage of the private KV (fp8: E4M3 codes with per-token scales; no CPU baseline)")
     ap.add_argument("--no-baseline", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample", type=int, default=16, help="requests in the CPU-oracle sample")

@@ -201,6 +201,21 @@ int moska_unique_attn(const uint16_t* q, const uint16_t* k_unique, const uint16_
                       moska_stream stream);
 
 /*
+ * Unique KV Attention over a private KV store kept in FP8 (E4M3), the KV precision the paper's
+ * evaluation assumes (Section IV) applied to the memory-bound per-request pass of Section III-A.
+ * Token t of KV head h has key k_scale[t][h] * e4m3(k8[t][h][:]) and value v_scale[t][h] *
+ * e4m3(v8[t][h][:]); everything else (split-K slots, empty requests, outputs) is as in
+ * moska_unique_attn.  The codes are widened exactly to f16 and multiplied on tensor cores with
+ * fp32 accumulation; P is rounded to f16.  D must be 128.
+ *   k8, v8            uint8 [T_total][Hkv][D]   OCP FP8 E4M3 codes (16-byte aligned)
+ *   k_scale, v_scale  float [T_total][Hkv]
+ */
+int moska_unique_attn_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v8,
+                          const float* k_scale, const float* v_scale, const int64_t* kv_start,
+                          const int32_t* kv_len, float* o_part, float* lse_part,
+                          float softmax_scale, const moska_shape* shape, moska_stream stream);
+
+/*
  * Combination of the shared and unique partial results.  The paper leaves this step implicit;
  * the log-sum-exp merge is the only combination that equals softmax attention over the union of
  * the tokens (Section III-A/III-B).  Per row: M = max_i lse_i, w_i = exp(lse_i - M),
@@ -252,6 +267,20 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
                       float* o_part, float* lse_part, uint16_t* out, float* lse_out,
                       float softmax_scale, const moska_shape* shape, void* ws, size_t ws_bytes,
                       moska_stream stream, moska_stream side_stream, moska_profiler* prof);
+
+/*
+ * moska_decode_step with the private KV store in FP8 (E4M3 codes + per-(token, head) fp32 scales,
+ * laid out as for moska_unique_attn_fp8); the shared store stays bf16.  Same schedule, buffers,
+ * outputs and error behaviour; D must be 128.
+ */
+int moska_decode_step_fp8kv(const uint16_t* q, const float* summaries, const uint16_t* k_shared,
+                            const uint16_t* v_shared, const uint8_t* k8_unique,
+                            const uint8_t* v8_unique, const float* k_scale, const float* v_scale,
+                            const int64_t* kv_start, const int32_t* kv_len, int32_t* topk_idx,
+                            int32_t* seg_offsets, int32_t* seg_entries, float* o_part,
+                            float* lse_part, uint16_t* out, float* lse_out, float softmax_scale,
+                            const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream,
+                            moska_stream side_stream, moska_profiler* prof);
 
 /*
  * moska_decode_step for a caller whose step inputs live in HOST memory: copies q_host (bf16

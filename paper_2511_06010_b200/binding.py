@@ -53,9 +53,11 @@ EXPORTS = {
     "moska_group_by_chunk_noalloc": (_i, [_vp, _vp, _vp, _sp, _vp]),
     "moska_shared_attn": (_i, [_vp] * 8 + [_f, _sp, _vp, _sz, _vp]),
     "moska_unique_attn": (_i, [_vp] * 7 + [_f, _sp, _vp]),
+    "moska_unique_attn_fp8": (_i, [_vp] * 9 + [_f, _sp, _vp]),
     "moska_merge": (_i, [_vp] * 5 + [_sp, _vp]),
     "moska_gemv_baseline": (_i, [_vp] * 6 + [_f, _sp, _vp]),
     "moska_decode_step": (_i, [_vp] * 15 + [_f, _sp, _vp, _sz, _vp, _vp, _vp]),
+    "moska_decode_step_fp8kv": (_i, [_vp] * 17 + [_f, _sp, _vp, _sz, _vp, _vp, _vp]),
     "moska_decode_step_host": (_i, [_vp] * 16 + [_f, _sp, _vp, _sz, _vp, _vp, _vp]),
     "moska_profiler_create": (_i, [ctypes.POINTER(_vp), ctypes.c_int32]),
     "moska_profiler_destroy": (None, [_vp]),
@@ -167,6 +169,14 @@ def unique_attn(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part, softm
                                   ctypes.byref(s), _stream(stream)), "moska_unique_attn")
 
 
+def unique_attn_fp8(q, k8, v8, k_scale, v_scale, kv_start, kv_len, o_part, lse_part, softmax_scale,
+                    s, stream=None) -> None:
+    _check(_lib.moska_unique_attn_fp8(_ptr(q), _ptr(k8), _ptr(v8), _ptr(k_scale), _ptr(v_scale),
+                                      _ptr(kv_start), _ptr(kv_len), _ptr(o_part), _ptr(lse_part),
+                                      softmax_scale, ctypes.byref(s), _stream(stream)),
+           "moska_unique_attn_fp8")
+
+
 def merge(o_part, lse_part, out, out_f32, lse_out, s, stream=None) -> None:
     _check(_lib.moska_merge(_ptr(o_part), _ptr(lse_part), _ptr(out), _ptr(out_f32),
                             _ptr(lse_out), ctypes.byref(s), _stream(stream)), "moska_merge")
@@ -189,6 +199,18 @@ def decode_step(q, summaries, k_shared, v_shared, k_unique, v_unique, kv_start, 
         _ptr(o_part), _ptr(lse_part), _ptr(out), _ptr(lse_out), softmax_scale, ctypes.byref(s),
         _ptr(ws), ws_bytes, _stream(stream),
         None if side_stream is None else _stream(side_stream), prof), "moska_decode_step")
+
+
+def decode_step_fp8kv(q, summaries, k_shared, v_shared, k8_unique, v8_unique, k_scale, v_scale,
+                      kv_start, kv_len, topk_idx, seg_offsets, seg_entries, o_part, lse_part, out,
+                      lse_out, softmax_scale, s, ws, stream=None, side_stream=None, prof=None) -> None:
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(_lib.moska_decode_step_fp8kv(
+        _ptr(q), _ptr(summaries), _ptr(k_shared), _ptr(v_shared), _ptr(k8_unique), _ptr(v8_unique),
+        _ptr(k_scale), _ptr(v_scale), _ptr(kv_start), _ptr(kv_len), _ptr(topk_idx),
+        _ptr(seg_offsets), _ptr(seg_entries), _ptr(o_part), _ptr(lse_part), _ptr(out),
+        _ptr(lse_out), softmax_scale, ctypes.byref(s), _ptr(ws), ws_bytes, _stream(stream),
+        None if side_stream is None else _stream(side_stream), prof), "moska_decode_step_fp8kv")
 
 
 def decode_step_host(q_host, q_dev, summaries, k_shared, v_shared, k_unique, v_unique, kv_start,

@@ -290,6 +290,27 @@ int moska_unique_attn(const uint16_t* q, const uint16_t* k_unique, const uint16_
                          shape, (cudaStream_t)stream);
 }
 
+int moska_unique_attn_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v8,
+                          const float* k_scale, const float* v_scale, const int64_t* kv_start,
+                          const int32_t* kv_len, float* o_part, float* lse_part,
+                          float softmax_scale, const moska_shape* shape, moska_stream stream)
+{
+    MOSKA_TRY(check_shape(shape, false));
+    if (shape->D != 128) return fail(MOSKA_ERR_UNSUPPORTED, "FP8 unique attention is built for D = 128");
+    MOSKA_TRY(check_device());
+    REQUIRE_PTR(q, 16);
+    REQUIRE_PTR(k8, 16);
+    REQUIRE_PTR(v8, 16);
+    REQUIRE_PTR(k_scale, 4);
+    REQUIRE_PTR(v_scale, 4);
+    REQUIRE_PTR(kv_start, 8);
+    REQUIRE_PTR(kv_len, 4);
+    REQUIRE_PTR(o_part, 16);
+    REQUIRE_PTR(lse_part, 4);
+    return launch_unique_fp8(q, k8, v8, k_scale, v_scale, kv_start, kv_len, o_part, lse_part,
+                             softmax_scale, shape, (cudaStream_t)stream);
+}
+
 int moska_merge(const float* o_part, const float* lse_part, uint16_t* out, float* out_f32,
                 float* lse_out, const moska_shape* shape, moska_stream stream)
 {
@@ -323,13 +344,36 @@ int moska_gemv_baseline(const uint16_t* q, const uint16_t* k_shared, const uint1
                                 shape, (cudaStream_t)stream);
 }
 
-int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t* k_shared,
-                      const uint16_t* v_shared, const uint16_t* k_unique,
-                      const uint16_t* v_unique, const int64_t* kv_start, const int32_t* kv_len,
-                      int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
-                      float* o_part, float* lse_part, uint16_t* out, float* lse_out,
-                      float softmax_scale, const moska_shape* shape, void* ws, size_t ws_bytes,
-                      moska_stream stream, moska_stream side_stream, moska_profiler* prof)
+namespace {
+// The private KV store of a decode step: bf16 (k, v) or FP8 E4M3 codes with per-token scales.
+struct UniqueKv {
+    const uint16_t* k = nullptr;
+    const uint16_t* v = nullptr;
+    const uint8_t* k8 = nullptr;
+    const uint8_t* v8 = nullptr;
+    const float* k_scale = nullptr;
+    const float* v_scale = nullptr;
+    bool fp8 = false;
+};
+
+int unique_impl(const uint16_t* q, const UniqueKv& kv, const int64_t* kv_start, const int32_t* kv_len,
+                float* o_part, float* lse_part, float softmax_scale, const moska_shape* shape,
+                cudaStream_t st)
+{
+    if (kv.fp8)
+        return moska_unique_attn_fp8(q, kv.k8, kv.v8, kv.k_scale, kv.v_scale, kv_start, kv_len, o_part,
+                                     lse_part, softmax_scale, shape, st);
+    return moska_unique_attn(q, kv.k, kv.v, kv_start, kv_len, o_part, lse_part, softmax_scale, shape,
+                             st);
+}
+
+int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* k_shared,
+                     const uint16_t* v_shared, const UniqueKv& kv, const int64_t* kv_start,
+                     const int32_t* kv_len, int32_t* topk_idx, int32_t* seg_offsets,
+                     int32_t* seg_entries, float* o_part, float* lse_part, uint16_t* out,
+                     float* lse_out, float softmax_scale, const moska_shape* shape, void* ws,
+                     size_t ws_bytes, moska_stream stream, moska_stream side_stream,
+                     moska_profiler* prof)
 {
     const bool dense = summaries == nullptr;
     cudaStream_t st = (cudaStream_t)stream, side = (cudaStream_t)side_stream;
@@ -345,8 +389,7 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
             MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 1, st));
         }
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 0, st));
-        MOSKA_TRY(moska_unique_attn(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part,
-                                    softmax_scale, shape, st));
+        MOSKA_TRY(unique_impl(q, kv, kv_start, kv_len, o_part, lse_part, softmax_scale, shape, st));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 1, st));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 0, st));
         MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, dense ? nullptr : topk_idx,
@@ -378,8 +421,7 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
         MOSKA_CUDA_TRY(cudaEventRecord(ev_fork, st));
         MOSKA_CUDA_TRY(cudaStreamWaitEvent(side, ev_fork, 0));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 0, st));
-        MOSKA_TRY(moska_unique_attn(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part,
-                                    softmax_scale, shape, st));
+        MOSKA_TRY(unique_impl(q, kv, kv_start, kv_len, o_part, lse_part, softmax_scale, shape, st));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 1, st));
         if (!dense) {
             MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 0, side));
@@ -396,7 +438,8 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
         // to start beside it (the routing chain in front of it takes a few hundred microseconds
         // under contention); for a short unique attention the tensor-core items run after it, on
         // all SMs.
-        const double unique_ms = (double)shape->unique_tokens * shape->Hkv * 4.0 * shape->D / 7.0e9;
+        const double unique_ms = (double)shape->unique_tokens * shape->Hkv *
+                                 (kv.fp8 ? 2.0 * shape->D + 8.0 : 4.0 * shape->D) / 7.0e9;
         const bool beside = tc && (dense || unique_ms >= 0.6);
         if (tc && beside)
             MOSKA_TRY(launch_shared_tc(q, k_shared, v_shared, dense ? nullptr : seg_entries, o_part,
@@ -419,6 +462,43 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
     MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_MERGE, 1, st));
     if (prof != nullptr && prof->n_steps < prof->max_steps) ++prof->n_steps;
     return MOSKA_OK;
+}
+}  // namespace
+
+int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t* k_shared,
+                      const uint16_t* v_shared, const uint16_t* k_unique,
+                      const uint16_t* v_unique, const int64_t* kv_start, const int32_t* kv_len,
+                      int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
+                      float* o_part, float* lse_part, uint16_t* out, float* lse_out,
+                      float softmax_scale, const moska_shape* shape, void* ws, size_t ws_bytes,
+                      moska_stream stream, moska_stream side_stream, moska_profiler* prof)
+{
+    UniqueKv kv;
+    kv.k = k_unique;
+    kv.v = v_unique;
+    return decode_step_impl(q, summaries, k_shared, v_shared, kv, kv_start, kv_len, topk_idx,
+                            seg_offsets, seg_entries, o_part, lse_part, out, lse_out, softmax_scale,
+                            shape, ws, ws_bytes, stream, side_stream, prof);
+}
+
+int moska_decode_step_fp8kv(const uint16_t* q, const float* summaries, const uint16_t* k_shared,
+                            const uint16_t* v_shared, const uint8_t* k8_unique,
+                            const uint8_t* v8_unique, const float* k_scale, const float* v_scale,
+                            const int64_t* kv_start, const int32_t* kv_len, int32_t* topk_idx,
+                            int32_t* seg_offsets, int32_t* seg_entries, float* o_part,
+                            float* lse_part, uint16_t* out, float* lse_out, float softmax_scale,
+                            const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream,
+                            moska_stream side_stream, moska_profiler* prof)
+{
+    UniqueKv kv;
+    kv.k8 = k8_unique;
+    kv.v8 = v8_unique;
+    kv.k_scale = k_scale;
+    kv.v_scale = v_scale;
+    kv.fp8 = true;
+    return decode_step_impl(q, summaries, k_shared, v_shared, kv, kv_start, kv_len, topk_idx,
+                            seg_offsets, seg_entries, o_part, lse_part, out, lse_out, softmax_scale,
+                            shape, ws, ws_bytes, stream, side_stream, prof);
 }
 
 int moska_profiler_create(moska_profiler** out, int32_t max_steps)

@@ -71,6 +71,10 @@ class MoskaLayer:
         M.unique_attn(q, k_unique, v_unique, kv_start, kv_len, self.o_part, self.lse_part,
                       self.scale, self.shape, stream)
 
+    def unique_fp8(self, q, f8, kv_start, kv_len, stream=None):
+        M.unique_attn_fp8(q, f8.k8, f8.v8, f8.k_scale, f8.v_scale, kv_start, kv_len, self.o_part,
+                          self.lse_part, self.scale, self.shape, stream)
+
     def merge(self):
         M.merge(self.o_part, self.lse_part, self.out, self.out_f32, self.lse_out, self.shape)
 
@@ -86,6 +90,20 @@ class MoskaLayer:
                       self.seg_entries, self.o_part, self.lse_part, self.out, self.lse_out,
                       self.scale, self.shape, self.ws, None,
                       self.side_stream if two_streams else None, prof)
+        return self.out
+
+    def step_fp8kv(self, q, k_shared, v_shared, f8, kv_start, kv_len, two_streams=False, prof=None,
+                   unique_tokens=0):
+        """One decode step with the private KV store in FP8 (`f8`: codes and per-token scales)."""
+        self.shape.unique_tokens = int(unique_tokens)
+        two_streams = two_streams and self.overlap_routing
+        if two_streams and self.side_stream is None:
+            self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
+        M.decode_step_fp8kv(q, None if self.dense else self.summaries, k_shared, v_shared, f8.k8,
+                            f8.v8, f8.k_scale, f8.v_scale, kv_start, kv_len, self.topk_idx,
+                            self.seg_offsets, self.seg_entries, self.o_part, self.lse_part,
+                            self.out, self.lse_out, self.scale, self.shape, self.ws, None,
+                            self.side_stream if two_streams else None, prof)
         return self.out
 
     def step_host(self, q_host, q_dev, out_host, k_shared, v_shared, k_unique, v_unique,

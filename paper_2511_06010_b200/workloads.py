@@ -168,17 +168,28 @@ class UniqueStoreFp8:
     v_scale: torch.Tensor   # fp32  [T_total][Hkv]
 
 
-def quantize_unique_store_fp8(un: UniqueStore) -> UniqueStoreFp8:
+def quantize_unique_store_fp8(un: UniqueStore, release: bool = False) -> UniqueStoreFp8:
     """Storage-format conversion of a private KV store to FP8 E4M3 with one scale per (token, KV
     head): scale = max|x| / 448 (the largest E4M3 value), codes by torch's round-to-nearest cast.
-    Input preparation only: the FP8 store is what both the CUDA path and the oracle are given."""
+    Input preparation only: the FP8 store is what both the CUDA path and the oracle are given.
+    `release` drops each bf16 tensor of `un` as soon as it is converted (for stores that fill most
+    of the device memory)."""
     def q8(x):
-        x = x.float()
-        amax = x.abs().amax(dim=-1)
-        scale = torch.where(amax > 0, amax / 448.0, torch.ones_like(amax))
-        codes = (x / scale[..., None]).to(torch.float8_e4m3fn).view(torch.uint8)
-        return codes.contiguous(), scale.contiguous()
+        codes = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+        scales = torch.empty(x.shape[:-1], dtype=torch.float32, device=x.device)
+        step = max(1, (1 << 26) // (x.shape[1] * x.shape[2]))  # bounded temporaries
+        for t0 in range(0, x.shape[0], step):
+            xs = x[t0:t0 + step].float()
+            amax = xs.abs().amax(dim=-1)
+            scale = torch.where(amax > 0, amax / 448.0, torch.ones_like(amax))
+            codes[t0:t0 + step] = (xs / scale[..., None]).to(torch.float8_e4m3fn).view(torch.uint8)
+            scales[t0:t0 + step] = scale
+        return codes, scales
 
     k8, ks = q8(un.k_unique)
+    if release:
+        un.k_unique = None
     v8, vs = q8(un.v_unique)
+    if release:
+        un.v_unique = None
     return UniqueStoreFp8(k8, v8, ks, vs)
