@@ -141,7 +141,7 @@ namespace {
 // 7 TB/s) and the SMs are divided so that neither waits for the other.  Unique attention reaches
 // most of the HBM bandwidth from about 96 SMs; if it is the longer job the tensor-core kernel
 // hides entirely on the remaining ones.
-int tc_sm_share(const moska_shape* s, bool dense)
+int tc_sm_share(const moska_shape* s, bool dense, double unique_ms)
 {
     int dev = 0, n_sms = 148;
     if (cudaGetDevice(&dev) == cudaSuccess)
@@ -151,7 +151,7 @@ int tc_sm_share(const moska_shape* s, bool dense)
     if (s->unique_tokens <= 0) {
         x = dense ? (n_sms * 4) / 5 : (n_sms * 35) / 100;  // no hint: tensor-heavy / HBM-heavy guess
     } else {
-        const double b = (double)s->unique_tokens * s->Hkv * 4.0 * s->D / 7.0e9;  // ms
+        const double b = unique_ms;
         const int hbm_sms = (n_sms * 65) / 100;
         if (a <= b * (n_sms - hbm_sms)) x = n_sms - hbm_sms;
         else x = (int)(a * n_sms / (a + b * 0.4 * n_sms));
@@ -440,11 +440,11 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
         // all SMs.
         const double unique_ms = (double)shape->unique_tokens * shape->Hkv *
                                  (kv.fp8 ? 2.0 * shape->D + 8.0 : 4.0 * shape->D) / 7.0e9;
-        const bool beside = tc && (dense || unique_ms >= 0.6);
+        const bool beside = tc && (dense || unique_ms >= 0.8);
         if (tc && beside)
             MOSKA_TRY(launch_shared_tc(q, k_shared, v_shared, dense ? nullptr : seg_entries, o_part,
                                        lse_part, softmax_scale, shape, ws, dense,
-                                       tc_sm_share(shape, dense), side));
+                                       tc_sm_share(shape, dense, unique_ms), side));
         if (!dense || !tc)
             MOSKA_TRY(launch_shared_small(q, k_shared, v_shared, dense ? nullptr : seg_entries, o_part,
                                           lse_part, softmax_scale, shape, ws, dense, side));
