@@ -272,7 +272,7 @@ def run_cuda(args, w):
     kv_lens = [(un.kv_len + s).to(torch.int32) for s in range(n_q)]
     max_len = int(lens0.max()) + w.steps
     layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, max_len, dense=w.dense,
-                       n_unique_splits=args.unique_splits)
+                       n_unique_splits=args.unique_splits, fp8_unique=fp8)
     S = layer.shape
     if not w.dense:
         layer.build_summaries(sh.k_shared)

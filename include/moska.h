@@ -100,6 +100,10 @@ size_t moska_workspace_bytes(const moska_shape* shape);
  * Host only, pure.                                                                              */
 int moska_default_unique_splits(int32_t B, int32_t Hkv, int32_t max_len);
 
+/* The same for a private store in FP8 (moska_unique_attn_fp8, moska_decode_step_fp8kv), whose
+ * kernel has more and shorter-lived CTAs per SM.  Host only, pure.                             */
+int moska_default_unique_splits_fp8(int32_t B, int32_t Hkv, int32_t max_len);
+
 /*
  * Chunk embeddings used by the router (Section III-B: "precomputed chunk embeddings"; the
  * embedding of a chunk is the arithmetic mean of its L keys, per KV head).  Offline step.

@@ -47,6 +47,7 @@ EXPORTS = {
     "moska_partial_slots": (_i, [_sp]),
     "moska_workspace_bytes": (_sz, [_sp]),
     "moska_default_unique_splits": (_i, [ctypes.c_int32] * 3),
+    "moska_default_unique_splits_fp8": (_i, [ctypes.c_int32] * 3),
     "moska_build_chunk_summaries": (_i, [_vp, _vp, _sp, _vp]),
     "moska_route": (_i, [_vp, _vp, _vp, _vp, _sp, _vp, _sz, _vp]),
     "moska_group_by_chunk": (_i, [_vp, _vp, _vp, _sp, _vp, _sz, _vp]),
@@ -125,6 +126,10 @@ def workspace_bytes(s: MoskaShape) -> int:
 
 def default_unique_splits(B: int, Hkv: int, max_len: int) -> int:
     return _lib.moska_default_unique_splits(B, Hkv, max_len)
+
+
+def default_unique_splits_fp8(B: int, Hkv: int, max_len: int) -> int:
+    return _lib.moska_default_unique_splits_fp8(B, Hkv, max_len)
 
 
 def build_chunk_summaries(k_shared, summaries, s, stream=None) -> None:

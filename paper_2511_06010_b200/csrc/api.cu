@@ -1,6 +1,8 @@
 // extern "C" boundary of the MoSKA library: argument validation and launch sequencing only.
 #include <cstring>
 
+#include <cmath>
+
 #include "common.cuh"
 
 namespace moska {
@@ -123,6 +125,22 @@ int moska_default_unique_splits(int32_t B, int32_t Hkv, int32_t max_len)
     if (n < 1) n = 1;
     if (n > 64) n = 64;
     return (int)n;
+}
+
+int moska_default_unique_splits_fp8(int32_t B, int32_t Hkv, int32_t max_len)
+{
+    // The FP8 kernel's CTAs stream half the bytes per token, three of them per SM.  Its time is
+    // about  n len / S  +  n s ov / S  +  a len / s  (n = B Hkv CTAs per split, S = CTA slots, ov =
+    // fixed cost of a CTA in tokens, a len / s = the tail while the last CTAs run alone), smallest
+    // at s = sqrt(a len S / (n ov)); a = 0.7 and ov = 128 tokens fit the measured sweeps.
+    if (B <= 0 || Hkv <= 0 || max_len <= 0) return 1;
+    const double slots = 148.0 * 3.0, n = (double)B * Hkv;
+    long long s = llround(sqrt(0.7 * max_len * slots / (n * 128.0)));
+    const long long cap = (max_len + 511) / 512;
+    if (s > cap) s = cap;
+    if (s < 1) s = 1;
+    if (s > 64) s = 64;
+    return (int)s;
 }
 
 int moska_build_chunk_summaries(const uint16_t* k_shared, float* summaries,

@@ -14,11 +14,12 @@ class MoskaLayer:
     """Owns the scratch of a decode step for a fixed shape and calls the C ABI in path order."""
 
     def __init__(self, B, Hq, Hkv, D, C, L, k, max_unique_len, dense=False, dense_slots=None,
-                 n_unique_splits=None, device="cuda"):
+                 n_unique_splits=None, device="cuda", fp8_unique=False):
         self.device = torch.device(device)
         self.dense = dense
         if n_unique_splits is None:
-            n_unique_splits = M.default_unique_splits(B, Hkv, max(1, max_unique_len))
+            default = M.default_unique_splits_fp8 if fp8_unique else M.default_unique_splits
+            n_unique_splits = default(B, Hkv, max(1, max_unique_len))
         if dense:
             shared_slots = dense_slots if dense_slots is not None else min(C, 16)
             k = C
