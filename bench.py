@@ -259,6 +259,14 @@ def run_cuda(args, w):
         raise SystemExit(f"workload {w.name} needs {need/1e9:.1f} GB, only {free/1e9:.1f} GB free")
     sh = W.make_shared_store(wr, dev)
     un = W.make_unique_store(wr, dev)
+    # --q-len T: every request brings T query tokens (speculative decoding); the batch rows are
+    # requests x T, token i of a request sees its context up to T - 1 - i tokens from the end
+    T = max(1, args.q_len)
+    if T > 1:
+        if args.unique_kv == "fp8" or w.D != 128 or T * w.G > 16:
+            raise SystemExit("--q-len needs the bf16 private store, head dimension 128 and q_len * G <= 16")
+        w = W.scaled(w, B=w.B * T)
+        wr = W.scaled(wr, B=wr.B * T)
     fp8 = args.unique_kv == "fp8"
     f8 = None
     if fp8:
@@ -272,7 +280,7 @@ def run_cuda(args, w):
     kv_lens = [(un.kv_len + s).to(torch.int32) for s in range(n_q)]
     max_len = int(lens0.max()) + w.steps
     layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, max_len, dense=w.dense,
-                       n_unique_splits=args.unique_splits, fp8_unique=fp8)
+                       n_unique_splits=args.unique_splits, fp8_unique=fp8, q_len=T)
     S = layer.shape
     if not w.dense:
         layer.build_summaries(sh.k_shared)
@@ -431,6 +439,8 @@ def run_cuda(args, w):
     t_bytes = work["shared_bytes"] / (peaks["hbm_gbs"] * 1e9)
     if unique_ms >= shared_ms:
         kernel = "unique_fp8_kernel" if fp8 else ("unique_staged_kernel" if w.D == 128 else "unique_attn_kernel")
+        if T > 1:
+            kernel = "unique_multi_kernel"
         roof = dict(bound="hbm", achieved=unique_gbs, peak=peaks["hbm_gbs"], unit="GB/s")
     elif t_flops > t_bytes:
         kernel = "shared_tc_kernel"
@@ -447,7 +457,7 @@ def run_cuda(args, w):
 
     # ---- CPU baseline: the oracle as it stands on the host cores, bounded sample (N = 1 only)
     cpu = None
-    if world == 1 and not args.no_cpu_baseline and not fp8:
+    if world == 1 and not args.no_cpu_baseline and not fp8 and T == 1:
         from oracle import oracle as O
 
         O.build()
@@ -485,6 +495,7 @@ def run_cuda(args, w):
             "unique_tokens_mean": float(lens.mean()), "n_unique_splits": S.n_unique_splits,
             "shared_slots": S.shared_slots, "streams": 2 if two_streams else 1,
             "unique_kv": "fp8_e4m3 + fp32 scale per (token, kv head)" if fp8 else "bf16",
+            "q_len": T, "requests": w.B // T,
             "l2": ("flushed between steps" if flush is not None
                    else f"inputs exceed L2 ({input_bytes / 2**20:.0f} MiB of K/V per step)"),
             "per_gpu": "own request batch, own copy of the shared store" if world > 1 else "single GPU",
@@ -534,6 +545,8 @@ def main():
     ap.add_argument("--unique-splits", type=int, default=None, help="override the split-K count of unique attention")
     ap.add_argument("--unique-kv", default="bf16", choices=["bf16", "fp8"],
                     help="storage of the private KV (fp8: E4M3 codes with per-token scales; no CPU baseline)")
+    ap.add_argument("--q-len", type=int, default=1,
+                    help="query tokens per request (batch rows = requests x q_len; queries/s counts rows; no CPU baseline)")
     ap.add_argument("--no-baseline", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-sample", type=int, default=16, help="requests in the CPU-oracle sample")

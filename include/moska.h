@@ -67,6 +67,15 @@ typedef struct moska_shape {
                              /* the host knows them, else 0.  Only moska_decode_step reads it,   */
                              /* to divide the SMs between shared and unique attention; results   */
                              /* never depend on it                                               */
+    int32_t q_len;           /* query tokens per request (speculative decoding, chunked prefill;  */
+                             /* Section II-A's multi-turn reuse): 0 or 1 = one.  With q_len > 1   */
+                             /* the B batch rows are B / q_len requests, row b = r * q_len + i is */
+                             /* token i of request r, kv_start / kv_len have B / q_len entries,   */
+                             /* kv_len[r] counts the tokens the LAST query token sees and token i */
+                             /* sees the first kv_len[r] - (q_len - 1 - i) of them.  Routing and  */
+                             /* shared attention treat every row as a request of its own; unique  */
+                             /* attention reads the request's K/V once for all its rows (needs    */
+                             /* D = 128, bf16 store, q_len * G <= 16)                             */
 } moska_shape;
 
 typedef void* moska_stream; /* a cudaStream_t */

@@ -26,7 +26,7 @@ _lib = ctypes.CDLL(LIB_PATH)
 class MoskaShape(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int32) for n in
                 ("B", "Hq", "Hkv", "D", "C", "L", "k", "shared_slots", "n_unique_splits")] + \
-               [("unique_tokens", ctypes.c_int64)]
+               [("unique_tokens", ctypes.c_int64), ("q_len", ctypes.c_int32)]
 
 
 class MoskaError(RuntimeError):
@@ -70,9 +70,9 @@ for _name, (_res, _args) in EXPORTS.items():
     _fn.argtypes = _args
 
 
-def shape(B, Hq, Hkv, D, C, L, k, shared_slots=None, n_unique_splits=1) -> MoskaShape:
+def shape(B, Hq, Hkv, D, C, L, k, shared_slots=None, n_unique_splits=1, q_len=0) -> MoskaShape:
     return MoskaShape(B, Hq, Hkv, D, C, L, k, k if shared_slots is None else shared_slots,
-                      n_unique_splits, 0)
+                      n_unique_splits, 0, q_len)
 
 
 def _ptr(t) -> Optional[int]:

@@ -38,6 +38,8 @@ int check_shape(const moska_shape* s, bool needs_k)
         return fail(MOSKA_ERR_INVALID_ARG, "k = %d outside [1, C = %d]", s->k, s->C);
     if (s->shared_slots < 1 || s->n_unique_splits < 1)
         return fail(MOSKA_ERR_INVALID_ARG, "shared_slots and n_unique_splits must be >= 1");
+    if (s->q_len < 0 || (s->q_len > 1 && s->B % s->q_len != 0))
+        return fail(MOSKA_ERR_INVALID_ARG, "q_len = %d must be >= 0 and divide B = %d", s->q_len, s->B);
     if ((long long)s->B * s->Hkv * (long long)(s->k > 0 ? s->k : 1) > 0x7fffffffLL ||
         (long long)s->Hkv * s->C >= 0x7fffffffLL)
         return fail(MOSKA_ERR_UNSUPPORTED, "index range exceeds int32");
@@ -296,6 +298,10 @@ int moska_unique_attn(const uint16_t* q, const uint16_t* k_unique, const uint16_
                       moska_stream stream)
 {
     MOSKA_TRY(check_shape(shape, false));
+    if (shape->q_len > 1 && (shape->D != 128 || shape->q_len * (shape->Hq / shape->Hkv) > 16))
+        return fail(MOSKA_ERR_UNSUPPORTED,
+                    "q_len = %d needs D = 128 and q_len * G <= 16; pass the tokens as batch rows "
+                    "with q_len = 1 and aliased kv_start instead", shape->q_len);
     MOSKA_TRY(check_device());
     REQUIRE_PTR(q, 16);
     REQUIRE_PTR(k_unique, 16);
@@ -315,6 +321,8 @@ int moska_unique_attn_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v
 {
     MOSKA_TRY(check_shape(shape, false));
     if (shape->D != 128) return fail(MOSKA_ERR_UNSUPPORTED, "FP8 unique attention is built for D = 128");
+    if (shape->q_len > 1)
+        return fail(MOSKA_ERR_UNSUPPORTED, "FP8 unique attention takes one query token per request");
     MOSKA_TRY(check_device());
     REQUIRE_PTR(q, 16);
     REQUIRE_PTR(k8, 16);

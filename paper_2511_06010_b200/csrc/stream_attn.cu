@@ -98,6 +98,47 @@ unique_staged_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict_
     attend_stream_staged<1>(rows, kb, vb, stride, t0, t1, scale, ring);
 }
 
+// ---- Unique KV Attention for several query tokens per request (D = 128) -------------------------
+// The q_len query tokens of request r are the batch rows r * q_len + i; token i sees the first
+// kv_len[r] - (q_len - 1 - i) tokens of the request's context.  Their q_len * G query rows of one
+// KV head share one pass over the request's K/V (one CTA per (request, KV head, split)).
+template <int NT>
+__global__ void __launch_bounds__(kThreads, 2)
+unique_multi_kernel(const uint16_t* __restrict__ q, const uint16_t* __restrict__ k_unique,
+                    const uint16_t* __restrict__ v_unique, const int64_t* __restrict__ kv_start,
+                    const int32_t* __restrict__ kv_len, float* __restrict__ o_part,
+                    float* __restrict__ lse_part, float scale, int Hq, int Hkv, int n_splits,
+                    int slot0, int n_slots, int q_len)
+{
+    constexpr int D = 128;
+    extern __shared__ __align__(128) unsigned char ring[];
+    __shared__ TileRows<NT> rows;
+    __shared__ int row_last[NT * 8];
+    const int G = Hq / Hkv;
+    const int h = blockIdx.x % Hkv;
+    const int s = (blockIdx.x / Hkv) % n_splits;
+    const int r = blockIdx.x / (Hkv * n_splits);
+    const int len = kv_len[r];
+    clear_rows(rows);
+    if (threadIdx.x < NT * 8) row_last[threadIdx.x] = 0x7fffffff;
+    __syncthreads();
+    if (threadIdx.x < q_len * G) {
+        const int i = threadIdx.x / G, g = threadIdx.x % G;
+        const int64_t row = ((int64_t)r * q_len + i) * Hq + h * G + g;
+        rows.q[threadIdx.x] = q + row * D;
+        rows.o[threadIdx.x] = o_part + (row * n_slots + slot0 + s) * D;
+        rows.lse[threadIdx.x] = lse_part + row * n_slots + slot0 + s;
+        row_last[threadIdx.x] = len - 1 - (q_len - 1 - i);
+    }
+    __syncthreads();
+    int t0, t1;
+    split_range(len, n_splits, s, t0, t1);
+    const int64_t stride = (int64_t)Hkv * D;
+    const uint16_t* kb = k_unique + kv_start[r] * stride + (int64_t)h * D;
+    const uint16_t* vb = v_unique + kv_start[r] * stride + (int64_t)h * D;
+    attend_stream_staged<NT, true>(rows, kb, vb, stride, t0, t1, scale, ring, row_last);
+}
+
 // ---- per-request GEMV baseline over shared chunks: one CTA per (request, KV head, slot) ---------
 template <int D>
 __global__ void __launch_bounds__(kThreads, D == 128 ? 2 : 3)
@@ -219,6 +260,27 @@ int launch_unique(const uint16_t* q, const uint16_t* k_unique, const uint16_t* v
     const long long grid = (long long)s->B * s->Hkv * s->n_unique_splits;
     if (grid == 0) return MOSKA_OK;
     if (grid > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "unique attention grid too large");
+    if (s->q_len > 1) {
+        // several query tokens per request: their rows share one pass over the request's K/V
+        constexpr int kRing = kWarps * kStagedWarpBytes;
+        const int rows = s->q_len * (s->Hq / s->Hkv);
+        const unsigned grid_r = (unsigned)(grid / s->q_len);
+        if (rows <= 8) {
+            MOSKA_CUDA_TRY(cudaFuncSetAttribute(unique_multi_kernel<1>,
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, kRing));
+            unique_multi_kernel<1><<<grid_r, kThreads, kRing, st>>>(
+                q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part, scale, s->Hq, s->Hkv,
+                s->n_unique_splits, s->shared_slots, n_slots, s->q_len);
+        } else {
+            MOSKA_CUDA_TRY(cudaFuncSetAttribute(unique_multi_kernel<2>,
+                                                cudaFuncAttributeMaxDynamicSharedMemorySize, kRing));
+            unique_multi_kernel<2><<<grid_r, kThreads, kRing, st>>>(
+                q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part, scale, s->Hq, s->Hkv,
+                s->n_unique_splits, s->shared_slots, n_slots, s->q_len);
+        }
+        MOSKA_LAUNCH_CHECK("unique_multi_kernel");
+        return MOSKA_OK;
+    }
     if (s->D == 128) {
         constexpr int kRing = kWarps * kStagedWarpBytes;
         MOSKA_CUDA_TRY(cudaFuncSetAttribute(unique_staged_kernel,

@@ -329,11 +329,14 @@ __device__ __forceinline__ uint4 lds16(uint32_t addr)
 // D = 128, NT column blocks of 8 query rows, the kWarps warps of the CTA take interleaved tiles.
 // `ring` is the CTA's staging memory (kWarps * kStagedWarpBytes bytes, 128-byte aligned); the
 // final combination of the warps reuses it.  All threads of the CTA must call this.
-template <int NT>
+// With kRowLast, row r only sees the tokens up to index row_last[r] of the stream (several query
+// tokens of one request, each one token further into the same context); `row_last` is an array of
+// NT * 8 ints visible to all threads.
+template <int NT, bool kRowLast = false>
 __device__ __forceinline__ void attend_stream_staged(const TileRows<NT>& rows, const uint16_t* k_base,
                                                      const uint16_t* v_base, int64_t tok_stride,
                                                      int t_begin, int t_end, float scale,
-                                                     unsigned char* ring)
+                                                     unsigned char* ring, const int* row_last = nullptr)
 {
     constexpr int D = 128, KU = 4, VL = 2, MT = 8;
     static_assert(sizeof(CombineSmem<D, NT>) <= kWarps * kStagedWarpBytes, "the combine step reuses the ring");
@@ -364,6 +367,17 @@ __device__ __forceinline__ void attend_stream_staged(const TileRows<NT>& rows, c
     const int n_tiles = (n_tok + kTileTokens - 1) / kTileTokens;
     const int last_tok = t_end - 1;
     const int my_tiles = n_tiles > warp ? (n_tiles - warp + kWarps - 1) / kWarps : 0;
+    // last visible token of the two query rows (columns 2c, 2c+1 of block n) this lane holds scores of
+    int lim[NT][2];
+    int min_last = last_tok;
+    if constexpr (kRowLast) {
+#pragma unroll
+        for (int n = 0; n < NT; ++n) {
+            lim[n][0] = row_last[n * 8 + 2 * c];
+            lim[n][1] = row_last[n * 8 + 2 * c + 1];
+        }
+        for (int r = 0; r < NT * 8; ++r) min_last = min(min_last, row_last[r]);
+    }
     const uint32_t ring_base = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + warp * kStagedWarpBytes;
     // chunk `ch` of token row `t` (0..15) of the K (kv = 0) or V (kv = 1) tile in ring stage s
     auto slot = [&](int s, int kv, int t, int ch) {
@@ -418,6 +432,14 @@ __device__ __forceinline__ void attend_stream_staged(const TileRows<NT>& rows, c
         for (int n = 0; n < NT; ++n) {
             if (!va) sc[n][0] = sc[n][1] = -INFINITY;
             if (!vb) sc[n][2] = sc[n][3] = -INFINITY;
+            if constexpr (kRowLast) {
+                if (t0 + kTileTokens - 1 > min_last) {  // the tile reaches past some row's context
+                    if (t0 + g > lim[n][0]) sc[n][0] = -INFINITY;
+                    if (t0 + g > lim[n][1]) sc[n][1] = -INFINITY;
+                    if (t0 + 8 + g > lim[n][0]) sc[n][2] = -INFINITY;
+                    if (t0 + 8 + g > lim[n][1]) sc[n][3] = -INFINITY;
+                }
+            }
             float mx0 = fmaxf(sc[n][0], sc[n][2]), mx1 = fmaxf(sc[n][1], sc[n][3]);
 #pragma unroll
             for (int off = 4; off < 32; off <<= 1) {
@@ -430,7 +452,12 @@ __device__ __forceinline__ void attend_stream_staged(const TileRows<NT>& rows, c
             alpha[n][1] = fast_exp2((m_run[n][1] - mn1) * sl2);
             m_run[n][0] = mn0;
             m_run[n][1] = mn1;
-            const float ms0 = mn0 * sl2, ms1 = mn1 * sl2;
+            float ms0 = mn0 * sl2, ms1 = mn1 * sl2;
+            if constexpr (kRowLast) {
+                // a row that has seen no token yet: keep its (empty) state free of inf - inf
+                if (mn0 == -INFINITY) { alpha[n][0] = 1.f; ms0 = 0.f; }
+                if (mn1 == -INFINITY) { alpha[n][1] = 1.f; ms1 = 0.f; }
+            }
             const float p0 = fast_exp2(fmaf(sc[n][0], sl2, -ms0)), p1 = fast_exp2(fmaf(sc[n][1], sl2, -ms1));
             const float p2 = fast_exp2(fmaf(sc[n][2], sl2, -ms0)), p3 = fast_exp2(fmaf(sc[n][3], sl2, -ms1));
             l_run[n][0] = fmaf(l_run[n][0], alpha[n][0], p0 + p2);

@@ -14,18 +14,19 @@ class MoskaLayer:
     """Owns the scratch of a decode step for a fixed shape and calls the C ABI in path order."""
 
     def __init__(self, B, Hq, Hkv, D, C, L, k, max_unique_len, dense=False, dense_slots=None,
-                 n_unique_splits=None, device="cuda", fp8_unique=False):
+                 n_unique_splits=None, device="cuda", fp8_unique=False, q_len=1):
+        """B counts batch rows; with q_len > 1 they are B / q_len requests of q_len query tokens."""
         self.device = torch.device(device)
         self.dense = dense
         if n_unique_splits is None:
             default = M.default_unique_splits_fp8 if fp8_unique else M.default_unique_splits
-            n_unique_splits = default(B, Hkv, max(1, max_unique_len))
+            n_unique_splits = default(B // max(1, q_len), Hkv, max(1, max_unique_len))
         if dense:
             shared_slots = dense_slots if dense_slots is not None else min(C, 16)
             k = C
         else:
             shared_slots = k
-        self.shape = M.shape(B, Hq, Hkv, D, C, L, k, shared_slots, n_unique_splits)
+        self.shape = M.shape(B, Hq, Hkv, D, C, L, k, shared_slots, n_unique_splits, q_len)
         self.n_slots = M.partial_slots(self.shape)
         self.scale = 1.0 / math.sqrt(D)
         dev = self.device

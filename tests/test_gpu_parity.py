@@ -360,6 +360,49 @@ def test_several_query_tokens_per_request_by_batch_expansion():
     assert M.device_status() == 0
 
 
+def test_several_query_tokens_per_request_native():
+    """shape.q_len > 1: unique attention reads a request's K/V once for all its query tokens (token
+    i sees kv_len - (q_len - 1 - i) tokens).  The definition is the batch-expanded problem, which
+    is what the oracle is given; also bit-compatible slots: partials per row, merged as usual.
+    Covers G * q_len <= 8 and <= 16, contexts shorter than q_len, empty ones, several splits."""
+    M, MoskaLayer = _mods()
+    for Hq, Hkv, t, splits in ((8, 2, 2, 1), (8, 2, 4, 3), (16, 2, 2, 2), (6, 2, 5, 2), (4, 4, 3, 1)):
+        lens_last = np.array([40, 1, 130, 77, 300, 16, 2, 0, 1000, 65], dtype=np.int64)
+        base = len(lens_last)
+        w = W.Workload("multi", B=base * t, Hq=Hq, Hkv=Hkv, D=128, C=8, L=256, k=2, unique_len=0, seed=43)
+        sh = W.make_shared_store(w, "cuda")
+        un = W.make_unique_store(W.scaled(w, B=base, steps=0), "cuda", lens_last)
+        q = W.make_queries(w, sh, 0, "cuda")
+        layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, int(lens_last.max()),
+                           n_unique_splits=splits, q_len=t)
+        layer.build_summaries(sh.k_shared)
+        out = layer.step(q, sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, un.kv_start, un.kv_len)
+        torch.cuda.synchronize()
+        # the same problem with every query token as a request of its own
+        kv_start = un.kv_start.repeat_interleave(t).cpu().numpy()
+        back = np.tile(np.arange(t - 1, -1, -1), base)
+        kv_len = np.maximum(0, np.repeat(lens_last, t) - back).astype(np.int32)
+        ref, ref_lse = O.attend_direct(q.cpu(), sh.k_shared.cpu(), sh.v_shared.cpu(), un.k_unique.cpu(),
+                                       un.v_unique.cpu(), kv_start, kv_len,
+                                       layer.topk_idx.cpu().numpy(), layer.scale)
+        PU.check_attention(out.float().cpu().numpy(), ref, f"q_len={t} G={Hq // Hkv} out")
+        PU.check_lse(layer.lse_out.cpu().numpy(), ref_lse, f"q_len={t} lse")
+        # the unique partials alone: rows that see no private token carry lse = -inf, o = 0
+        n_sh = layer.shape.shared_slots
+        l_un = layer.lse_part[:, :, n_sh:].cpu().numpy()
+        o_un = layer.o_part[:, :, n_sh:].cpu().numpy()
+        empty = kv_len == 0
+        assert np.isneginf(l_un[empty]).all() and (o_un[empty] == 0).all()
+        assert np.isfinite(o_un).all() and not np.isnan(l_un).any()
+        assert M.device_status() == 0
+    # beyond 16 rows per (request, KV head) the call says so instead of computing something else
+    big = MoskaLayer(8, 32, 4, 128, 8, 256, 2, 64, q_len=4)
+    with pytest.raises(M.MoskaError) as err:
+        big.unique(torch.zeros(8, 32, 128, dtype=torch.bfloat16, device="cuda"), un.k_unique, un.v_unique,
+                   un.kv_start, un.kv_len)
+    assert err.value.status == M.ERR_UNSUPPORTED
+
+
 def test_decode_step_can_be_captured_in_a_cuda_graph():
     """Nothing in the step reads device results back on the host, so the whole two-stream step
     (fork and join included) is one CUDA graph; replaying it gives the eager result bit for bit."""
