@@ -205,7 +205,7 @@ __device__ __forceinline__ Item decode_item(const TcParams& p, int item, int G, 
 // Roles of the third warp group (after it has given registers up): TMA producer, MMA issuer and
 // the two query-gather warps.
 __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
-                                         const TcParams& p, int n_items, int G, int per_tile,
+                                         const CUtensorMap& tm_q, const TcParams& p, int n_items, int G, int per_tile,
                                          uint32_t tmem, int warp, int lane)
 {
     volatile int* ab = &sm.abort_flag;
@@ -240,19 +240,22 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
         __syncwarp();
     } else if (warp >= kGatherWarp0) {
         // =========================== query gather of tile u ======================================
-        // Copies the tile's query rows into the 128-byte-swizzled K-major operand layout as soon
-        // as the MMAs of the previous item have stopped reading the buffer.
+        // Brings the tile's query rows into the 128-byte-swizzled K-major operand layout as soon
+        // as the MMAs of the previous item have stopped reading the buffer: TMA row gathers, four
+        // rows per copy (lane l owns tile rows 4l .. 4l+3), so the copies do not queue behind the
+        // softmax groups' result stores in the load/store pipe.  Rows past the item's last one hold
+        // stale or repeated query rows; their results are never written.
         const int u = warp - kGatherWarp0;
         uint32_t uses = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
             const Item it = decode_item(p, item, G, per_tile);
             if (it.n_kv == 0 || it.n_e[u] == 0) continue;
-            long long rr[4];  // global query row of tile rows lane, lane + 32, lane + 64, lane + 96
+            int rr[4];  // global query rows of tile rows 4 * lane .. 4 * lane + 3
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
-                const int i = lane + 32 * m;
-                rr[m] = -1;
+                const int i = 4 * lane + m;
+                rr[m] = 0;
                 if (i < it.n_e[u] * G) {
                     const int e = i / G, g = i % G;
                     int b;
@@ -260,7 +263,7 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
                         b = __ldg(p.seg_entries + it.entry_begin + u * per_tile + e) / (p.k * p.Hkv);
                     else
                         b = it.b0 + u * per_tile + e;
-                    rr[m] = (long long)b * p.Hq + it.h * G + g;
+                    rr[m] = b * p.Hq + it.h * G + g;
                 }
             }
             if (uses > 0) {
@@ -268,24 +271,21 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
                 if (!ok) break;
             }
             ++uses;
-            const uint32_t q_base = smem_u32(sm.q[u]);
-#pragma unroll
-            for (int m = 0; m < 4; ++m) {
-#pragma unroll 4
-                for (int n = 0; n < 16; ++n) {
-                    const int lr = 2 * n + (lane >> 4), c = lane & 15;
-                    const long long src_row = __shfl_sync(0xffffffffu, rr[m], lr);
-                    const int row = 32 * m + lr;
-                    const uint32_t dst = q_base + (c >> 3) * kHalfBytes + row * 128 + (((c & 7) ^ (row & 7)) << 4);
-                    const uint16_t* src = src_row >= 0 ? p.q + src_row * kD + c * 8 : p.q;
-                    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src),
-                                 "r"(src_row >= 0 ? 16 : 0)
-                                 : "memory");
-                }
+            // only the groups of four rows that hold a query row are copied; the tile rows after
+            // them keep whatever an earlier item left there
+            const int n_groups = (it.n_e[u] * G + 3) >> 2;
+            if (lane == 0) mbar_arrive_expect_tx(&sm.q_full[u], n_groups * 2 * (4 * 128));
+            __syncwarp();
+            if (lane < n_groups) {
+                uint8_t* dst = sm.q[u] + lane * (4 * 128);
+                tma_gather4_2d(dst, &tm_q, 0, rr[0], rr[1], rr[2], rr[3], &sm.q_full[u]);
+                tma_gather4_2d(dst + kHalfBytes, &tm_q, 64, rr[0], rr[1], rr[2], rr[3], &sm.q_full[u]);
             }
-            asm volatile("cp.async.wait_all;" ::: "memory");
-            fence_proxy_async_smem();
-            mbar_arrive(&sm.q_full[u]);
+        }
+        if (*ab && uses > 0) {
+            // giving up: let the copies still in flight land before the CTA leaves
+            volatile int never = 0;
+            mbar_wait(&sm.q_full[u], (uses - 1) & 1, &never);
         }
     } else {
         // =========================== MMA issuer ===================================================
@@ -387,7 +387,7 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
 
 __global__ void __launch_bounds__(kThreads, 1)
 shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
-                 const TcParams p)
+                 const __grid_constant__ CUtensorMap tm_q, const TcParams p)
 {
     extern __shared__ uint8_t smem_raw[];
     TcSmem& sm = *reinterpret_cast<TcSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
@@ -405,7 +405,7 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             mbar_init(&sm.empty[s], 1);
         }
         for (int u = 0; u < 2; ++u) {
-            mbar_init(&sm.q_full[u], 32);
+            mbar_init(&sm.q_full[u], 1);
             mbar_init(&sm.q_free[u], 1);
             mbar_init(&sm.s_full[u], 1);
             mbar_init(&sm.p_full[u], 128);
@@ -424,6 +424,7 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     if (warp == kMmaWarp && lane == 0) {
         tma_prefetch_desc(&tm_k);
         tma_prefetch_desc(&tm_v);
+        tma_prefetch_desc(&tm_q);
     }
     tc_fence_before_sync();
     __syncthreads();
@@ -629,7 +630,7 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         }
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
-        other_roles(sm, tm_k, tm_v, p, n_items, G, per_tile, tmem, warp, lane);
+        other_roles(sm, tm_k, tm_v, tm_q, p, n_items, G, per_tile, tmem, warp, lane);
     }
 
     // ---- teardown -------------------------------------------------------------------------------
@@ -680,6 +681,23 @@ int make_kv_map(CUtensorMap* tm, const uint16_t* base, long long rows)
     return MOSKA_OK;
 }
 
+// The [rows][128] bf16 query matrix for row gathers: boxes of one row x 64 columns.
+int make_q_map(CUtensorMap* tm, const uint16_t* base, long long rows)
+{
+    EncodeTiledFn enc = nullptr;
+    MOSKA_TRY_STATUS(encoder(&enc));
+    const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)kD * 2};
+    const cuuint32_t box[2] = {64, 1};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                           const_cast<uint16_t*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(MOSKA_ERR_CUDA, "cuTensorMapEncodeTiled failed for q (%d)", (int)r);
+    return MOSKA_OK;
+}
+
 }  // namespace
 
 bool shared_tc_supported(const moska_shape* s) { return s->D == kD && s->L % kKvTile == 0; }
@@ -711,9 +729,10 @@ int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t
     if (max_ctas > 0 && grid > max_ctas) grid = max_ctas;  // the caller keeps the other SMs for another kernel
     const long long kv_rows = (long long)s->Hkv * s->C * s->L;
     if (kv_rows > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "shared store exceeds 2^31 tokens");
-    CUtensorMap tm_k, tm_v;
+    CUtensorMap tm_k, tm_v, tm_q;
     MOSKA_TRY_STATUS(make_kv_map(&tm_k, k_shared, kv_rows));
     MOSKA_TRY_STATUS(make_kv_map(&tm_v, v_shared, kv_rows));
+    MOSKA_TRY_STATUS(make_q_map(&tm_q, q, (long long)s->B * s->Hq));
     int* status = nullptr;
     MOSKA_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_tc_status));
     p.q = q;
@@ -733,7 +752,7 @@ int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t
     p.dense = dense ? 1 : 0;
     const int smem = (int)sizeof(TcSmem) + 1024;
     MOSKA_CUDA_TRY(cudaFuncSetAttribute(shared_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    shared_tc_kernel<<<(unsigned)grid, kThreads, smem, st>>>(tm_k, tm_v, p);
+    shared_tc_kernel<<<(unsigned)grid, kThreads, smem, st>>>(tm_k, tm_v, tm_q, p);
     MOSKA_LAUNCH_CHECK("shared_tc_kernel");
     return MOSKA_OK;
 }

@@ -111,6 +111,19 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const void* tmap, in
         : "memory");
 }
 
+// Four rows y0..y3 of a 2-D tensor (tensor map with a box one row high) -> four consecutive rows of
+// a shared-memory tile; x as above.  Completion is counted in bytes on `bar`.
+__device__ __forceinline__ void tma_gather4_2d(void* smem_dst, const void* tmap, int x, int y0, int y1,
+                                               int y2, int y3, uint64_t* bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile::gather4.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%2, %3, %4, %5, %6}], [%7];"
+        ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(x), "r"(y0), "r"(y1),
+        "r"(y2), "r"(y3), "r"(smem_u32(bar))
+        : "memory");
+}
+
 // ---- tensor memory -----------------------------------------------------------------------------
 // All four of these are warp-collective (.sync.aligned): call them with the whole warp converged.
 __device__ __forceinline__ void tmem_alloc(uint32_t* smem_result, uint32_t n_cols)
