@@ -43,6 +43,10 @@ def test_pure_host_helpers(M):
     assert 1 <= M.default_unique_splits(64, 8, 4096) <= 8
     assert M.default_unique_splits(1024, 8, 32768) >= 1
     assert M.default_unique_splits(4, 1, 100) == 1
+    # the FP8 kernel has shorter-lived CTAs: never fewer splits than one, capped by the context
+    assert M.default_unique_splits_fp8(64, 8, 4096) == 4
+    assert M.default_unique_splits_fp8(4, 1, 100) == 1
+    assert 1 <= M.default_unique_splits_fp8(1, 8, 1 << 20) <= 64
 
 
 @pytest.mark.parametrize("kwargs,status", [
@@ -52,6 +56,8 @@ def test_pure_host_helpers(M):
     (dict(L=100), -2),            # L not a multiple of 128
     (dict(k=0), -1),
     (dict(k=129), -1),            # k > C
+    (dict(q_len=3), -1),          # q_len does not divide B
+    (dict(q_len=-1), -1),
 ])
 def test_bad_shapes_are_rejected_on_the_host(M, kwargs, status):
     base = dict(B=4, Hq=32, Hkv=8, D=128, C=128, L=512, k=8)
@@ -69,6 +75,19 @@ def test_null_pointer_and_workspace_errors_come_before_any_launch(M):
         M.merge(None, 0x1000, 0x1000, None, None, s, stream=0)
     # NULL is reported as invalid argument unless the device check (no GPU here) comes first
     assert e.value.status in (M.ERR_INVALID_ARG, M.ERR_CUDA, M.ERR_UNSUPPORTED)
+    # several query tokens per request: more than 16 rows per (request, KV head), D = 64 and the
+    # FP8 store are refused before anything is launched
+    for kw, call in ((dict(Hq=64, q_len=4), "bf16"), (dict(D=64, q_len=2), "bf16"), (dict(q_len=2), "fp8")):
+        base = dict(B=4, Hq=32, Hkv=8, D=128, C=128, L=512, k=8)
+        base.update(kw)
+        sq = M.shape(**base)
+        with pytest.raises(M.MoskaError) as e:
+            if call == "bf16":
+                M.unique_attn(0x1000, 0x1000, 0x1000, 0x1000, 0x1000, 0x1000, 0x1000, 1.0, sq, stream=0)
+            else:
+                M.unique_attn_fp8(0x1000, 0x1000, 0x1000, 0x1000, 0x1000, 0x1000, 0x1000, 0x1000, 0x1000,
+                                  1.0, sq, stream=0)
+        assert e.value.status == M.ERR_UNSUPPORTED
     bad = M.shape(4, 32, 8, 128, 128, 512, 8, shared_slots=0)
     with pytest.raises(M.MoskaError) as e:
         M.partial_slots(bad)
