@@ -403,6 +403,31 @@ def test_several_query_tokens_per_request_native():
     assert err.value.status == M.ERR_UNSUPPORTED
 
 
+def test_host_buffer_step_equals_device_step():
+    """moska_decode_step_host: q from host memory, result into host memory, bit-identical to the
+    device-buffer step, from page-locked and from pageable host buffers, one and two streams."""
+    M, MoskaLayer = _mods()
+    w = W.scaled(W.CONFIGS[1], B=24, C=16, k=4, unique_len=700)
+    sh = W.make_shared_store(w, "cuda")
+    un = W.make_unique_store(w, "cuda")
+    q = W.make_queries(w, sh, 0, "cuda")
+    layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, 700)
+    layer.build_summaries(sh.k_shared)
+    ref = layer.step(q, sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, un.kv_start, un.kv_len).clone()
+    torch.cuda.synchronize()
+    q_dev = torch.empty_like(q)
+    for pinned, two in ((True, False), (False, False), (True, True)):
+        q_host = q.cpu().pin_memory() if pinned else q.cpu()
+        out_host = torch.zeros(w.B, w.Hq, w.D, dtype=torch.bfloat16)
+        if pinned:
+            out_host = out_host.pin_memory()
+        layer.out.zero_()
+        layer.step_host(q_host, q_dev, out_host, sh.k_shared, sh.v_shared, un.k_unique, un.v_unique,
+                        un.kv_start, un.kv_len, two_streams=two)
+        assert torch.equal(out_host, ref.cpu()), f"pinned={pinned} two_streams={two}"
+    assert M.device_status() == 0
+
+
 def test_decode_step_can_be_captured_in_a_cuda_graph():
     """Nothing in the step reads device results back on the host, so the whole two-stream step
     (fork and join included) is one CUDA graph; replaying it gives the eager result bit for bit."""
