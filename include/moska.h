@@ -254,6 +254,11 @@ int moska_gemv_baseline(const uint16_t* q, const uint16_t* k_shared, const uint1
 /* Creates a profiler able to hold `max_steps` recorded steps (host object owning CUDA events). */
 int moska_profiler_create(moska_profiler** out, int32_t max_steps);
 void moska_profiler_destroy(moska_profiler* prof);
+/* Restricts recording to the stages whose bit (1 << MOSKA_STAGE_x) is set in stage_mask (all
+ * stages by default).  Every recorded stage costs two event records per step on the stream it
+ * runs on -- about 3 us per stage on a B200 -- so a caller timing whole steps records only the
+ * stage it needs.  Stages that are not recorded read as 0. */
+int moska_profiler_select(moska_profiler* prof, uint32_t stage_mask);
 /* Waits for the recorded events, adds up the elapsed milliseconds per stage over the steps
  * recorded since the last read into stage_ms[MOSKA_N_STAGES] (host), stores their number in
  * *n_steps (host) and clears the profiler. */

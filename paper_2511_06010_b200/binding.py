@@ -62,6 +62,7 @@ EXPORTS = {
     "moska_decode_step_host": (_i, [_vp] * 16 + [_f, _sp, _vp, _sz, _vp, _vp, _vp]),
     "moska_profiler_create": (_i, [ctypes.POINTER(_vp), ctypes.c_int32]),
     "moska_profiler_destroy": (None, [_vp]),
+    "moska_profiler_select": (_i, [_vp, ctypes.c_uint32]),
     "moska_profiler_read": (_i, [_vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_int32)]),
 }
 for _name, (_res, _args) in EXPORTS.items():
@@ -243,6 +244,14 @@ def profiler_create(max_steps: int):
 
 def profiler_destroy(prof) -> None:
     _lib.moska_profiler_destroy(prof)
+
+
+def profiler_select(prof, stages) -> None:
+    """Record only the named stages (an iterable of names from STAGES)."""
+    mask = 0
+    for name in stages:
+        mask |= 1 << STAGES.index(name)
+    _check(_lib.moska_profiler_select(prof, mask), "moska_profiler_select")
 
 
 def profiler_read(prof):

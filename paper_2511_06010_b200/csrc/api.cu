@@ -71,13 +71,14 @@ struct moska_profiler {
     int n_steps = 0;
     cudaEvent_t* ev = nullptr;  // [max_steps][MOSKA_N_STAGES][2]
     bool* used = nullptr;       // [max_steps][MOSKA_N_STAGES]
+    unsigned mask = ~0u;        // stages that are recorded (bit = stage index)
 };
 
 namespace {
 // Records the begin/end event of one stage of the step being recorded (no-op without profiler).
 inline cudaError_t prof_mark(moska_profiler* p, int stage, int which, cudaStream_t st)
 {
-    if (p == nullptr || p->n_steps >= p->max_steps) return cudaSuccess;
+    if (p == nullptr || p->n_steps >= p->max_steps || !((p->mask >> stage) & 1u)) return cudaSuccess;
     const int i = p->n_steps * MOSKA_N_STAGES + stage;
     p->used[i] = true;
     return cudaEventRecord(p->ev[2 * i + which], st);
@@ -556,6 +557,13 @@ void moska_profiler_destroy(moska_profiler* p)
     delete[] p->ev;
     delete[] p->used;
     delete p;
+}
+
+int moska_profiler_select(moska_profiler* p, uint32_t stage_mask)
+{
+    if (p == nullptr) return fail(MOSKA_ERR_INVALID_ARG, "profiler is NULL");
+    p->mask = stage_mask;
+    return MOSKA_OK;
 }
 
 int moska_profiler_read(moska_profiler* p, float* stage_ms, int32_t* n_steps)
