@@ -263,8 +263,8 @@ def run_cuda(args, w):
     # requests x T, token i of a request sees its context up to T - 1 - i tokens from the end
     T = max(1, args.q_len)
     if T > 1:
-        if args.unique_kv == "fp8" or w.D != 128 or T * w.G > 16:
-            raise SystemExit("--q-len needs the bf16 private store, head dimension 128 and q_len * G <= 16")
+        if w.D != 128 or T * w.G > (8 if args.unique_kv == "fp8" else 16):
+            raise SystemExit("--q-len needs head dimension 128 and q_len * G <= 16 (8 with --unique-kv fp8)")
         w = W.scaled(w, B=w.B * T)
         wr = W.scaled(wr, B=wr.B * T)
     fp8 = args.unique_kv == "fp8"
@@ -453,7 +453,7 @@ def run_cuda(args, w):
     t_bytes = work["shared_bytes"] / (peaks["hbm_gbs"] * 1e9)
     if unique_ms >= shared_ms:
         kernel = "unique_fp8_kernel" if fp8 else ("unique_staged_kernel" if w.D == 128 else "unique_attn_kernel")
-        if T > 1:
+        if T > 1 and not fp8:
             kernel = "unique_multi_kernel"
         roof = dict(bound="hbm", achieved=unique_gbs, peak=peaks["hbm_gbs"], unit="GB/s")
     elif t_flops > t_bytes:

@@ -75,7 +75,7 @@ typedef struct moska_shape {
                              /* sees the first kv_len[r] - (q_len - 1 - i) of them.  Routing and  */
                              /* shared attention treat every row as a request of its own; unique  */
                              /* attention reads the request's K/V once for all its rows (needs    */
-                             /* D = 128, bf16 store, q_len * G <= 16)                             */
+                             /* D = 128 and q_len * G <= 16; <= 8 with the FP8 store)             */
 } moska_shape;
 
 typedef void* moska_stream; /* a cudaStream_t */

@@ -322,8 +322,10 @@ int moska_unique_attn_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v
 {
     MOSKA_TRY(check_shape(shape, false));
     if (shape->D != 128) return fail(MOSKA_ERR_UNSUPPORTED, "FP8 unique attention is built for D = 128");
-    if (shape->q_len > 1)
-        return fail(MOSKA_ERR_UNSUPPORTED, "FP8 unique attention takes one query token per request");
+    if (shape->q_len > 1 && shape->q_len * (shape->Hq / shape->Hkv) > 8)
+        return fail(MOSKA_ERR_UNSUPPORTED,
+                    "FP8 unique attention with q_len = %d needs q_len * G <= 8; pass the tokens as "
+                    "batch rows with q_len = 1 and aliased kv_start instead", shape->q_len);
     MOSKA_TRY(check_device());
     REQUIRE_PTR(q, 16);
     REQUIRE_PTR(k8, 16);

@@ -75,7 +75,7 @@ unique_fp8_kernel(const uint16_t* __restrict__ q, const uint8_t* __restrict__ k8
                   const float* __restrict__ v_scale, const int64_t* __restrict__ kv_start,
                   const int32_t* __restrict__ kv_len, float* __restrict__ o_part,
                   float* __restrict__ lse_part, float scale, int Hq, int Hkv, int n_splits,
-                  int slot0, int n_slots)
+                  int slot0, int n_slots, int q_len)
 {
     constexpr int D = kD8, MT = 8;
     extern __shared__ __align__(128) unsigned char ring[];
@@ -84,8 +84,12 @@ unique_fp8_kernel(const uint16_t* __restrict__ q, const uint8_t* __restrict__ k8
     const int G = Hq / Hkv;
     const int h = blockIdx.x % Hkv;
     const int sp = (blockIdx.x / Hkv) % n_splits;
-    const int b = blockIdx.x / (Hkv * n_splits);
+    const int b = blockIdx.x / (Hkv * n_splits);  // request
     const float sl2 = scale * kLog2e;
+    // Query rows of this (request, KV head): row j = i * G + g' is head g' of query token i (one
+    // token unless q_len > 1), a batch row of its own that sees the context up to q_len - 1 - i
+    // tokens before its end.
+    const int n_rows = q_len * G;
 
     // token range of this split (same rule as the bf16 kernel: equal parts rounded up to 64)
     const int len = kv_len[b];
@@ -101,8 +105,8 @@ unique_fp8_kernel(const uint16_t* __restrict__ q, const uint8_t* __restrict__ k8
     const int64_t tok_stride = (int64_t)Hkv * D;  // bytes between consecutive tokens of one head
 
     // Q as the B operand in f16: step s = 4u + w covers dimensions 16 (2c + u) + 4 w .. + 3
-    const bool live = g < G;
-    const uint16_t* qp = q + ((int64_t)b * Hq + h * G + g) * D;
+    const bool live = g < n_rows;
+    const uint16_t* qp = q + (((int64_t)b * q_len + g / G) * Hq + h * G + g % G) * D;
     uint32_t qf[8][2];
 #pragma unroll
     for (int s = 0; s < 8; ++s) {
@@ -126,6 +130,11 @@ unique_fp8_kernel(const uint16_t* __restrict__ q, const uint8_t* __restrict__ k8
 
     const int n_tiles = (t_end - t_begin + kTileTokens - 1) / kTileTokens;
     const int last_tok = t_end - 1;
+    // last visible token of the two query rows (columns 2c, 2c + 1) this lane holds scores of
+    const int min_last = len - q_len;
+    int lim0 = 0x7fffffff, lim1 = 0x7fffffff;
+    if (2 * c < n_rows) lim0 = len - 1 - (q_len - 1 - (2 * c) / G);
+    if (2 * c + 1 < n_rows) lim1 = len - 1 - (q_len - 1 - (2 * c + 1) / G);
     const int my_tiles = n_tiles > warp ? (n_tiles - warp + kWarps - 1) / kWarps : 0;
     const uint32_t ring_base = static_cast<uint32_t>(__cvta_generic_to_shared(ring)) + warp * kF8WarpBytes;
     // 16-byte chunk `ch` (0..7) of token row t of the K (kv = 0) / V (kv = 1) tile in stage s
@@ -183,6 +192,12 @@ unique_fp8_kernel(const uint16_t* __restrict__ q, const uint8_t* __restrict__ k8
         const bool va = (t0 + g) <= last_tok, vb = (t0 + 8 + g) <= last_tok;
         if (!va) sc[0] = sc[1] = -INFINITY;
         if (!vb) sc[2] = sc[3] = -INFINITY;
+        if (t0 + kTileTokens - 1 > min_last) {  // q_len > 1: the tile reaches past some row's context
+            if (t0 + g > lim0) sc[0] = -INFINITY;
+            if (t0 + g > lim1) sc[1] = -INFINITY;
+            if (t0 + 8 + g > lim0) sc[2] = -INFINITY;
+            if (t0 + 8 + g > lim1) sc[3] = -INFINITY;
+        }
         float mx0 = fmaxf(sc[0], sc[2]), mx1 = fmaxf(sc[1], sc[3]);
 #pragma unroll
         for (int off = 4; off < 32; off <<= 1) {
@@ -191,10 +206,13 @@ unique_fp8_kernel(const uint16_t* __restrict__ q, const uint8_t* __restrict__ k8
         }
         const float mn0 = fmaxf(m_run[0], mx0), mn1 = fmaxf(m_run[1], mx1);
         const bool grew = (mn0 > m_run[0]) | (mn1 > m_run[1]);
-        const float al0 = fast_exp2((m_run[0] - mn0) * sl2), al1 = fast_exp2((m_run[1] - mn1) * sl2);
+        float al0 = fast_exp2((m_run[0] - mn0) * sl2), al1 = fast_exp2((m_run[1] - mn1) * sl2);
         m_run[0] = mn0;
         m_run[1] = mn1;
-        const float ms0 = mn0 * sl2, ms1 = mn1 * sl2;
+        float ms0 = mn0 * sl2, ms1 = mn1 * sl2;
+        // a row that has seen no token yet: keep its (empty) state free of inf - inf
+        if (mn0 == -INFINITY) { al0 = 1.f; ms0 = 0.f; }
+        if (mn1 == -INFINITY) { al1 = 1.f; ms1 = 0.f; }
         const float p0 = fast_exp2(fmaf(sc[0], sl2, -ms0)), p1 = fast_exp2(fmaf(sc[1], sl2, -ms1));
         const float p2 = fast_exp2(fmaf(sc[2], sl2, -ms0)), p3 = fast_exp2(fmaf(sc[3], sl2, -ms1));
         l_run[0] = fmaf(l_run[0], al0, p0 + p2);
@@ -256,8 +274,8 @@ unique_fp8_kernel(const uint16_t* __restrict__ q, const uint8_t* __restrict__ k8
     __syncthreads();
     for (int i = threadIdx.x; i < 8 * D; i += kThreads) {
         const int r = i / D, d = i % D;
-        if (r >= G) continue;
-        const int64_t row = (int64_t)b * Hq + h * G + r;
+        if (r >= n_rows) continue;
+        const int64_t row = ((int64_t)b * q_len + r / G) * Hq + h * G + r % G;
         float M = sm.m[0][r];
 #pragma unroll
         for (int w = 1; w < kWarps; ++w) M = fmaxf(M, sm.m[w][r]);
@@ -283,14 +301,15 @@ int launch_unique_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v8, c
                       cudaStream_t st)
 {
     const int n_slots = s->shared_slots + s->n_unique_splits;
-    const long long grid = (long long)s->B * s->Hkv * s->n_unique_splits;
+    const int q_len = s->q_len > 1 ? s->q_len : 1;
+    const long long grid = (long long)(s->B / q_len) * s->Hkv * s->n_unique_splits;
     if (grid == 0) return MOSKA_OK;
     if (grid > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "unique attention grid too large");
     MOSKA_CUDA_TRY(cudaFuncSetAttribute(unique_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         kF8RingBytes));
     unique_fp8_kernel<<<(unsigned)grid, kThreads, kF8RingBytes, st>>>(
         q, k8, v8, k_scale, v_scale, kv_start, kv_len, o_part, lse_part, scale, s->Hq, s->Hkv,
-        s->n_unique_splits, s->shared_slots, n_slots);
+        s->n_unique_splits, s->shared_slots, n_slots, q_len);
     MOSKA_LAUNCH_CHECK("unique_fp8_kernel");
     return MOSKA_OK;
 }

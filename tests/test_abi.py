@@ -77,7 +77,7 @@ def test_null_pointer_and_workspace_errors_come_before_any_launch(M):
     assert e.value.status in (M.ERR_INVALID_ARG, M.ERR_CUDA, M.ERR_UNSUPPORTED)
     # several query tokens per request: more than 16 rows per (request, KV head), D = 64 and the
     # FP8 store are refused before anything is launched
-    for kw, call in ((dict(Hq=64, q_len=4), "bf16"), (dict(D=64, q_len=2), "bf16"), (dict(q_len=2), "fp8")):
+    for kw, call in ((dict(Hq=64, q_len=4), "bf16"), (dict(D=64, q_len=2), "bf16"), (dict(q_len=4), "fp8")):
         base = dict(B=4, Hq=32, Hkv=8, D=128, C=128, L=512, k=8)
         base.update(kw)
         sq = M.shape(**base)

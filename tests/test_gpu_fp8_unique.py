@@ -99,3 +99,38 @@ def test_fp8kv_decode_step_one_and_two_streams():
     _step_case(w, two_streams=True, lengths=lens)
     # the share of SMs branch of the schedule (long unique attention announced by the hint)
     _step_case(w, two_streams=True, lengths=lens, unique_tokens=1 << 26)
+
+
+def test_fp8_unique_several_query_tokens_per_request():
+    """shape.q_len > 1 with the FP8 store: one pass over a request's codes for all its query tokens;
+    the oracle is given the same problem with every token as a request of its own."""
+    from paper_2511_06010_b200 import binding as M
+    from paper_2511_06010_b200.engine import MoskaLayer
+
+    lens_last = np.array([40, 1, 130, 77, 300, 16, 2, 0, 1000, 65, 3], dtype=np.int64)
+    base = len(lens_last)
+    for Hq, Hkv, t, splits in ((8, 2, 2, 1), (8, 2, 2, 3), (4, 2, 4, 2), (6, 2, 2, 2), (4, 4, 5, 1)):
+        w = W.Workload("fp8multi", B=base * t, Hq=Hq, Hkv=Hkv, D=128, C=4, L=128, k=2, unique_len=0, seed=11)
+        sh = W.make_shared_store(w, "cuda")
+        un = W.make_unique_store(W.scaled(w, B=base, steps=0), "cuda", lens_last)
+        f8 = W.quantize_unique_store_fp8(un)
+        q = W.make_queries(w, sh, 0, "cuda")
+        layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, int(lens_last.max()),
+                           n_unique_splits=splits, q_len=t, fp8_unique=True)
+        n_sh = layer.shape.shared_slots
+        layer.o_part.fill_(float("nan"))
+        layer.lse_part.fill_(float("nan"))
+        layer.unique_fp8(q, f8, un.kv_start, un.kv_len)
+        torch.cuda.synchronize()
+        o_un = layer.o_part[:, :, n_sh:].cpu().numpy()
+        l_un = layer.lse_part[:, :, n_sh:].cpu().numpy()
+        assert not np.isnan(l_un).any() and np.isfinite(o_un).all(), "a unique slot was left unwritten"
+        o_m, l_m = O.merge(o_un, l_un)
+        kv_start = un.kv_start.repeat_interleave(t).cpu().numpy()
+        back = np.tile(np.arange(t - 1, -1, -1), base)
+        kv_len = np.maximum(0, np.repeat(lens_last, t) - back).astype(np.int32)
+        ref_o, ref_l = O.attend_unique_fp8(q.cpu(), f8.k8.cpu(), f8.v8.cpu(), f8.k_scale.cpu(),
+                                           f8.v_scale.cpu(), kv_start, kv_len, layer.scale)
+        PU.check_lse(l_m, ref_l, f"fp8 q_len={t} lse")
+        PU.check_attention(o_m, ref_o, f"fp8 q_len={t} o")
+        assert M.device_status() == 0
