@@ -69,6 +69,7 @@ __device__ __forceinline__ float lds_f32(uint32_t addr)
 // Head dimension that lane group g holds as row g (half = 0) / row g + 8 (half = 1) of block mt.
 __device__ __forceinline__ int v8_dim_of(int g, int mt, int half) { return 16 * g + 2 * mt + half; }
 
+template <bool kMulti>  // several query tokens per request (q_len > 1)
 __global__ void __launch_bounds__(kThreads, 3)
 unique_fp8_kernel(const uint16_t* __restrict__ q, const uint8_t* __restrict__ k8,
                   const uint8_t* __restrict__ v8, const float* __restrict__ k_scale,
@@ -89,6 +90,7 @@ unique_fp8_kernel(const uint16_t* __restrict__ q, const uint8_t* __restrict__ k8
     // Query rows of this (request, KV head): row j = i * G + g' is head g' of query token i (one
     // token unless q_len > 1), a batch row of its own that sees the context up to q_len - 1 - i
     // tokens before its end.
+    if (!kMulti) q_len = 1;
     const int n_rows = q_len * G;
 
     // token range of this split (same rule as the bf16 kernel: equal parts rounded up to 64)
@@ -192,7 +194,7 @@ unique_fp8_kernel(const uint16_t* __restrict__ q, const uint8_t* __restrict__ k8
         const bool va = (t0 + g) <= last_tok, vb = (t0 + 8 + g) <= last_tok;
         if (!va) sc[0] = sc[1] = -INFINITY;
         if (!vb) sc[2] = sc[3] = -INFINITY;
-        if (t0 + kTileTokens - 1 > min_last) {  // q_len > 1: the tile reaches past some row's context
+        if (kMulti && t0 + kTileTokens - 1 > min_last) {  // the tile reaches past some row's context
             if (t0 + g > lim0) sc[0] = -INFINITY;
             if (t0 + g > lim1) sc[1] = -INFINITY;
             if (t0 + 8 + g > lim0) sc[2] = -INFINITY;
@@ -211,8 +213,8 @@ unique_fp8_kernel(const uint16_t* __restrict__ q, const uint8_t* __restrict__ k8
         m_run[1] = mn1;
         float ms0 = mn0 * sl2, ms1 = mn1 * sl2;
         // a row that has seen no token yet: keep its (empty) state free of inf - inf
-        if (mn0 == -INFINITY) { al0 = 1.f; ms0 = 0.f; }
-        if (mn1 == -INFINITY) { al1 = 1.f; ms1 = 0.f; }
+        if (kMulti && mn0 == -INFINITY) { al0 = 1.f; ms0 = 0.f; }
+        if (kMulti && mn1 == -INFINITY) { al1 = 1.f; ms1 = 0.f; }
         const float p0 = fast_exp2(fmaf(sc[0], sl2, -ms0)), p1 = fast_exp2(fmaf(sc[1], sl2, -ms1));
         const float p2 = fast_exp2(fmaf(sc[2], sl2, -ms0)), p3 = fast_exp2(fmaf(sc[3], sl2, -ms1));
         l_run[0] = fmaf(l_run[0], al0, p0 + p2);
@@ -305,11 +307,19 @@ int launch_unique_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v8, c
     const long long grid = (long long)(s->B / q_len) * s->Hkv * s->n_unique_splits;
     if (grid == 0) return MOSKA_OK;
     if (grid > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "unique attention grid too large");
-    MOSKA_CUDA_TRY(cudaFuncSetAttribute(unique_fp8_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                        kF8RingBytes));
-    unique_fp8_kernel<<<(unsigned)grid, kThreads, kF8RingBytes, st>>>(
-        q, k8, v8, k_scale, v_scale, kv_start, kv_len, o_part, lse_part, scale, s->Hq, s->Hkv,
-        s->n_unique_splits, s->shared_slots, n_slots, q_len);
+    if (q_len > 1) {
+        MOSKA_CUDA_TRY(cudaFuncSetAttribute(unique_fp8_kernel<true>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kF8RingBytes));
+        unique_fp8_kernel<true><<<(unsigned)grid, kThreads, kF8RingBytes, st>>>(
+            q, k8, v8, k_scale, v_scale, kv_start, kv_len, o_part, lse_part, scale, s->Hq, s->Hkv,
+            s->n_unique_splits, s->shared_slots, n_slots, q_len);
+    } else {
+        MOSKA_CUDA_TRY(cudaFuncSetAttribute(unique_fp8_kernel<false>,
+                                            cudaFuncAttributeMaxDynamicSharedMemorySize, kF8RingBytes));
+        unique_fp8_kernel<false><<<(unsigned)grid, kThreads, kF8RingBytes, st>>>(
+            q, k8, v8, k_scale, v_scale, kv_start, kv_len, o_part, lse_part, scale, s->Hq, s->Hkv,
+            s->n_unique_splits, s->shared_slots, n_slots, q_len);
+    }
     MOSKA_LAUNCH_CHECK("unique_fp8_kernel");
     return MOSKA_OK;
 }
