@@ -554,6 +554,7 @@ def main():
     ap.add_argument("--steps", type=int, default=500)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", type=int, default=1, help="workload index 0..4 (default 1)")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (sweeps)")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--one-stream", action="store_true", help="run unique attention on the main stream")
     ap.add_argument("--unique-splits", type=int, default=None, help="override the split-K count of unique attention")
@@ -568,6 +569,8 @@ def main():
     ap.add_argument("--ref-sample", type=int, default=8, help="requests per step of --impl reference")
     args = ap.parse_args()
     w = W.CONFIGS[args.config]
+    if args.batch:
+        w = W.scaled(w, name=f"{w.name}@B{args.batch}", B=args.batch)
     if args.impl == "reference":
         run_reference(args, w)
     else:
