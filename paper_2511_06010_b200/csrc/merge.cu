@@ -27,17 +27,32 @@ merge_kernel(const float* __restrict__ o_part, const float* __restrict__ lse_par
     float W = 0.f;
     const bool active = lane < D / 4;
     if (M != -INFINITY) {
-        const float* o = o_part + r * n_slots * D + lane * 4;
-        for (int i = 0; i < n_slots; ++i) {
-            const float w = __expf(lse[i] - M);  // warp-uniform
-            if (w == 0.f) continue;              // empty slots hold no meaningful o
-            W += w;
-            if (active) {
-                const float4 v = *reinterpret_cast<const float4*>(o + (long long)i * D);
-                acc.x = fmaf(w, v.x, acc.x);
-                acc.y = fmaf(w, v.y, acc.y);
-                acc.z = fmaf(w, v.z, acc.z);
-                acc.w = fmaf(w, v.w, acc.w);
+        const float* o = o_part + r * n_slots * D + (active ? lane * 4 : 0);
+        // Slots in groups of 32: lane i holds the weight of slot base + i; the partial rows are then
+        // read four slots at a time with all four loads in flight (a slot of weight 0 is read but
+        // not used: it holds no meaningful o).
+        for (int base = 0; base < n_slots; base += 32) {
+            const int mine = base + lane;
+            const float w_mine = mine < n_slots ? __expf(lse[mine] - M) : 0.f;
+            const int n = min(32, n_slots - base);
+            for (int i0 = 0; i0 < n; i0 += 4) {
+                float w[4];
+                float4 v[4];
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    w[j] = __shfl_sync(0xffffffffu, w_mine, (i0 + j) & 31);
+                    const int slot = min(base + i0 + j, n_slots - 1);
+                    v[j] = *reinterpret_cast<const float4*>(o + (long long)slot * D);
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    if (i0 + j >= n || w[j] == 0.f) continue;
+                    W += w[j];
+                    acc.x = fmaf(w[j], v[j].x, acc.x);
+                    acc.y = fmaf(w[j], v[j].y, acc.y);
+                    acc.z = fmaf(w[j], v[j].z, acc.z);
+                    acc.w = fmaf(w[j], v[j].w, acc.w);
+                }
             }
         }
         const float inv = 1.f / W;
