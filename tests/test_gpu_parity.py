@@ -428,6 +428,44 @@ def test_host_buffer_step_equals_device_step():
     assert M.device_status() == 0
 
 
+def test_shared_and_unique_roles_compose_to_the_single_gpu_step():
+    """The two roles of the disaggregated step, run one after the other on one GPU with the exchange
+    replaced by direct hand-over: the shared role's result, merged over the routed chunks, placed in
+    slot 0 of the unique role's partials and merged with its split-K partials equals the oracle's
+    direct attention (and the single-GPU step within the output's rounding)."""
+    M, MoskaLayer = _mods()
+    from paper_2511_06010_b200 import disaggregated as DG
+
+    lens = np.array([300, 1, 0, 1000, 64, 17, 129, 511, 700, 77, 5, 900], dtype=np.int64)
+    w = W.scaled(W.CONFIGS[1], B=len(lens), C=16, k=4, unique_len=0)
+    sh = W.make_shared_store(w, "cuda")
+    un = W.make_unique_store(w, "cuda", lens)
+    q = W.make_queries(w, sh, 0, "cuda")
+    shared_layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, 1, n_unique_splits=1)
+    shared_role = DG.SharedRank(shared_layer, sh.k_shared, sh.v_shared)
+    o_s, lse_s = shared_role.compute(q)
+    outs = []
+    for rank, b0, b1 in DG.request_blocks(w.B, [1, 2]):
+        # every unique rank: its own requests, its own slice of the private store
+        t0 = int(un.kv_start[b0].item())
+        layer = MoskaLayer(b1 - b0, w.Hq, w.Hkv, w.D, 1, w.L, 1, int(lens.max()), n_unique_splits=2)
+        role = DG.UniqueRank(layer, un.k_unique[t0:], un.v_unique[t0:], (un.kv_start[b0:b1] - t0).contiguous())
+        role.start(q[b0:b1].contiguous(), un.kv_len[b0:b1].contiguous())
+        outs.append(role.finish(o_s[b0:b1], lse_s[b0:b1]).clone())
+    out = torch.cat(outs)
+    torch.cuda.synchronize()
+    ref, _ = O.attend_direct(q.cpu(), sh.k_shared.cpu(), sh.v_shared.cpu(), un.k_unique.cpu(),
+                             un.v_unique.cpu(), un.kv_start.cpu().numpy(), un.kv_len.cpu().numpy(),
+                             shared_layer.topk_idx.cpu().numpy(), shared_layer.scale)
+    PU.check_attention(out.float().cpu().numpy(), ref, "two roles composed")
+    single = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, int(lens.max()), n_unique_splits=2)
+    single.build_summaries(sh.k_shared)
+    one = single.step(q, sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, un.kv_start, un.kv_len)
+    torch.cuda.synchronize()
+    assert (out.float() - one.float()).abs().max().item() <= 2 ** -7 * max(1.0, one.float().abs().max().item())
+    assert M.device_status() == 0
+
+
 def test_decode_step_can_be_captured_in_a_cuda_graph():
     """Nothing in the step reads device results back on the host, so the whole two-stream step
     (fork and join included) is one CUDA graph; replaying it gives the eager result bit for bit."""
