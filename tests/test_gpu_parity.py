@@ -466,6 +466,17 @@ def test_shared_and_unique_roles_compose_to_the_single_gpu_step():
     assert M.device_status() == 0
 
 
+def test_group_sizes_that_do_not_divide_the_tiles():
+    """G = 3, 5, 6, 7: query tiles of 128 rows hold floor(128 / G) requests, streaming tiles
+    floor(16 / G) or floor(8 / G); large and small segments, routed and dense."""
+    lens = np.array([0, 1, 100, 257, 64, 33, 700, 15], dtype=np.int64)
+    for G in (3, 5, 6, 7):
+        # few chunks and many requests: segments of every size up to B requests
+        w = W.Workload(f"g{G}", B=56, Hq=2 * G, Hkv=2, D=128, C=6, L=256, k=2, unique_len=0, seed=G)
+        run_case(w, lengths=np.resize(lens, w.B), n_unique_splits=2)
+        run_case(W.scaled(w, B=40, C=3, k=3), lengths=np.resize(lens, 40), dense_slots=2, two_streams=True)
+
+
 def test_decode_step_can_be_captured_in_a_cuda_graph():
     """Nothing in the step reads device results back on the host, so the whole two-stream step
     (fork and join included) is one CUDA graph; replaying it gives the eager result bit for bit."""
