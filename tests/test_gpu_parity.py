@@ -295,6 +295,16 @@ def test_dense_tensor_core_tiles_and_empty_runs():
     run_case(W.scaled(base, B=70, Hq=16, C=3, k=3, L=512), n_unique_splits=2, dense_slots=1)
 
 
+def test_chunk_lengths_of_one_three_and_five_kv_tiles():
+    """L = 128, 384, 640: items of a single K/V tile (no split between the two slots), odd numbers
+    of tiles (the slots of a split item get unequal shares), routed and dense."""
+    for L in (128, 384, 640):
+        w = W.Workload(f"L{L}", B=80, Hq=8, Hkv=2, D=128, C=5, L=L, k=2, unique_len=40, seed=L)
+        run_case(w, n_unique_splits=1)                       # segments of up to 320 rows
+        run_case(W.scaled(w, B=12), n_unique_splits=1)       # only small segments
+        run_case(W.scaled(w, B=24, C=3, k=3), n_unique_splits=1, dense_slots=2)
+
+
 def _sample(w, n):
     return np.sort(np.random.default_rng(7).choice(w.B, size=min(n, w.B), replace=False))
 
