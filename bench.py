@@ -495,6 +495,8 @@ def run_cuda(args, w):
                "sample": f"first {n_s} of {w.B} requests (all heads, full context), {reps} repeats, "
                          f"{dt * reps:.1f} s"}
 
+    # the merge reads every partial once more and writes the bf16 result
+    rows_merge_bytes = w.B * w.Hq * ((S.shared_slots + S.n_unique_splits) * (w.D + 1) * 4 + w.D * 2)
     # kernels of one step: route (scoring + selection beyond 256 chunks), 2-3 grouping passes, unique,
     # shared (tensor-core items, 16-row tiles, 8-row tiles), merge
     n_launch = 3 if w.dense else (1 + (w.C > 256)) + (3 if w.B > 64 else 2) + 1 + (3 if w.D == 128 else 2) + 1
@@ -535,6 +537,13 @@ def run_cuda(args, w):
                    "amortisation_factor": P / max(1, touched)},
         "unique": {"gbs": unique_gbs, "frac_of_measured_hbm": (unique_gbs or 0) / peaks["hbm_gbs"],
                    "frac_of_nominal_8000": (unique_gbs or 0) / 8000.0},
+        # all HBM-bound work of the step against the step time: the two streams share the bandwidth,
+        # so a kernel's own in-step rate (roofline.achieved) understates how busy HBM is
+        "step_hbm": {
+            "bytes": work["unique_bytes"] + work["shared_bytes"] + rows_merge_bytes,
+            "gbs": (work["unique_bytes"] + work["shared_bytes"] + rows_merge_bytes) / (ms_per_step * 1e-3) / 1e9,
+            "frac_of_measured_hbm": (work["unique_bytes"] + work["shared_bytes"] + rows_merge_bytes)
+                                    / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"]},
         "gemv_baseline": None if gemv_ms is None else {
             "ms": gemv_ms,
             # both kernels alone on the GPU (in the step part of shared attention overlaps unique)
