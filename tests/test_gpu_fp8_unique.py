@@ -59,6 +59,15 @@ def test_fp8_unique_full_cfg1_sampled():
     _run(w, sample=np.sort(np.random.default_rng(7).choice(w.B, size=6, replace=False)))
 
 
+def test_fp8_unique_full_cfg2_sampled_with_the_default_splits():
+    """Workload 2 at full size (2 M private tokens), the split count the bench uses for FP8."""
+    from paper_2511_06010_b200 import binding as M
+
+    w = W.CONFIGS[2]
+    splits = M.default_unique_splits_fp8(w.B, w.Hkv, w.unique_len)
+    _run(w, n_unique_splits=splits, sample=np.sort(np.random.default_rng(9).choice(w.B, size=3, replace=False)))
+
+
 def _step_case(w, two_streams, lengths=None, unique_tokens=0):
     """The whole decode step with an FP8 private store against the oracle's shared partials
     (bf16 store) and FP8 unique partial, combined by the oracle's merge."""
