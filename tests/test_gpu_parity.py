@@ -487,6 +487,35 @@ def test_group_sizes_that_do_not_divide_the_tiles():
         run_case(W.scaled(w, B=40, C=3, k=3), lengths=np.resize(lens, 40), dense_slots=2, two_streams=True)
 
 
+def test_several_query_tokens_full_cfg1_sampled():
+    """Workload 1 with four query tokens per request (256 batch rows, the configuration
+    `bench.py --q-len 4` times), two-stream step, sampled rows against the direct definition."""
+    import types
+
+    M, MoskaLayer = _mods()
+    t = 4
+    w0 = W.CONFIGS[1]
+    w = W.scaled(w0, B=w0.B * t)
+    sh = W.make_shared_store(w, "cuda")
+    un = W.make_unique_store(w0, "cuda")
+    q = W.make_queries(w, sh, 0, "cuda")
+    layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, w0.unique_len, q_len=t)
+    layer.build_summaries(sh.k_shared)
+    out = layer.step(q, sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, un.kv_start, un.kv_len,
+                     two_streams=True, unique_tokens=int(un.kv_len.sum().item()))
+    torch.cuda.synchronize()
+    rows = np.sort(np.random.default_rng(3).choice(w.B, size=6, replace=False))
+    back = torch.arange(t - 1, -1, -1, device="cuda", dtype=torch.int32).repeat(w0.B)
+    expanded = types.SimpleNamespace(k_unique=un.k_unique, v_unique=un.v_unique,
+                                     kv_start=un.kv_start.repeat_interleave(t))
+    kv_len_rows = (un.kv_len.repeat_interleave(t) - back).to(torch.int32)
+    q_s, topk_s, ks, vs, ku, vu, st_s, len_s = _subproblem(q, layer.topk_idx, sh, expanded, kv_len_rows, rows)
+    ref, ref_lse = O.attend_direct(q_s, ks, vs, ku, vu, st_s, len_s, topk_s, layer.scale)
+    PU.check_attention(out[rows].float().cpu().numpy(), ref, "q_len = 4, workload 1")
+    PU.check_lse(layer.lse_out[rows].cpu().numpy(), ref_lse, "q_len = 4, workload 1, lse")
+    assert M.device_status() == 0
+
+
 def test_decode_step_can_be_captured_in_a_cuda_graph():
     """Nothing in the step reads device results back on the host, so the whole two-stream step
     (fork and join included) is one CUDA graph; replaying it gives the eager result bit for bit."""
