@@ -232,6 +232,28 @@ def decode_step_host(q_host, q_dev, summaries, k_shared, v_shared, k_unique, v_u
         None if side_stream is None else _stream(side_stream), prof), "moska_decode_step_host")
 
 
+def bind_decode_step_host(q_host, q_dev, summaries, k_shared, v_shared, k_unique, v_unique, kv_start,
+                          kv_len, topk_idx, seg_offsets, seg_entries, o_part, lse_part, out_dev,
+                          out_host, softmax_scale, s, ws, stream=None, side_stream=None, prof=None):
+    """decode_step_host with its arguments marshalled once: returns a callable for a serving loop
+    that repeats the call on the same buffers (the tensors must stay alive and in place; the shape
+    struct is passed by reference, so later changes of its fields are seen)."""
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    args = (_ptr(q_host), _ptr(q_dev), _ptr(summaries), _ptr(k_shared), _ptr(v_shared),
+            _ptr(k_unique), _ptr(v_unique), _ptr(kv_start), _ptr(kv_len), _ptr(topk_idx),
+            _ptr(seg_offsets), _ptr(seg_entries), _ptr(o_part), _ptr(lse_part), _ptr(out_dev),
+            _ptr(out_host), softmax_scale, ctypes.byref(s), _ptr(ws), ws_bytes, _stream(stream),
+            None if side_stream is None else _stream(side_stream), prof)
+    fn = _lib.moska_decode_step_host
+
+    def call() -> None:
+        status = fn(*args)
+        if status != OK:
+            raise MoskaError(status, "moska_decode_step_host")
+
+    return call
+
+
 STAGES = ("route", "group", "shared", "unique", "merge")
 
 

@@ -108,6 +108,20 @@ class MoskaLayer:
                             self.side_stream if two_streams else None, prof)
         return self.out
 
+    def bind_step_host(self, q_host, q_dev, out_host, k_shared, v_shared, k_unique, v_unique,
+                       kv_start, kv_len, two_streams=False, unique_tokens=0):
+        """step_host for a loop over fixed buffers: marshals the arguments once and returns a
+        callable that only makes the C call (no per-call Python work between two steps)."""
+        self.shape.unique_tokens = int(unique_tokens)
+        two_streams = two_streams and self.overlap_routing
+        if two_streams and self.side_stream is None:
+            self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
+        return M.bind_decode_step_host(q_host, q_dev, None if self.dense else self.summaries, k_shared,
+                                       v_shared, k_unique, v_unique, kv_start, kv_len, self.topk_idx,
+                                       self.seg_offsets, self.seg_entries, self.o_part, self.lse_part,
+                                       self.out, out_host, self.scale, self.shape, self.ws, None,
+                                       self.side_stream if two_streams else None)
+
     def step_host(self, q_host, q_dev, out_host, k_shared, v_shared, k_unique, v_unique,
                   kv_start, kv_len, two_streams=False, prof=None, unique_tokens=0):
         self.shape.unique_tokens = int(unique_tokens)

@@ -435,6 +435,13 @@ def test_host_buffer_step_equals_device_step():
         layer.step_host(q_host, q_dev, out_host, sh.k_shared, sh.v_shared, un.k_unique, un.v_unique,
                         un.kv_start, un.kv_len, two_streams=two)
         assert torch.equal(out_host, ref.cpu()), f"pinned={pinned} two_streams={two}"
+    # the same call with its arguments marshalled once, repeated on the same buffers
+    call = layer.bind_step_host(q_host, q_dev, out_host, sh.k_shared, sh.v_shared, un.k_unique,
+                                un.v_unique, un.kv_start, un.kv_len, two_streams=True)
+    for _ in range(3):
+        out_host.zero_()
+        call()
+        assert torch.equal(out_host, ref.cpu())
     assert M.device_status() == 0
 
 
