@@ -5,8 +5,18 @@
 
 One step = one decode step of one attention layer over one batch of synthetic requests:
 route -> group -> shared attention || unique attention -> merge, through the C ABI.  Prints ONE
-JSON line (rank 0).  With N > 1 (torchrun) every rank runs the same workload on its own batch of
-requests against its own copy of the shared store (no data-path collective; weak scaling).
+JSON line (rank 0).
+
+Without --config the headline is the largest workload (index 4: serving mix, batch 1024, 8
+re-routed decode steps) and the same line carries a `per_config` record for workloads 1, 2 and 3,
+each timed on blocks of its own.  The timed region is R blocks of K steps (R chosen so that the
+blocks add up to at least half a second of device time); `ms_per_step` is the median block / K.
+
+With N > 1 (torchrun) ONE batch is split by KV head: every rank holds Hkv / N heads of the shared
+store and of every request's private store and computes those heads' outputs, no data-path
+collective (strong scaling).  `--shard replicas` gives every rank its own batch and its own copy
+of the shared store instead (weak scaling); `--shard disaggregated` runs rank 0 as the Shared-KV
+rank and the others as Unique-KV ranks with one point-to-point exchange each way per step.
 
 `--impl reference` times the fp64 CPU oracle on the host cores instead (bounded sample per step).
 """
@@ -14,6 +24,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -34,9 +45,13 @@ from paper_2511_06010_b200 import workloads as W
 METRIC = "decode_queries_per_s_per_layer"
 UNIT = "queries/s"
 L2_BYTES = 126e6
+HEADLINE_CONFIG = 4            # the largest single-GPU workload
+PER_CONFIG = (1, 2, 3)         # further workloads recorded on the same line
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from ncu captures of the same kernels
-# (summaries under profiles/).  Keyed by (kernel, workload name).
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from ncu captures (summaries under
+# profiles/).  Keyed by (kernel, workload name); "ratio" entries are traffic / algorithmic bytes
+# measured on a smaller launch of the same kernel and scaled by the units a full launch processes
+# (the traffic of these streaming kernels grows in proportion to the tokens they read).
 NCU_TRAFFIC_BYTES = {
     # profiles/unique_staged_kernel_cfg1.md: 1.0744 GB read + 7.3 MB written
     ("unique_staged_kernel", "cfg1_llama8b_b64"): 1.0817e9,
@@ -44,6 +59,10 @@ NCU_TRAFFIC_BYTES = {
     ("unique_fp8_kernel", "cfg1_llama8b_b64"): 5.615e8,
     # profiles/shared_tc_kernel_cfg3.md: 559.2 MB read + 139.8 MB written
     ("shared_tc_kernel", "cfg3_dense_b512"): 6.995e8,
+}
+NCU_TRAFFIC_RATIO = {
+    # unique_staged_kernel: 1.0817 GB measured for 1.0785 GB algorithmic on workload 1
+    "unique_staged_kernel": (1.0817e9 / 1.0785e9, "scaled from the workload-1 capture by bytes"),
 }
 
 
@@ -152,7 +171,8 @@ class ClockSampler:
                 self.proc.kill()
         sm = [r[0] for r in self.rows]
         reasons = set().union(*[r[1] for r in self.rows]) if self.rows else set()
-        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": self.sm_max,
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_mhz_min": min(sm) if sm else None, "sm_max_mhz": self.sm_max,
                 "samples": len(sm), "source": self.source, "reasons": sorted(reasons)}
 
 
@@ -238,27 +258,77 @@ def run_reference(args, w):
     print(json.dumps(line), flush=True)
 
 
-def run_cuda(args, w):
-    rank, local_rank, world = DD.init("nccl")
-    torch.cuda.set_device(local_rank)
-    dev = torch.device("cuda", local_rank)
-    from paper_2511_06010_b200 import build as B
+def timed_blocks(run_block, min_total_ms: float, dev, max_blocks: int = 200, min_blocks: int = 3):
+    """Runs run_block() -> milliseconds (device-timed, this rank) repeatedly: the first block fixes
+    the number of blocks R (same on every rank: derived from the slowest rank's first block) so
+    that the blocks add up to min_total_ms; returns the per-block maxima over ranks."""
+    first = DD.max_over_ranks(run_block(), dev)
+    n = int(min(max_blocks, max(min_blocks, math.ceil(min_total_ms / max(first, 1e-3)))))
+    blocks = [first]
+    for _ in range(n - 1):
+        blocks.append(DD.max_over_ranks(run_block(), dev))
+    return blocks
 
-    if rank == 0:
-        B.build()
-    DD.barrier()
+
+def cpu_baseline(w, sh, un, q0, kv_len0, n_sample: int, seconds: float):
+    """The oracle as it stands on the host cores: a bounded sample of the workload's requests
+    (all heads, full context), repeated for about `seconds`."""
+    from oracle import oracle as O
+
+    O.build()
+    n_s = min(w.B, n_sample)
+    sample = np.arange(n_s)
+    qh = q0.cpu()
+    lens_s = kv_len0.cpu().numpy()
+    end = int((un.kv_start[n_s - 1] + un.capacity[n_s - 1]).item())
+    un_host = (un.k_unique[:end].cpu(), un.v_unique[:end].cpu(), un.kv_start.cpu().numpy())
+    sh_host = (sh.k_shared.cpu(), sh.v_shared.cpu())
+    summ = None if w.dense else O.chunk_summaries(sh_host[0])
+    t0 = time.perf_counter()
+    reps = 0
+    while True:
+        cpu_oracle_step(w, sh_host, un_host, qh, lens_s, summ, sample)
+        reps += 1
+        if time.perf_counter() - t0 > seconds or reps >= 500:
+            break
+    dt = (time.perf_counter() - t0) / reps
+    return {"value": n_s / dt, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
+            "sample": f"first {n_s} of {w.B} requests (all heads, full context), {reps} repeats, "
+                      f"{dt * reps:.1f} s"}
+
+
+def measure(args, w_full, rank, world, dev, headline: bool):
+    """Everything measured on one workload; returns the record (rank 0) or None."""
     from paper_2511_06010_b200 import binding as M
     from paper_2511_06010_b200.engine import MoskaLayer
 
-    # every rank: its own request batch (seed offset), its own copy of the shared store
-    wr = W.scaled(w, seed=w.seed + 7919 * rank) if world > 1 else w
+    local_rank = dev.index
+    # ---- what this rank holds
+    if world > 1 and args.shard == "kv_head":
+        if w_full.Hkv % world != 0:
+            raise SystemExit(f"{w_full.name}: {w_full.Hkv} KV heads do not split over {world} ranks "
+                             "(use --shard replicas)")
+        w = W.kv_head_shard(w_full, rank, world)
+        per_gpu = f"KV heads [{rank * w.Hkv}, {(rank + 1) * w.Hkv}) of one batch: 1/{world} of the shared and private stores"
+        units_this_rank = w.B / world      # every request is served by all ranks together
+        scaling = "strong"
+    elif world > 1:
+        w = W.scaled(w_full, seed=w_full.seed + 7919 * rank)
+        per_gpu = "own request batch, own copy of the shared store"
+        units_this_rank = w.B
+        scaling = "weak"
+    else:
+        w = w_full
+        per_gpu = "single GPU"
+        units_this_rank = w.B
+        scaling = "weak"
     free, _ = torch.cuda.mem_get_info()
-    lens0 = W.unique_lengths(wr)
+    lens0 = W.unique_lengths(w)
     need = (2 * w.Hkv * w.C * w.L * w.D + 2 * int((lens0 + w.steps).sum()) * w.Hkv * w.D) * 2
     if need * 1.15 > free:
         raise SystemExit(f"workload {w.name} needs {need/1e9:.1f} GB, only {free/1e9:.1f} GB free")
-    sh = W.make_shared_store(wr, dev)
-    un = W.make_unique_store(wr, dev)
+    sh = W.make_shared_store(w, dev)
+    un = W.make_unique_store(w, dev)
     # --q-len T: every request brings T query tokens (speculative decoding); the batch rows are
     # requests x T, token i of a request sees its context up to T - 1 - i tokens from the end
     T = max(1, args.q_len)
@@ -266,7 +336,7 @@ def run_cuda(args, w):
         if w.D != 128 or T * w.G > (8 if args.unique_kv == "fp8" else 16):
             raise SystemExit("--q-len needs head dimension 128 and q_len * G <= 16 (8 with --unique-kv fp8)")
         w = W.scaled(w, B=w.B * T)
-        wr = W.scaled(wr, B=wr.B * T)
+        units_this_rank *= T
     fp8 = args.unique_kv == "fp8"
     f8 = None
     if fp8:
@@ -276,7 +346,7 @@ def run_cuda(args, w):
         f8 = W.quantize_unique_store_fp8(un, release=True)
         torch.cuda.empty_cache()
     n_q = max(1, w.steps)
-    qs = [W.make_queries(wr, sh, s, dev) for s in range(n_q)]
+    qs = [W.make_queries(w, sh, s, dev) for s in range(n_q)]
     kv_lens = [(un.kv_len + s).to(torch.int32) for s in range(n_q)]
     max_len = int(lens0.max()) + w.steps
     layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, max_len, dense=w.dense,
@@ -331,21 +401,24 @@ def run_cuda(args, w):
         else:
             layer.unique(qs[0], un.k_unique, un.v_unique, un.kv_start, kv_lens[0])
 
-    for i in range(max(3, args.warmup)):
+    K = args.steps
+    n_warm = max(3, args.warmup)
+    for i in range(n_warm):
         step(i)
     torch.cuda.synchronize()
 
     # Per-stage device times of every stage from a short untimed pass (two event records per stage
-    # and step cost about 3 us each, 6 % of a step of the default workload); in the timed region only
-    # the dominant kernel's stage is recorded, for the roofline.
-    prof = M.profiler_create(max(args.steps, 32))
-    n_pre = min(32, max(8, args.steps))
+    # and step cost about 3 us each); in the timed region only the dominant kernel's stage is
+    # recorded, for the roofline.
+    n_pre = min(16, max(8, K))
+    prof_pre = M.profiler_create(n_pre)
     for i in range(n_pre):
         if flush is not None:
             flush()
-        step(i, prof)
+        step(i, prof_pre)
     torch.cuda.synchronize()
-    stage_ms_pre, n_rec = M.profiler_read(prof)
+    stage_ms_pre, n_rec = M.profiler_read(prof_pre)
+    M.profiler_destroy(prof_pre)
     stage_ms_pre = {k: v / max(1, n_rec) for k, v in stage_ms_pre.items()}
     # The dominant kernel is the one with the longest roofline time for its algorithmic work (the
     # in-step durations do not say: a kernel that shares the SMs with another one is stretched).
@@ -363,39 +436,48 @@ def run_cuda(args, w):
     t_bytes = work["shared_bytes"] / (peaks["hbm_gbs"] * 1e9)
     t_unique = work["unique_bytes"] / (peaks["hbm_gbs"] * 1e9)
     dominant = "unique" if t_unique >= max(t_flops, t_bytes) else "shared"
+
+    # ---- the timed region: R blocks of K steps, barrier + synchronize on both sides of a block
+    prof = M.profiler_create(K)
     M.profiler_select(prof, [dominant])
-    sampler = ClockSampler(local_rank)
-    DD.barrier()
-    torch.cuda.synchronize()
-    sampler.start()
-    if flush is None:
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for i in range(args.steps):
-            step(i, prof)
-        e1.record()
+    dom_ms = []
+
+    def run_block():
+        DD.barrier()
         torch.cuda.synchronize()
-        total_ms = e0.elapsed_time(e1)
-    else:
-        total_ms = 0.0
-        for i in range(args.steps):
-            flush()
+        if flush is None:
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            step(i, prof)
+            for i in range(K):
+                step(i, prof)
             e1.record()
-            e1.synchronize()
-            total_ms += e0.elapsed_time(e1)
-    DD.barrier()
-    torch.cuda.synchronize()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1)
+        else:
+            ms = 0.0
+            for i in range(K):
+                flush()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                step(i, prof)
+                e1.record()
+                e1.synchronize()
+                ms += e0.elapsed_time(e1)
+        DD.barrier()
+        t, n = M.profiler_read(prof)
+        dom_ms.append(t[dominant] / max(1, n))
+        return ms
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    blocks = timed_blocks(run_block, args.min_timed_ms if headline else args.min_timed_ms / 2, dev)
     clocks = sampler.stop()
-    timed_ms, n_rec = M.profiler_read(prof)
     M.profiler_destroy(prof)
+    block_ms = statistics.median(blocks)
+    ms_per_step = block_ms / K
+    value = DD.sum_over_ranks(units_this_rank * K, dev) / (block_ms * 1e-3)
     stage_ms = dict(stage_ms_pre)
-    stage_ms[dominant] = timed_ms[dominant] / max(1, n_rec)  # from the timed region itself
-    ms_per_step = total_ms / args.steps
-    value, ms_max = DD.whole_job_throughput(w.B * args.steps, total_ms, dev)
-    ms_per_step_max = ms_max / args.steps
+    stage_ms[dominant] = statistics.median(dom_ms)  # from the timed region itself
 
     # ---- end to end through the host-buffer entry point (pinned q in, out back, every step)
     q_host = [q.cpu().pin_memory() for q in qs]
@@ -403,27 +485,39 @@ def run_cuda(args, w):
     q_dev = torch.empty_like(qs[0])
     for i in range(3):
         step_host(i)
-    DD.barrier()
-    torch.cuda.synchronize()
-    t0 = time.perf_counter()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(args.steps):
-        if flush is not None:
+
+    def run_block_host():
+        DD.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        if flush is None:
+            e0.record()
+            for i in range(K):
+                step_host(i)
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1)
+        ms = 0.0
+        for i in range(K):
             flush()
-        step_host(i)
-    e1.record()
-    torch.cuda.synchronize()
-    e2e_ms = e0.elapsed_time(e1)
-    e2e_value, _ = DD.whole_job_throughput(w.B * args.steps, e2e_ms, dev)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            step_host(i)
+            e1.record()
+            e1.synchronize()
+            ms += e0.elapsed_time(e1)
+        return ms
+
+    e2e_blocks = timed_blocks(run_block_host, args.min_timed_ms / 2 if headline else args.min_timed_ms / 4, dev)
+    e2e_block_ms = statistics.median(e2e_blocks)
+    e2e_value = DD.sum_over_ranks(units_this_rank * K, dev) / (e2e_block_ms * 1e-3)
     io_bytes = w.B * w.Hq * w.D * 2
 
     if rank != 0:
-        DD.finalize()
-        return
+        return None
 
     # ---- per-kernel detail (rank 0, outside the timed region)
-    iters = max(3, min(args.steps, 10))
+    iters = max(3, min(K, 10))
     gemv_ms = None
     if not args.no_baseline:
         big = w.dense and w.B * w.C > 20000   # 256 GiB of re-reads in the dense config: sample it
@@ -465,57 +559,53 @@ def run_cuda(args, w):
         if T > 1 and not fp8:
             kernel = "unique_multi_kernel"
         roof = dict(bound="hbm", achieved=unique_gbs, peak=peaks["hbm_gbs"], unit="GB/s")
+        algo = work["unique_bytes"]
     elif t_flops > t_bytes:
         kernel = "shared_tc_kernel"
         roof = dict(bound="tensor", achieved=shared_tflops, peak=peaks["bf16_tflops_sustained"],
                     unit="TFLOP/s")
+        algo = None
     else:
-        kernel = "shared_tc_kernel+shared_small_kernel" if w.D == 128 else "shared_small_kernel"
+        kernel = "shared_tc_kernel" if w.D == 128 else "shared_small_kernel"
         roof = dict(bound="hbm", achieved=shared_gbs, peak=peaks["hbm_gbs"], unit="GB/s")
+        algo = work["shared_bytes"]
     roof["frac"] = roof["achieved"] / roof["peak"] if roof["achieved"] else None
     roof["traffic"] = NCU_TRAFFIC_BYTES.get((kernel, w.name))
+    if roof["traffic"] is None and kernel in NCU_TRAFFIC_RATIO and algo is not None:
+        ratio, how = NCU_TRAFFIC_RATIO[kernel]
+        roof["traffic"] = ratio * algo
+        roof["traffic_source"] = how
     roof["kernel"] = kernel
     roof["peak_source"] = "of " + peaks["source"]
     roof["avg_launch_ms"] = unique_ms if kernel.startswith("unique") else shared_ms
+    roof["alone"] = {
+        "avg_launch_ms": iso["unique"] if kernel.startswith("unique") else iso["shared"],
+        "frac": ((work["unique_bytes"] / (iso["unique"] * 1e-3) / 1e9 / peaks["hbm_gbs"])
+                 if kernel.startswith("unique") else
+                 (work["shared_flops"] / (iso["shared"] * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"])
+                 if roof["bound"] == "tensor" else
+                 (work["shared_bytes"] / (iso["shared"] * 1e-3) / 1e9 / peaks["hbm_gbs"]))}
 
     # ---- CPU baseline: the oracle as it stands on the host cores, bounded sample (N = 1 only)
     cpu = None
     if world == 1 and not args.no_cpu_baseline and not fp8 and T == 1:
-        from oracle import oracle as O
-
-        O.build()
-        n_s = min(w.B, args.cpu_sample)
-        sample = np.arange(n_s)
-        qh = qs[0].cpu()
-        lens_s = kv_lens[0].cpu().numpy()
-        end = int((un.kv_start[n_s - 1] + un.capacity[n_s - 1]).item())
-        un_host = (un.k_unique[:end].cpu(), un.v_unique[:end].cpu(), un.kv_start.cpu().numpy())
-        sh_host = (sh.k_shared.cpu(), sh.v_shared.cpu())
-        summ = None if w.dense else O.chunk_summaries(sh_host[0])
-        t0 = time.perf_counter()
-        reps = 0
-        while True:
-            cpu_oracle_step(w, sh_host, un_host, qh, lens_s, summ, sample)
-            reps += 1
-            if time.perf_counter() - t0 > args.cpu_seconds or reps >= 500:
-                break
-        dt = (time.perf_counter() - t0) / reps
-        cpu = {"value": n_s / dt, "unit": UNIT, "cores": O.num_threads(), "kind": "oracle",
-               "sample": f"first {n_s} of {w.B} requests (all heads, full context), {reps} repeats, "
-                         f"{dt * reps:.1f} s"}
+        cpu = cpu_baseline(w, sh, un, qs[0], kv_lens[0], args.cpu_sample,
+                           args.cpu_seconds if headline else args.cpu_seconds / 2)
 
     # the merge reads every partial once more and writes the bf16 result
     rows_merge_bytes = w.B * w.Hq * ((S.shared_slots + S.n_unique_splits) * (w.D + 1) * 4 + w.D * 2)
     # kernels of one step: route (scoring + selection beyond 256 chunks), 2-3 grouping passes, unique,
-    # shared (tensor-core items, 16-row tiles, 8-row tiles), merge
-    n_launch = 3 if w.dense else (1 + (w.C > 256)) + (3 if w.B > 64 else 2) + 1 + (3 if w.D == 128 else 2) + 1
-    n_launch *= args.steps
-    line = {
-        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step_max, "higher_is_better": True,
-        "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+    # shared, merge
+    n_shared_launches = 3 if (w.D == 128) else 2   # tensor-core items, 16-row tiles, 8-row tiles
+    n_launch = 3 if w.dense else (1 + (w.C > 256)) + (3 if w.B > 64 else 2) + 1 + n_shared_launches + 1
+    hbm_bytes = work["unique_bytes"] + work["shared_bytes"] + rows_merge_bytes
+    amort = P / max(1, touched)
+    rec = {
+        "workload": w_full.name, "value": value, "ms_per_step": ms_per_step, "steps_per_block": K,
+        "blocks": len(blocks), "block_ms": {"median": block_ms, "min": min(blocks), "max": max(blocks)},
+        "timed_ms_total": sum(blocks), "scaling": scaling,
         "config": {
-            "workload": w.name, "batch": w.B, "q_heads": w.Hq, "kv_heads": w.Hkv, "head_dim": w.D,
+            "workload": w_full.name, "batch": w.B, "q_heads": w.Hq, "kv_heads": w.Hkv, "head_dim": w.D,
             "shared_tokens": w.C * w.L, "chunk_tokens": w.L, "top_k": None if w.dense else w.k,
             "unique_tokens_mean": float(lens.mean()), "n_unique_splits": S.n_unique_splits,
             "shared_slots": S.shared_slots, "streams": 2 if two_streams else 1,
@@ -523,12 +613,15 @@ def run_cuda(args, w):
             "q_len": T, "requests": w.B // T,
             "l2": ("flushed between steps" if flush is not None
                    else f"inputs exceed L2 ({input_bytes / 2**20:.0f} MiB of K/V per step)"),
-            "per_gpu": "own request batch, own copy of the shared store" if world > 1 else "single GPU",
+            "per_gpu": per_gpu,
+            "timed_region": f"{len(blocks)} blocks of {K} steps, median block",
         },
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": io_bytes,
-                "d2h_bytes_per_step": io_bytes, "ms_per_step": e2e_ms / args.steps},
-        "gpu_launches": n_launch,
+                "d2h_bytes_per_step": io_bytes, "ms_per_step": e2e_block_ms / K,
+                "blocks": len(e2e_blocks)},
+        "gpu_launches": n_launch * K * len(blocks),
+        "gpu_launches_per_step": n_launch,
         "roofline": roof,
         "cpu_baseline": cpu,
         "stage_ms": stage_ms,
@@ -537,43 +630,170 @@ def run_cuda(args, w):
             "unique_gbs": work["unique_bytes"] / (iso["unique"] * 1e-3) / 1e9,
             "unique_frac_of_measured_hbm": work["unique_bytes"] / (iso["unique"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
             "shared_tflops": work["shared_flops"] / (iso["shared"] * 1e-3) / 1e12,
+            "shared_frac_of_measured_sustained": work["shared_flops"] / (iso["shared"] * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+            "shared_frac_of_nominal_2250": work["shared_flops"] / (iso["shared"] * 1e-3) / 1e12 / 2250.0,
             "shared_gbs": work["shared_bytes"] / (iso["shared"] * 1e-3) / 1e9,
+            "shared_frac_of_measured_hbm": work["shared_bytes"] / (iso["shared"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
         },
         "shared": {"tflops": shared_tflops, "frac_of_measured_sustained": (shared_tflops or 0) / peaks["bf16_tflops_sustained"],
                    "frac_of_nominal_2250": (shared_tflops or 0) / 2250.0, "gbs": shared_gbs,
                    "frac_of_measured_hbm": (shared_gbs or 0) / peaks["hbm_gbs"],
                    "touched_segments": touched, "pairs": P,
-                   "amortisation_factor": P / max(1, touched)},
+                   "amortisation_factor": amort},
         "unique": {"gbs": unique_gbs, "frac_of_measured_hbm": (unique_gbs or 0) / peaks["hbm_gbs"],
                    "frac_of_nominal_8000": (unique_gbs or 0) / 8000.0},
         # all HBM-bound work of the step against the step time: the two streams share the bandwidth,
         # so a kernel's own in-step rate (roofline.achieved) understates how busy HBM is
-        "step_hbm": {
-            "bytes": work["unique_bytes"] + work["shared_bytes"] + rows_merge_bytes,
-            "gbs": (work["unique_bytes"] + work["shared_bytes"] + rows_merge_bytes) / (ms_per_step * 1e-3) / 1e9,
-            "frac_of_measured_hbm": (work["unique_bytes"] + work["shared_bytes"] + rows_merge_bytes)
-                                    / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"]},
+        "step_hbm": {"bytes": hbm_bytes, "gbs": hbm_bytes / (ms_per_step * 1e-3) / 1e9,
+                     "frac_of_measured_hbm": hbm_bytes / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"]},
         "gemv_baseline": None if gemv_ms is None else {
             "ms": gemv_ms,
+            # algorithmic bytes of the baseline (every routed chunk once per request and KV head);
+            # where they fit the 126 MB L2 part of them never reaches DRAM
+            "algorithmic_gbs": work["gemv_bytes"] / (gemv_ms * 1e-3) / 1e9,
             # both kernels alone on the GPU (in the step part of shared attention overlaps unique)
             "shared_speedup": gemv_ms / iso["shared"] if iso["shared"] > 0 else None,
+            "amortisation_factor": amort,
+            "shared_speedup_over_amortisation": (gemv_ms / iso["shared"] / amort) if iso["shared"] > 0 else None,
             # the step with the per-request baseline in the place of shared attention, stages
             # back to back on one stream, against the real step
             "step_ms_with_baseline": gemv_step_ms,
             "step_speedup": None if gemv_step_ms is None else gemv_step_ms / ms_per_step},
     }
-    print(json.dumps(line), flush=True)
+    return rec
+
+
+def measure_disaggregated(args, w, rank, world, dev):
+    """Rank 0 as the Shared-KV rank, the others as Unique-KV ranks (Section III-C in miniature): per
+    step the unique ranks send their queries, run Unique KV Attention, receive the shared result of
+    their requests and merge.  Point-to-point over the process group; no kernel reads a peer."""
+    from paper_2511_06010_b200 import disaggregated as DG
+    from paper_2511_06010_b200.engine import MoskaLayer
+
+    if world < 2:
+        raise SystemExit("--shard disaggregated needs at least 2 ranks")
+    unique_ranks = list(range(1, world))
+    blocks = DG.request_blocks(w.B, unique_ranks)
+    lens_all = W.unique_lengths(w)
+    K = args.steps
+    if rank == 0:
+        sh = W.make_shared_store(w, dev)
+        layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, 1, dense=w.dense, n_unique_splits=1)
+        role = DG.SharedRank(layer, sh.k_shared, sh.v_shared)
+        q_all = torch.empty(w.B, w.Hq, w.D, dtype=torch.bfloat16, device=dev)
+        q_local = kv_len = None
+    else:
+        _, b0, b1 = [b for b in blocks if b[0] == rank][0]
+        wl = W.scaled(w, B=b1 - b0, shard=rank)
+        un = W.make_unique_store(wl, dev, lens_all[b0:b1])
+        mu = W.shared_centres(w, dev)
+        q_local = W.make_queries(w, W.SharedStore(None, None, mu), 0, dev)[b0:b1].contiguous()
+        kv_len = un.kv_len
+        layer = MoskaLayer(b1 - b0, w.Hq, w.Hkv, w.D, 1, w.L, 1, int(lens_all.max()) + w.steps)
+        role = DG.UniqueRank(layer, un.k_unique, un.v_unique, un.kv_start)
+        q_all = None
+
+    def one():
+        DG.step(role, q_local, kv_len, 0, blocks, q_all=q_all)
+
+    for _ in range(max(3, args.warmup)):
+        one()
+
+    def run_block():
+        DD.barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(K):
+            one()
+        e1.record()
+        torch.cuda.synchronize()
+        DD.barrier()
+        return e0.elapsed_time(e1)
+
+    sampler = ClockSampler(dev.index)
+    sampler.start()
+    blocks_ms = timed_blocks(run_block, args.min_timed_ms, dev)
+    clocks = sampler.stop()
+    if rank != 0:
+        return None
+    block_ms = statistics.median(blocks_ms)
+    rows = w.B * w.Hq
+    return {
+        "workload": w.name, "value": w.B * K / (block_ms * 1e-3), "ms_per_step": block_ms / K,
+        "steps_per_block": K, "blocks": len(blocks_ms), "scaling": "strong",
+        "config": {"workload": w.name, "batch": w.B,
+                   "per_gpu": f"rank 0: shared store, routing, grouping, Shared KV Attention for all {w.B} requests; "
+                              f"ranks 1..{world - 1}: private KV and Unique KV Attention of {w.B // (world - 1)} requests each",
+                   "exchange_bytes_per_step": {"queries_up": rows * w.D * 2, "shared_partials_down": rows * (w.D + 1) * 4},
+                   "timed_region": f"{len(blocks_ms)} blocks of {K} steps, median block"},
+        "clocks": clocks, "e2e": None, "gpu_launches": None, "roofline": None, "cpu_baseline": None,
+    }
+
+
+def run_cuda(args):
+    rank, local_rank, world = DD.init("nccl")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    from paper_2511_06010_b200 import build as B
+
+    if rank == 0:
+        B.build()
+    DD.barrier()
+
+    def pick(i):
+        w = W.CONFIGS[i]
+        if args.batch:
+            w = W.scaled(w, name=f"{w.name}@B{args.batch}", B=args.batch)
+        return w
+
+    headline_idx = HEADLINE_CONFIG if args.config is None else args.config
+    if world > 1 and args.shard == "disaggregated":
+        rec = measure_disaggregated(args, pick(headline_idx), rank, world, dev)
+        per = {}
+    else:
+        per = {}
+        if args.config is None and not args.no_per_config and world == 1:
+            for i in PER_CONFIG:
+                r = measure(args, pick(i), rank, world, dev, headline=False)
+                torch.cuda.empty_cache()
+                if r is not None:
+                    per[r["workload"]] = {
+                        k: r[k] for k in ("value", "ms_per_step", "blocks", "timed_ms_total", "roofline",
+                                          "gemv_baseline", "cpu_baseline", "stage_ms",
+                                          "stage_ms_isolated", "isolated", "shared", "unique", "step_hbm",
+                                          "e2e", "clocks")}
+        rec = measure(args, pick(headline_idx), rank, world, dev, headline=True)
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": rec["value"], "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": rec["ms_per_step"], "higher_is_better": True,
+            "scaling": rec["scaling"], "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        }
+        for k, v in rec.items():
+            if k not in ("workload", "value", "ms_per_step", "scaling"):
+                line[k] = v
+        if per:
+            line["per_config"] = per
+        print(json.dumps(line), flush=True)
     DD.finalize()
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=500)
+    ap.add_argument("--steps", type=int, default=20, help="K: steps per timed block")
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", type=int, default=1, help="workload index 0..4 (default 1)")
+    ap.add_argument("--config", type=int, default=None,
+                    help="workload index 0..4; default: 4 as the headline plus per_config records of 1, 2, 3")
+    ap.add_argument("--no-per-config", action="store_true", help="headline workload only")
+    ap.add_argument("--min-timed-ms", type=float, default=500.0,
+                    help="blocks of K steps are repeated until they add up to this much device time")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's batch size (sweeps)")
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
+    ap.add_argument("--shard", default="kv_head", choices=["kv_head", "replicas", "disaggregated"],
+                    help="what N > 1 ranks hold: KV heads of one batch (default), own batches, or the "
+                         "Shared-KV / Unique-KV roles")
     ap.add_argument("--one-stream", action="store_true", help="run unique attention on the main stream")
     ap.add_argument("--unique-splits", type=int, default=None, help="override the split-K count of unique attention")
     ap.add_argument("--unique-kv", default="bf16", choices=["bf16", "fp8"],
@@ -586,13 +806,13 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--ref-sample", type=int, default=8, help="requests per step of --impl reference")
     args = ap.parse_args()
-    w = W.CONFIGS[args.config]
-    if args.batch:
-        w = W.scaled(w, name=f"{w.name}@B{args.batch}", B=args.batch)
     if args.impl == "reference":
+        w = W.CONFIGS[HEADLINE_CONFIG if args.config is None else args.config]
+        if args.batch:
+            w = W.scaled(w, name=f"{w.name}@B{args.batch}", B=args.batch)
         run_reference(args, w)
     else:
-        run_cuda(args, w)
+        run_cuda(args)
 
 
 if __name__ == "__main__":

@@ -30,6 +30,16 @@
  *  * Return value: MOSKA_OK or a negative moska_status.  moska_last_error() gives a text for
  *    the last failure on the calling thread.  Invalid arguments are detected on the host
  *    before anything is launched.
+ *  * What a kernel can only find out while it runs (routing indices that break the grouping's
+ *    preconditions, an entry outside the batch, a bounded wait that ran out) goes to one sticky
+ *    status word per device, read and cleared by moska_device_status().  A kernel that raises it
+ *    never traps and never writes outside the caller's buffers; the results of that step are not
+ *    valid.
+ *  * Hidden state: none that outlives a call on the device side.  On the host side the library
+ *    keeps, per device ordinal, the address of its status word (and of the built-in scratch of
+ *    moska_group_by_chunk_noalloc), and per (host thread, device) the two CUDA events that order
+ *    the side stream of a two-stream moska_decode_step; all are created on first use with that
+ *    device current and are not valid across a cudaDeviceReset.
  */
 #ifndef MOSKA_H_
 #define MOSKA_H_
@@ -93,9 +103,13 @@ int moska_version(void);
 const char* moska_last_error(void);
 
 /* Waits for the current device to finish, stores the sticky device-side status word in
- * *status_host (host pointer) and clears it.  0 means no kernel of the library raised anything;
- * MOSKA_ERR_TIMEOUT means a CTA of the tensor-core Shared KV Attention kernel gave up on one of
- * its bounded waits (TMA or MMA completion) and its outputs are not valid. */
+ * *status_host (host pointer) and clears it.  0 means no kernel of the library raised anything.
+ * MOSKA_ERR_TIMEOUT: a CTA of the tensor-core Shared KV Attention kernel gave up on one of its
+ * bounded waits (TMA or MMA completion).  MOSKA_ERR_INVALID_ARG: a grouping call (either entry
+ * point) met a chunk index outside [0, C) or a (request, KV head) list that is not strictly
+ * ascending, or shared attention met an entry of seg_entries outside [0, B*Hkv*k).  In every
+ * case the outputs of the steps since the last read are not valid.  The most negative code
+ * raised since the last read is the one reported. */
 int moska_device_status(int32_t* status_host);
 
 /* n_slots = shared_slots + n_unique_splits; negative status if the shape is invalid. Host only. */
@@ -147,6 +161,12 @@ int moska_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, fl
  *   seg_entries  int32 [B*Hkv*k]    out, positions p, key-major, ascending p inside one key
  * The result is deterministic.  It also writes the tile work lists that moska_shared_attn
  * consumes into `ws` (give both calls the same, unmodified workspace).
+ * Precondition (what moska_route produces): every list topk_idx[b][h][0..k) is STRICTLY ASCENDING,
+ * hence without repeated chunks, and lies in [0, C).  The sort is done on one bit per (key,
+ * request), which only describes such lists.  The marking pass checks it on the device: an index
+ * outside [0, C) is skipped and a list out of order is flagged, both as MOSKA_ERR_INVALID_ARG in
+ * the device status word (moska_device_status); seg_entries then still holds only positions that
+ * exist, but a repeated or skipped chunk is missing from it, so the step's results are not valid.
  */
 int moska_group_by_chunk(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
                          const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream);
@@ -163,7 +183,8 @@ int moska_group_by_chunk(const int32_t* topk_idx, int32_t* seg_offsets, int32_t*
  * that loads the library keeps that buffer until the process exits.  The call allocates and
  * frees nothing, neither directly nor through another library.
  *
- *   inputs / outputs      as moska_group_by_chunk (topk_idx in; seg_offsets, seg_entries out)
+ *   inputs / outputs      as moska_group_by_chunk (topk_idx in; seg_offsets, seg_entries out),
+ *                         same precondition on topk_idx, same report through moska_device_status
  *   limit                 shapes whose grouping scratch (moska_workspace_bytes) exceeds the
  *                         buffer are rejected with MOSKA_ERR_WORKSPACE before anything runs
  *   first call            the first call on each device looks up the buffer's device address

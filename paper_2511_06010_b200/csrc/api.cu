@@ -1,7 +1,9 @@
 // extern "C" boundary of the MoSKA library: argument validation and launch sequencing only.
-#include <cstring>
-
 #include <cmath>
+#include <cstring>
+#include <mutex>
+
+#include <nvtx3/nvToolsExt.h>
 
 #include "common.cuh"
 
@@ -85,6 +87,15 @@ inline cudaError_t prof_mark(moska_profiler* p, int stage, int which, cudaStream
 }
 }  // namespace
 
+// One NVTX range per entry point (visible in a timeline profiler; a no-op when no tool is attached).
+struct ApiRange {
+    explicit ApiRange(const char* name) { nvtxRangePushA(name); }
+    ~ApiRange() { nvtxRangePop(); }
+    ApiRange(const ApiRange&) = delete;
+    ApiRange& operator=(const ApiRange&) = delete;
+};
+#define MOSKA_API_RANGE() ApiRange api_range__(__func__)
+
 #define MOSKA_TRY(expr)              \
     do {                             \
         int st__ = (expr);           \
@@ -149,10 +160,11 @@ int moska_default_unique_splits_fp8(int32_t B, int32_t Hkv, int32_t max_len)
 int moska_build_chunk_summaries(const uint16_t* k_shared, float* summaries,
                                 const moska_shape* shape, moska_stream stream)
 {
+    MOSKA_API_RANGE();
     MOSKA_TRY(check_shape(shape, false));
-    MOSKA_TRY(check_device());
     REQUIRE_PTR(k_shared, 16);
     REQUIRE_PTR(summaries, 16);
+    MOSKA_TRY(check_device());
     return launch_summaries(k_shared, summaries, shape, (cudaStream_t)stream);
 }
 
@@ -182,13 +194,32 @@ int tc_sm_share(const moska_shape* s, bool dense, double unique_ms)
     return x;
 }
 
+// The event pair that orders the side stream of a two-stream step after / before the main
+// stream.  Events belong to the device they were created on, so there is one pair per (host
+// thread, device ordinal), created on first use with that device current and kept.
+int fork_join_events(cudaEvent_t* fork, cudaEvent_t* join)
+{
+    constexpr int kMaxDevices = 64;
+    static thread_local cudaEvent_t ev[kMaxDevices][2] = {};
+    int dev = 0;
+    MOSKA_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices)
+        return fail(MOSKA_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
+    if (ev[dev][0] == nullptr) {
+        MOSKA_CUDA_TRY(cudaEventCreateWithFlags(&ev[dev][0], cudaEventDisableTiming));
+        MOSKA_CUDA_TRY(cudaEventCreateWithFlags(&ev[dev][1], cudaEventDisableTiming));
+    }
+    *fork = ev[dev][0];
+    *join = ev[dev][1];
+    return MOSKA_OK;
+}
+
 // Validation + launch of the router; mark_groups also runs the grouping's first pass in it.
 int route_impl(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
                const moska_shape* shape, void* ws, size_t ws_bytes, bool mark_groups,
                cudaStream_t stream)
 {
     MOSKA_TRY(check_shape(shape, true));
-    MOSKA_TRY(check_device());
     REQUIRE_PTR(q, 16);
     REQUIRE_PTR(summaries, 16);
     REQUIRE_PTR(topk_idx, 4);
@@ -196,6 +227,7 @@ int route_impl(const uint16_t* q, const float* summaries, int32_t* topk_idx, flo
         (ws == nullptr || !aligned(ws, 256) || ws_bytes < ws_layout(shape).total))
         return fail(MOSKA_ERR_WORKSPACE, "workspace missing, misaligned or smaller than %zu bytes",
                     ws_layout(shape).total);
+    MOSKA_TRY(check_device());
     return launch_route(q, summaries, topk_idx, topk_score, shape, ws, mark_groups, stream);
 }
 
@@ -204,13 +236,13 @@ int group_impl(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entri
                cudaStream_t stream)
 {
     MOSKA_TRY(check_shape(shape, true));
-    MOSKA_TRY(check_device());
     REQUIRE_PTR(topk_idx, 4);
     REQUIRE_PTR(seg_offsets, 4);
     REQUIRE_PTR(seg_entries, 4);
     if (ws == nullptr || !aligned(ws, 256) || ws_bytes < ws_layout(shape).total)
         return fail(MOSKA_ERR_WORKSPACE, "workspace missing, misaligned or smaller than %zu bytes",
                     ws_layout(shape).total);
+    MOSKA_TRY(check_device());
     return launch_group(topk_idx, seg_offsets, seg_entries, shape, ws, premarked, stream);
 }
 }  // namespace
@@ -218,6 +250,7 @@ int group_impl(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entri
 int moska_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
                 const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream)
 {
+    MOSKA_API_RANGE();
     return route_impl(q, summaries, topk_idx, topk_score, shape, ws, ws_bytes, false,
                       (cudaStream_t)stream);
 }
@@ -225,6 +258,7 @@ int moska_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, fl
 int moska_group_by_chunk(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
                          const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream)
 {
+    MOSKA_API_RANGE();
     return group_impl(topk_idx, seg_offsets, seg_entries, shape, ws, ws_bytes, false,
                       (cudaStream_t)stream);
 }
@@ -233,6 +267,7 @@ int moska_group_by_chunk_noalloc(const int32_t* topk_idx, int32_t* seg_offsets,
                                  int32_t* seg_entries, const moska_shape* shape,
                                  moska_stream stream)
 {
+    MOSKA_API_RANGE();
     MOSKA_TRY(check_shape(shape, true));
     REQUIRE_PTR(topk_idx, 4);
     REQUIRE_PTR(seg_offsets, 4);
@@ -246,9 +281,9 @@ int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_
                       float softmax_scale, const moska_shape* shape, void* ws, size_t ws_bytes,
                       moska_stream stream)
 {
+    MOSKA_API_RANGE();
     const bool dense = (topk_idx == nullptr && seg_offsets == nullptr && seg_entries == nullptr);
     MOSKA_TRY(check_shape(shape, !dense));
-    MOSKA_TRY(check_device());
     REQUIRE_PTR(q, 16);
     REQUIRE_PTR(k_shared, 128);
     REQUIRE_PTR(v_shared, 128);
@@ -266,6 +301,7 @@ int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_
     } else if (shape->shared_slots > shape->C) {
         return fail(MOSKA_ERR_INVALID_ARG, "dense mode needs shared_slots <= C");
     }
+    MOSKA_TRY(check_device());
     cudaStream_t st = (cudaStream_t)stream;
     const bool tc = shared_tc_supported(shape);
     if (dense) {
@@ -288,7 +324,7 @@ int moska_device_status(int32_t* status_host)
 {
     if (status_host == nullptr) return fail(MOSKA_ERR_INVALID_ARG, "status_host is NULL");
     int v = 0;
-    MOSKA_TRY(read_tc_status(&v));
+    MOSKA_TRY(read_status(&v));
     *status_host = v;
     return MOSKA_OK;
 }
@@ -298,12 +334,12 @@ int moska_unique_attn(const uint16_t* q, const uint16_t* k_unique, const uint16_
                       float* lse_part, float softmax_scale, const moska_shape* shape,
                       moska_stream stream)
 {
+    MOSKA_API_RANGE();
     MOSKA_TRY(check_shape(shape, false));
     if (shape->q_len > 1 && (shape->D != 128 || shape->q_len * (shape->Hq / shape->Hkv) > 16))
         return fail(MOSKA_ERR_UNSUPPORTED,
                     "q_len = %d needs D = 128 and q_len * G <= 16; pass the tokens as batch rows "
                     "with q_len = 1 and aliased kv_start instead", shape->q_len);
-    MOSKA_TRY(check_device());
     REQUIRE_PTR(q, 16);
     REQUIRE_PTR(k_unique, 16);
     REQUIRE_PTR(v_unique, 16);
@@ -311,6 +347,7 @@ int moska_unique_attn(const uint16_t* q, const uint16_t* k_unique, const uint16_
     REQUIRE_PTR(kv_len, 4);
     REQUIRE_PTR(o_part, 16);
     REQUIRE_PTR(lse_part, 4);
+    MOSKA_TRY(check_device());
     return launch_unique(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part, softmax_scale,
                          shape, (cudaStream_t)stream);
 }
@@ -320,13 +357,13 @@ int moska_unique_attn_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v
                           const int32_t* kv_len, float* o_part, float* lse_part,
                           float softmax_scale, const moska_shape* shape, moska_stream stream)
 {
+    MOSKA_API_RANGE();
     MOSKA_TRY(check_shape(shape, false));
     if (shape->D != 128) return fail(MOSKA_ERR_UNSUPPORTED, "FP8 unique attention is built for D = 128");
     if (shape->q_len > 1 && shape->q_len * (shape->Hq / shape->Hkv) > 8)
         return fail(MOSKA_ERR_UNSUPPORTED,
                     "FP8 unique attention with q_len = %d needs q_len * G <= 8; pass the tokens as "
                     "batch rows with q_len = 1 and aliased kv_start instead", shape->q_len);
-    MOSKA_TRY(check_device());
     REQUIRE_PTR(q, 16);
     REQUIRE_PTR(k8, 16);
     REQUIRE_PTR(v8, 16);
@@ -336,6 +373,7 @@ int moska_unique_attn_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v
     REQUIRE_PTR(kv_len, 4);
     REQUIRE_PTR(o_part, 16);
     REQUIRE_PTR(lse_part, 4);
+    MOSKA_TRY(check_device());
     return launch_unique_fp8(q, k8, v8, k_scale, v_scale, kv_start, kv_len, o_part, lse_part,
                              softmax_scale, shape, (cudaStream_t)stream);
 }
@@ -343,11 +381,12 @@ int moska_unique_attn_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v
 int moska_merge(const float* o_part, const float* lse_part, uint16_t* out, float* out_f32,
                 float* lse_out, const moska_shape* shape, moska_stream stream)
 {
+    MOSKA_API_RANGE();
     MOSKA_TRY(check_shape(shape, false));
-    MOSKA_TRY(check_device());
     REQUIRE_PTR(o_part, 16);
     REQUIRE_PTR(lse_part, 4);
     REQUIRE_PTR(out, 8);
+    MOSKA_TRY(check_device());
     if (out_f32 != nullptr && !aligned(out_f32, 16))
         return fail(MOSKA_ERR_INVALID_ARG, "out_f32 is not 16-byte aligned");
     return launch_merge(o_part, lse_part, out, out_f32, lse_out, shape, (cudaStream_t)stream);
@@ -357,14 +396,15 @@ int moska_gemv_baseline(const uint16_t* q, const uint16_t* k_shared, const uint1
                         const int32_t* topk_idx, float* o_part, float* lse_part,
                         float softmax_scale, const moska_shape* shape, moska_stream stream)
 {
+    MOSKA_API_RANGE();
     const bool dense = topk_idx == nullptr;
     MOSKA_TRY(check_shape(shape, !dense));
-    MOSKA_TRY(check_device());
     REQUIRE_PTR(q, 16);
     REQUIRE_PTR(k_shared, 16);
     REQUIRE_PTR(v_shared, 16);
     REQUIRE_PTR(o_part, 16);
     REQUIRE_PTR(lse_part, 4);
+    MOSKA_TRY(check_device());
     if (!dense && shape->shared_slots != shape->k)
         return fail(MOSKA_ERR_INVALID_ARG, "routed mode needs shared_slots == k");
     if (dense && shape->shared_slots > shape->C)
@@ -433,11 +473,8 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
         // only a share of the SMs so that unique attention keeps the others and HBM stays busy
         // while the tensor pipe works -- the single-GPU form of the paper's split into Shared-KV
         // and Unique-KV nodes (Section III-C).
-        static thread_local cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
-        if (ev_fork == nullptr) {
-            MOSKA_CUDA_TRY(cudaEventCreateWithFlags(&ev_fork, cudaEventDisableTiming));
-            MOSKA_CUDA_TRY(cudaEventCreateWithFlags(&ev_join, cudaEventDisableTiming));
-        }
+        cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+        MOSKA_TRY(fork_join_events(&ev_fork, &ev_join));
         MOSKA_TRY(check_shape(shape, !dense));
         REQUIRE_PTR(k_shared, 128);
         REQUIRE_PTR(v_shared, 128);
@@ -502,6 +539,7 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
                       float softmax_scale, const moska_shape* shape, void* ws, size_t ws_bytes,
                       moska_stream stream, moska_stream side_stream, moska_profiler* prof)
 {
+    MOSKA_API_RANGE();
     UniqueKv kv;
     kv.k = k_unique;
     kv.v = v_unique;
@@ -519,6 +557,7 @@ int moska_decode_step_fp8kv(const uint16_t* q, const float* summaries, const uin
                             const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream,
                             moska_stream side_stream, moska_profiler* prof)
 {
+    MOSKA_API_RANGE();
     UniqueKv kv;
     kv.k8 = k8_unique;
     kv.v8 = v8_unique;
@@ -596,6 +635,7 @@ int moska_decode_step_host(const uint16_t* q_host, uint16_t* q_dev, const float*
                            size_t ws_bytes, moska_stream stream, moska_stream side_stream,
                            moska_profiler* prof)
 {
+    MOSKA_API_RANGE();
     MOSKA_TRY(check_shape(shape, summaries != nullptr));
     if (q_host == nullptr || q_dev == nullptr || out_dev == nullptr || out_host == nullptr)
         return fail(MOSKA_ERR_INVALID_ARG, "q_host, q_dev, out_dev and out_host must not be NULL");

@@ -58,7 +58,7 @@ struct TileItem {
 struct WsHeader {
     int32_t n_small_tiles;  // items in the small-tile list
     int32_t n_big_tiles;    // items in the big-tile list
-    int32_t status;         // 0, or a negative code set by a device-side range check
+    int32_t reserved;
     int32_t n_tiny_tiles;   // items in the 8-row tile list
     int32_t pad[60];
 };
@@ -107,8 +107,11 @@ int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t
                      const moska_shape* s, void* ws, bool dense, int max_ctas, cudaStream_t st);
 // Estimated SM-milliseconds of the tensor-core kernel for this shape (host, pure).
 double shared_tc_cost_sm_ms(const moska_shape* s, bool dense);
-// Synchronises the device, returns the sticky status of the tensor-core kernel and clears it.
-int read_tc_status(int* out);
+// Device address (on the current device) of the library's sticky status word: kernels lower it
+// with atomicMin to a negative moska_status when they detect a problem while running.
+int status_word(int** out);
+// Synchronises the device, returns the sticky status word and clears it.
+int read_status(int* out);
 int launch_unique(const uint16_t* q, const uint16_t* k_unique, const uint16_t* v_unique,
                   const int64_t* kv_start, const int32_t* kv_len, float* o_part, float* lse_part,
                   float scale, const moska_shape* s, cudaStream_t st);

@@ -49,18 +49,20 @@ WsLayout ws_layout(const moska_shape* s)
 
 namespace {
 
-// Pass 1: one thread per routed pair p = (b*Hkv + h)*k + j.
+// Pass 1: one thread per routed pair p = (b*Hkv + h)*k + j.  Also checks what the bit-set form
+// relies on: every index inside [0, C) and every (b, h) list strictly ascending (hence distinct).
 __global__ void __launch_bounds__(256)
 group_mark_kernel(const int32_t* __restrict__ topk_idx, uint32_t* __restrict__ bitmap,
-                  WsHeader* __restrict__ hdr, long long P, int Hkv, int C, int k, int words)
+                  int* __restrict__ status, long long P, int Hkv, int C, int k, int words)
 {
     const long long p = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (p >= P) return;
     const int c = topk_idx[p];
     if (c < 0 || c >= C) {  // corrupt routing: record it, touch nothing
-        atomicMin(&hdr->status, (int)MOSKA_ERR_INVALID_ARG);
+        atomicMin(status, (int)MOSKA_ERR_INVALID_ARG);
         return;
     }
+    if (p % k != 0 && topk_idx[p - 1] >= c) atomicMin(status, (int)MOSKA_ERR_INVALID_ARG);
     const int h = (int)((p / k) % Hkv);
     const int b = (int)(p / ((long long)k * Hkv));
     atomicOr(&bitmap[((size_t)h * C + c) * words + (b >> 5)], 1u << (b & 31));
@@ -178,7 +180,7 @@ group_scan_kernel(const uint32_t* __restrict__ bitmap, int words, const int32_t*
 __global__ void __launch_bounds__(256)
 group_emit_kernel(const int32_t* __restrict__ topk_idx, const uint32_t* __restrict__ bitmap,
                   const int32_t* __restrict__ seg_offsets, int32_t* __restrict__ seg_entries,
-                  int n_keys, int Hkv, int C, int k, int words)
+                  int* __restrict__ status, int n_keys, int Hkv, int C, int k, int words)
 {
     const int key = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
@@ -209,6 +211,16 @@ group_emit_kernel(const int32_t* __restrict__ topk_idx, const uint32_t* __restri
                 const int mid = (lo + hi) >> 1;
                 if (lst[mid] < c) lo = mid + 1; else hi = mid;
             }
+            if (lst[lo] != c) {
+                // the list is not ascending (reported by the marking pass): find the slot by a
+                // plain scan so that the entry written is a position that exists
+                atomicMin(status, (int)MOSKA_ERR_INVALID_ARG);
+                for (int j = 0; j < k; ++j)
+                    if (lst[j] == c) {
+                        lo = j;
+                        break;
+                    }
+            }
             seg_entries[rank++] = (b * Hkv + h) * k + lo;
         }
         rank0 += __shfl_sync(0xffffffffu, inc, 31);
@@ -228,11 +240,13 @@ int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_ent
     TileItem* big_items = reinterpret_cast<TileItem*>(base + lay.off_big);
     TileItem* tiny_items = reinterpret_cast<TileItem*>(base + lay.off_tiny);
     const long long P = (long long)s->B * s->Hkv * s->k;
+    int* status = nullptr;
+    MOSKA_TRY_STATUS(status_word(&status));
     // header and bit sets must start at zero; the router has done both passes already when the
     // two calls run back to back inside moska_decode_step
     if (!premarked) MOSKA_CUDA_TRY(cudaMemsetAsync(base, 0, lay.off_totals, st));
     if (!premarked && P > 0) {
-        group_mark_kernel<<<(unsigned)((P + 255) / 256), 256, 0, st>>>(topk_idx, bitmap, hdr, P,
+        group_mark_kernel<<<(unsigned)((P + 255) / 256), 256, 0, st>>>(topk_idx, bitmap, status, P,
                                                                        s->Hkv, s->C, s->k, lay.words);
         MOSKA_LAUNCH_CHECK("group_mark_kernel");
     }
@@ -247,7 +261,7 @@ int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_ent
                                           lay.big_entries, lay.big_min_entries);
     MOSKA_LAUNCH_CHECK("group_scan_kernel");
     group_emit_kernel<<<(lay.n_keys + 7) / 8, 256, 0, st>>>(topk_idx, bitmap, seg_offsets, seg_entries,
-                                                            lay.n_keys, s->Hkv, s->C, s->k, lay.words);
+                                                            status, lay.n_keys, s->Hkv, s->C, s->k, lay.words);
     MOSKA_LAUNCH_CHECK("group_emit_kernel");
     return MOSKA_OK;
 }

@@ -42,8 +42,6 @@ constexpr int kSoftmaxRegs = 208, kOtherRegs = 80;  // per-thread register budge
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.f;       // log2 units a row maximum may lag behind
-// Of every kPolyPeriod pairs of score columns, kPolyPairs take exp2 as a polynomial on the FMA pipe.
-constexpr int kPolyPeriod = 2, kPolyPairs = 0;
 
 struct __align__(1024) TcSmem {
     uint8_t q[2][kTileBytes];
@@ -68,8 +66,6 @@ struct TcParams {
     float scale;
     int B, Hq, Hkv, C, L, k, shared_slots, n_slots, dense, n_items_dense;
 };
-
-__device__ int g_tc_status = 0;  // sticky: first negative status raised by a tensor-core CTA
 
 __device__ __forceinline__ float fast_exp2(float x)
 {
@@ -123,27 +119,6 @@ __device__ __forceinline__ float fmax3(float a, float b, float c)
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
     return d;
-}
-
-// 2^x for two values on the FMA pipe instead of the special-function unit: round x to the nearest
-// integer n with the 1.5 * 2^23 trick, 2^(x - n) by a cubic with relative error 7.6e-5 on
-// [-0.5, 0.5], then n is added into the exponent field.  x is clamped at -125 (result ~ 2^-125).
-__device__ __forceinline__ float2 exp2_poly2(float2 x)
-{
-    const float kMagic = 12582912.f;  // 1.5 * 2^23
-    x.x = fmaxf(x.x, -125.f);
-    x.y = fmaxf(x.y, -125.f);
-    const float2 t = fadd2(x, make_float2(kMagic, kMagic));
-    const float2 n = fadd2(t, make_float2(-kMagic, -kMagic));
-    const float2 f = ffma2(n, make_float2(-1.f, -1.f), x);
-    float2 q = ffma2(f, make_float2(0.05521666631102562f, 0.05521666631102562f),
-                     make_float2(0.24261489510536194f, 0.24261489510536194f));
-    q = ffma2(q, f, make_float2(0.693252682685852f, 0.693252682685852f));
-    q = ffma2(q, f, make_float2(0.9999276399612427f, 0.9999276399612427f));
-    float2 r;
-    r.x = __int_as_float(__float_as_int(q.x) + (__float_as_int(t.x) << 23));
-    r.y = __int_as_float(__float_as_int(q.y) + (__float_as_int(t.y) << 23));
-    return r;
 }
 
 // One work item.  The CTA has two "slots" (t = 0, 1), each with its own S/P and O accumulator in
@@ -523,8 +498,6 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     }
                 }
                 // P = exp2((S - m_ref) * scale * log2 e) as bf16, written over the columns of S
-                // Every other pair of columns takes its exponential on the FMA pipe, the rest on the
-                // special-function unit, so that neither pipe alone bounds the row.
                 const float2 sl2_2 = make_float2(sl2, sl2);
                 const float2 nmb_2 = make_float2(-m_ref * sl2, -m_ref * sl2);
                 float2 ls[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};  // partial row sums
@@ -537,12 +510,8 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                                                            __uint_as_float(r[c][2 * x + 1])),
                                                sl2_2, nmb_2);
                         float2 pr;
-                        if ((x % kPolyPeriod) < kPolyPairs) {
-                            pr = exp2_poly2(e);
-                        } else {
-                            pr.x = fast_exp2(e.x);
-                            pr.y = fast_exp2(e.y);
-                        }
+                        pr.x = fast_exp2(e.x);
+                        pr.y = fast_exp2(e.y);
                         ls[x & 1] = fadd2(ls[x & 1], pr);
                         __nv_bfloat162 b2 = __floats2bfloat162_rn(pr.x, pr.y);
                         pk[x] = *reinterpret_cast<uint32_t*>(&b2);
@@ -734,7 +703,7 @@ int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t
     MOSKA_TRY_STATUS(make_kv_map(&tm_v, v_shared, kv_rows));
     MOSKA_TRY_STATUS(make_q_map(&tm_q, q, (long long)s->B * s->Hq));
     int* status = nullptr;
-    MOSKA_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&status), g_tc_status));
+    MOSKA_TRY_STATUS(status_word(&status));
     p.q = q;
     p.seg_entries = seg_entries;
     p.o_part = o_part;
@@ -777,15 +746,6 @@ double shared_tc_cost_sm_ms(const moska_shape* s, bool dense)
         two_tiles = P / segs > kBigTileRows / G;
     }
     return items * (6.0 + (two_tiles ? 2.2 : 1.1) * n_kv) * 1e-3;
-}
-
-int read_tc_status(int* out)
-{
-    MOSKA_CUDA_TRY(cudaDeviceSynchronize());
-    MOSKA_CUDA_TRY(cudaMemcpyFromSymbol(out, g_tc_status, sizeof(int)));
-    const int zero = 0;
-    MOSKA_CUDA_TRY(cudaMemcpyToSymbol(g_tc_status, &zero, sizeof(int)));
-    return MOSKA_OK;
 }
 
 }  // namespace moska

@@ -291,14 +291,9 @@ int launch_unique(const uint16_t* q, const uint16_t* k_unique, const uint16_t* v
         MOSKA_LAUNCH_CHECK("unique_staged_kernel");
         return MOSKA_OK;
     }
-    if (s->D == 128)
-        unique_attn_kernel<128><<<(unsigned)grid, kThreads, 0, st>>>(
-            q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part, scale, s->Hq, s->Hkv,
-            s->n_unique_splits, s->shared_slots, n_slots);
-    else
-        unique_attn_kernel<64><<<(unsigned)grid, kThreads, 0, st>>>(
-            q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part, scale, s->Hq, s->Hkv,
-            s->n_unique_splits, s->shared_slots, n_slots);
+    unique_attn_kernel<64><<<(unsigned)grid, kThreads, 0, st>>>(
+        q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part, scale, s->Hq, s->Hkv,
+        s->n_unique_splits, s->shared_slots, n_slots);
     MOSKA_LAUNCH_CHECK("unique_attn_kernel");
     return MOSKA_OK;
 }

@@ -72,6 +72,8 @@ def receive_shared_partial(o_buf: torch.Tensor, lse_buf: torch.Tensor, shared_ra
 class SharedRank:
     """Routing, grouping and Shared KV Attention for all requests, merged over the routed chunks."""
 
+    is_shared_rank = True
+
     def __init__(self, layer, k_shared, v_shared):
         # `layer`: a MoskaLayer for ALL requests with n_unique_splits = 1; its one unique slot stays
         # empty (lse = -inf), so the merge combines the shared slots only.
@@ -96,6 +98,8 @@ class SharedRank:
 
 class UniqueRank:
     """Unique KV Attention of this rank's requests and the final merge with the shared result."""
+
+    is_shared_rank = False
 
     def __init__(self, layer, k_unique, v_unique, kv_start):
         # `layer`: a MoskaLayer for this rank's requests with shared_slots = 1: slot 0 takes the
@@ -123,7 +127,7 @@ def step(role, q_local, kv_len, shared_rank: int, blocks, q_all=None, group=None
     """One decode step on this rank.  `role` is a SharedRank (pass q_all, its [B][Hq][D] buffer)
     or a UniqueRank (pass q_local and kv_len); returns the outputs of the rank's own requests
     (None on the shared rank)."""
-    if isinstance(role, SharedRank):
+    if getattr(role, "is_shared_rank", False):
         gather_queries(q_all, blocks, group)
         o, lse = role.compute(q_all)
         return_shared_partials(o, lse, blocks, group)

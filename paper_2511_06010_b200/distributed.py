@@ -1,9 +1,12 @@
 """Host-side multi-process plumbing of the benchmark (torch.distributed; NCCL on GPUs, gloo on CPU).
 
 The decode-attention path needs no data-path collective: routing, shared attention, unique
-attention and the merge are independent per (request, KV head), so ranks either take disjoint
-request batches against a replicated shared store (what the benchmark does, weak scaling) or
-disjoint KV heads of the same batch (`kv_head_shard`).  Only the timing is reduced over ranks.
+attention and the merge are independent per (request, KV head).  One batch is therefore split by
+KV HEAD: rank r holds heads [h0, h1) of the shared store and of every request's private store,
+receives those heads' queries and produces those heads' outputs, with no exchange on the path
+(`kv_head_shard`, `slice_kv_heads`; the paper's point is that the shared store is NOT replicated,
+Section I).  Replicas (every rank its own batch and its own copy of the shared store) remain
+available to the benchmark behind a flag.  Only the timing is reduced over ranks.
 """
 from __future__ import annotations
 
@@ -63,6 +66,15 @@ def kv_head_shard(Hkv: int, rank: int, world: int) -> Tuple[int, int]:
     per = (Hkv + world - 1) // world
     h0 = min(Hkv, rank * per)
     return h0, min(Hkv, h0 + per)
+
+
+def slice_kv_heads(h0: int, h1: int, G: int, q, k_shared, v_shared, k_unique, v_unique):
+    """The tensors of KV heads [h0, h1) of one batch, as dense buffers of their own (what the rank
+    that owns those heads holds): q [B][(h1-h0)*G][D], shared K/V [h1-h0][C][L][D], private K/V
+    [T][h1-h0][D].  Indexing only; request structure (kv_start, kv_len) is the same on every rank."""
+    return (q[:, h0 * G:h1 * G].contiguous(), k_shared[h0:h1].contiguous(),
+            v_shared[h0:h1].contiguous(), k_unique[:, h0:h1].contiguous(),
+            v_unique[:, h0:h1].contiguous())
 
 
 def finalize() -> None:

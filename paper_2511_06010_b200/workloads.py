@@ -34,6 +34,8 @@ class Workload:
     zipf_s: float = 0.0     # > 0: query target chunk ~ Zipf(s) over chunk rank c+1; else uniform
     steps: int = 1          # consecutive decode steps (re-routing every step)
     seed: int = 0
+    shard: int = 0          # index of a KV-head shard of the workload: changes the drawn K/V values
+                            # only, never the request structure (lengths, query targets)
 
     @property
     def G(self) -> int:
@@ -87,9 +89,18 @@ def _gen(seed: int, device) -> torch.Generator:
     return g
 
 
+def kv_head_shard(w: Workload, rank: int, world: int) -> Workload:
+    """The part of workload `w` that rank `rank` of `world` holds when ONE batch is split by KV
+    head: the same requests (lengths, query targets), Hkv / world KV heads with their G query heads
+    each, and that many heads' share of the shared and private stores."""
+    if w.Hkv % world != 0:
+        raise ValueError(f"{w.Hkv} KV heads do not split evenly over {world} ranks")
+    return scaled(w, Hq=w.Hq // world, Hkv=w.Hkv // world, shard=rank)
+
+
 def make_shared_store(w: Workload, device="cpu") -> SharedStore:
     """Keys of chunk c (per KV head) are mu[h][c] + 0.5 N(0, I); values are N(0, I); bf16."""
-    g = _gen(w.seed * 1000 + 1, device)
+    g = _gen(w.seed * 1000 + 1 + 7919 * w.shard, device)
     mu = torch.randn(w.Hkv, w.C, w.D, generator=g, device=device, dtype=torch.float32)
     k_shared = torch.empty(w.Hkv, w.C, w.L, w.D, device=device, dtype=torch.bfloat16)
     v_shared = torch.empty(w.Hkv, w.C, w.L, w.D, device=device, dtype=torch.bfloat16)
@@ -106,6 +117,13 @@ def make_shared_store(w: Workload, device="cpu") -> SharedStore:
     return SharedStore(k_shared, v_shared, mu)
 
 
+def shared_centres(w: Workload, device="cpu") -> torch.Tensor:
+    """The cluster centres mu [Hkv][C][D] of make_shared_store(w) without the store itself (the
+    first draw of the same generator): what a rank that holds no shared KV needs to draw queries."""
+    g = _gen(w.seed * 1000 + 1 + 7919 * w.shard, device)
+    return torch.randn(w.Hkv, w.C, w.D, generator=g, device=device, dtype=torch.float32)
+
+
 def unique_lengths(w: Workload) -> np.ndarray:
     """Per-request unique context length at step 0 (host-side seeded draw)."""
     rng = np.random.default_rng(w.seed * 1000 + 2)
@@ -120,7 +138,7 @@ def make_unique_store(w: Workload, device="cpu", lengths: Optional[np.ndarray] =
     cap = lens + w.steps
     start = np.concatenate([[0], np.cumsum(cap)[:-1]]).astype(np.int64)
     total = int(cap.sum())
-    g = _gen(w.seed * 1000 + 3, device)
+    g = _gen(w.seed * 1000 + 3 + 7919 * w.shard, device)
     k_unique = torch.empty(max(total, 1), w.Hkv, w.D, device=device, dtype=torch.bfloat16)
     v_unique = torch.empty(max(total, 1), w.Hkv, w.D, device=device, dtype=torch.bfloat16)
     step = max(1, (1 << 25) // (w.Hkv * w.D))
@@ -153,7 +171,7 @@ def query_targets(w: Workload, step: int = 0) -> np.ndarray:
 def make_queries(w: Workload, shared: SharedStore, step: int = 0, device="cpu") -> torch.Tensor:
     """q[b][hq] = mu[hq // G][target_b] + 0.5 N(0, I), independent noise per query head; bf16."""
     tgt = torch.from_numpy(query_targets(w, step)).to(device)
-    g = _gen(w.seed * 1000 + 100 + step, device)
+    g = _gen(w.seed * 1000 + 100 + step + 7919 * w.shard, device)
     noise = torch.randn(w.B, w.Hq, w.D, generator=g, device=device, dtype=torch.float32)
     head_of = torch.arange(w.Hq, device=device) // w.G
     centre = shared.mu[head_of[None, :], tgt[:, None], :]          # [B][Hq][D]

@@ -93,3 +93,39 @@ def test_null_pointer_and_workspace_errors_come_before_any_launch(M):
         M.partial_slots(bad)
     assert e.value.status == M.ERR_INVALID_ARG
     assert M.workspace_bytes(bad) == 0
+
+
+def test_misaligned_pointers_are_rejected_on_the_host(M):
+    """Every entry point names its alignment (16 bytes for q and the private store, 128 for the
+    TMA-read shared store, 32 for the partial outputs, 256 for the workspace); a pointer that
+    breaks it is an invalid argument before any launch, whatever the other arguments are."""
+    s = M.shape(4, 32, 8, 128, 128, 512, 8)
+    A = 0x10000  # aligned to everything asked for
+    cases = [
+        lambda: M.route(A + 2, A, A, None, s, stream=0),
+        lambda: M.route(A, A + 4, A, None, s, stream=0),
+        lambda: M.build_chunk_summaries(A + 8, A, s, stream=0),
+        lambda: M.shared_attn(A, A + 64, A, A, A, A, A, A, 1.0, s, None, stream=0),
+        lambda: M.shared_attn(A, A, A + 16, A, A, A, A, A, 1.0, s, None, stream=0),
+        lambda: M.shared_attn(A, A, A, A, A, A, A + 16, A, 1.0, s, None, stream=0),
+        lambda: M.unique_attn(A, A + 2, A, A, A, A, A, 1.0, s, stream=0),
+        lambda: M.unique_attn(A, A, A, A + 4, A, A, A, 1.0, s, stream=0),
+        lambda: M.merge(A + 8, A, A, None, None, s, stream=0),
+        lambda: M.merge(A, A, A + 2, None, None, s, stream=0),
+        lambda: M.gemv_baseline(A, A, A + 8, A, A, A, 1.0, s, stream=0),
+        lambda: M.group_by_chunk_noalloc(A + 2, A, A, s, stream=0),
+    ]
+    for i, call in enumerate(cases):
+        with pytest.raises(M.MoskaError) as e:
+            call()
+        assert e.value.status == M.ERR_INVALID_ARG, f"case {i}: {M.last_error()}"
+        assert "aligned" in M.last_error(), f"case {i}: {M.last_error()}"
+    # a misaligned (or missing) workspace is a workspace error
+    import ctypes
+
+    lib = ctypes.CDLL(M.LIB_PATH)
+    lib.moska_group_by_chunk.restype = ctypes.c_int
+    lib.moska_group_by_chunk.argtypes = M.EXPORTS["moska_group_by_chunk"][1]
+    need = M.workspace_bytes(s)
+    assert lib.moska_group_by_chunk(A, A, A, ctypes.byref(s), A + 128, need, 0) == M.ERR_WORKSPACE
+    assert lib.moska_group_by_chunk(A, A, A, ctypes.byref(s), A, need - 1, 0) == M.ERR_WORKSPACE

@@ -89,8 +89,7 @@ def run_case(w: W.Workload, sample=None, lengths=None, n_unique_splits=None, ste
         off_ref, ent_ref = O.group_by_chunk(gpu_idx, w.C, fast=True)
         assert np.array_equal(layer.seg_offsets.cpu().numpy(), off_ref)
         assert np.array_equal(layer.seg_entries.cpu().numpy()[: len(ent_ref)], ent_ref)
-        status = layer.ws[:12].view(torch.int32).cpu().numpy()
-        assert status[2] == 0, "device-side range check of the grouping fired"
+        assert M.device_status() == 0, "a device-side check of the grouping fired"
         topk = layer.topk_idx
     else:
         topk = torch.arange(w.C, dtype=torch.int32, device=dev).repeat(w.B, w.Hkv, 1)
@@ -305,23 +304,40 @@ def test_chunk_lengths_of_one_three_and_five_kv_tiles():
         run_case(W.scaled(w, B=24, C=3, k=3), n_unique_splits=1, dense_slots=2)
 
 
-def _sample(w, n):
-    return np.sort(np.random.default_rng(7).choice(w.B, size=min(n, w.B), replace=False))
+def _sample(w, n, seed=7):
+    """Stratified sample of n requests of a full-size workload: the first and the last request,
+    one request from every block of 128 / G requests (the rows of one 128-row query tile of a
+    dense item, and the position inside a routed item's tiles varies with it), the rest spread
+    evenly over the batch with a seeded offset, so that no part of the batch, no tile of an item
+    and no stride of the persistent CTAs is left to luck."""
+    rng = np.random.default_rng(seed)
+    per_tile = max(1, 128 // w.G)
+    picks = {0, w.B - 1}
+    blocks = np.arange(0, w.B, per_tile)
+    for b0 in blocks[np.linspace(0, len(blocks) - 1, num=min(len(blocks), max(1, n - 2))).astype(int)]:
+        picks.add(int(min(w.B - 1, b0 + rng.integers(0, per_tile))))
+    picks = sorted(picks)
+    if len(picks) > n:  # keep the ends, thin the middle evenly
+        keep = np.unique(np.linspace(0, len(picks) - 1, num=n).astype(int))
+        picks = [picks[i] for i in keep]
+    return np.asarray(picks)
 
 
 def test_full_cfg1_sampled():
     w = W.CONFIGS[1]
-    run_case(w, sample=_sample(w, 6))
+    r = run_case(w, sample=_sample(w, 8))
+    assert r["routing_excused_rows"] == 0, r
 
 
 def test_full_cfg2_sampled():
     w = W.CONFIGS[2]
-    run_case(w, sample=_sample(w, 4), check_baseline=False)
+    r = run_case(w, sample=_sample(w, 8), check_baseline=False)
+    assert r["routing_excused_rows"] == 0, r
 
 
 def test_full_cfg3_dense_sampled():
     w = W.CONFIGS[3]
-    run_case(w, sample=_sample(w, 2), check_baseline=False)
+    run_case(w, sample=_sample(w, 8), check_baseline=False)
 
 
 def test_full_cfg4_sampled_steps():
@@ -330,7 +346,9 @@ def test_full_cfg4_sampled_steps():
     if free < 110e9:
         pytest.skip("not enough free device memory for the 71 GB ragged unique store")
     for step in (0, w.steps - 1):
-        run_case(w, sample=_sample(w, 3), check_baseline=False, step=step, two_streams=True)
+        r = run_case(w, sample=_sample(w, 6, seed=7 + step), check_baseline=False, step=step,
+                     two_streams=True)
+        assert r["routing_excused_rows"] == 0, r
         torch.cuda.empty_cache()
 
 
@@ -553,4 +571,46 @@ def test_decode_step_can_be_captured_in_a_cuda_graph():
         graph.replay()
         torch.cuda.synchronize()
         assert torch.equal(layer.out, eager)
+    assert M.device_status() == 0
+
+
+def test_grouping_reports_lists_that_break_its_precondition():
+    """The grouping works on one bit per (key, request), which only describes (request, KV head)
+    lists that are strictly ascending and inside [0, C).  Host-made lists that are out of range,
+    unsorted or hold a chunk twice must raise MOSKA_ERR_INVALID_ARG in the device status word,
+    through the workspace entry point and the allocation-free one, without a fault and without an
+    entry in seg_entries that is no valid position; a clean list afterwards reads status 0."""
+    M, MoskaLayer = _mods()
+    B, Hq, Hkv, D, C, L, k = 6, 8, 2, 128, 10, 128, 3
+    layer = MoskaLayer(B, Hq, Hkv, D, C, L, k, 16)
+    P = B * Hkv * k
+    good = np.tile(np.array([1, 4, 7], dtype=np.int32), (B, Hkv, 1))
+    bad = {
+        "out of range high": (2, 1, [1, 4, C]),
+        "negative": (0, 0, [-1, 4, 7]),
+        "unsorted": (3, 1, [7, 1, 4]),
+        "repeated": (5, 0, [4, 4, 7]),
+    }
+    for name, (b, h, lst) in bad.items():
+        for entry in ("workspace", "noalloc"):
+            t = good.copy()
+            t[b, h] = lst
+            layer.topk_idx.copy_(torch.from_numpy(t))
+            off = torch.full_like(layer.seg_offsets, -1)
+            ent = torch.full_like(layer.seg_entries, -1)
+            if entry == "workspace":
+                M.group_by_chunk(layer.topk_idx, off, ent, layer.shape, layer.ws)
+            else:
+                M.group_by_chunk_noalloc(layer.topk_idx, off, ent, layer.shape)
+            assert M.device_status() == M.ERR_INVALID_ARG, f"{name} / {entry}"
+            n = int(off[-1].item())
+            assert 0 <= n <= P
+            e = ent[:n].cpu().numpy()
+            assert ((e >= 0) & (e < P)).all(), f"{name} / {entry}: entry outside [0, P)"
+            if name == "unsorted":
+                # distinct chunks in any order still group correctly (the slot is found by a scan)
+                off_ref, ent_ref = O.group_by_chunk(t, C, fast=True)
+                assert np.array_equal(off.cpu().numpy(), off_ref) and np.array_equal(e, ent_ref)
+    layer.topk_idx.copy_(torch.from_numpy(good))
+    layer.group()
     assert M.device_status() == 0

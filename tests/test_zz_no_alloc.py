@@ -34,6 +34,45 @@ def test_noalloc_rejects_shapes_beyond_its_buffer_on_the_host():
 
 
 @pytest.mark.gpu
+def test_noalloc_wide_bit_sets_against_the_oracle_and_allocates_nothing():
+    """More than 64 requests (bit sets wider than two words take the separate counting pass) on a
+    shape whose scratch nearly fills the built-in buffer, compared with the CPU oracle's grouping
+    directly; the device's free memory must not move across a call."""
+    from oracle import oracle as O
+
+    M = _binding()
+    rng = np.random.default_rng(5)
+    B, Hq, Hkv, D, C, L, k = 300, 8, 8, 128, 12288, 128, 24
+    s = M.shape(B, Hq, Hkv, D, C, L, k)
+    # grouping scratch = the whole workspace minus the router's score array (C > 256)
+    scratch = M.workspace_bytes(s) - (4 * B * Hkv * C + 255) // 256 * 256
+    assert 0.8 * (8 << 20) < scratch <= (8 << 20), scratch
+    topk = np.empty((B, Hkv, k), dtype=np.int32)
+    # skewed: the low chunks are popular, so some segments hold most of the batch
+    p = 1.0 / np.arange(1, C + 1) ** 1.2
+    p /= p.sum()
+    for b in range(B):
+        for h in range(Hkv):
+            topk[b, h] = np.sort(rng.choice(C, size=k, replace=False, p=p))
+    t_dev = torch.from_numpy(topk).cuda()
+    off = torch.full((Hkv * C + 1,), -1, dtype=torch.int32, device="cuda")
+    ent = torch.full((B * Hkv * k,), -1, dtype=torch.int32, device="cuda")
+    M.group_by_chunk_noalloc(t_dev, off, ent, s)          # first call on the device: set-up
+    torch.cuda.synchronize()
+    free0, _ = torch.cuda.mem_get_info()
+    off.fill_(-1)
+    ent.fill_(-1)
+    M.group_by_chunk_noalloc(t_dev, off, ent, s)
+    torch.cuda.synchronize()
+    free1, _ = torch.cuda.mem_get_info()
+    assert free1 == free0, "the allocation-free call changed the device's free memory"
+    off_ref, ent_ref = O.group_by_chunk(topk, C, fast=True)
+    assert np.array_equal(off.cpu().numpy(), off_ref)
+    assert np.array_equal(ent.cpu().numpy(), ent_ref)
+    assert M.device_status() == 0
+
+
+@pytest.mark.gpu
 def test_noalloc_matches_regular_grouping_on_two_calls_in_a_row():
     M = _binding()
     from paper_2511_06010_b200.engine import MoskaLayer
