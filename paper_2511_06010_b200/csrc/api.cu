@@ -306,16 +306,16 @@ int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_
     const bool tc = shared_tc_supported(shape);
     if (dense) {
         // enough rows to fill a good part of a 128-row tile: tensor cores; else 16-row tiles
-        if (tc && (long long)shape->B * (shape->Hq / shape->Hkv) >= kBigMinRows)
+        if (tc && (long long)shape->B * (shape->Hq / shape->Hkv) >= kDenseTcMinRows)
             return launch_shared_tc(q, k_shared, v_shared, nullptr, o_part, lse_part, softmax_scale,
                                     shape, ws, true, 0, st);
         return launch_shared_small(q, k_shared, v_shared, nullptr, o_part, lse_part, softmax_scale,
                                    shape, ws, true, st);
     }
-    // routed: the grouping pass split every segment into tensor-core tiles and 16-row tiles
+    // routed: the grouping pass cut every segment into work items for the kernel that serves the shape
     if (tc)
-        MOSKA_TRY(launch_shared_tc(q, k_shared, v_shared, seg_entries, o_part, lse_part,
-                                   softmax_scale, shape, ws, false, 0, st));
+        return launch_shared_tc(q, k_shared, v_shared, seg_entries, o_part, lse_part, softmax_scale,
+                                shape, ws, false, 0, st);
     return launch_shared_small(q, k_shared, v_shared, seg_entries, o_part, lse_part, softmax_scale,
                                shape, ws, false, st);
 }
@@ -499,7 +499,7 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
         }
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 0, side));
         const bool tc = shared_tc_supported(shape) &&
-                        (!dense || (long long)shape->B * (shape->Hq / shape->Hkv) >= kBigMinRows);
+                        (!dense || (long long)shape->B * (shape->Hq / shape->Hkv) >= kDenseTcMinRows);
         // Sharing the SMs pays when unique attention runs long enough for the tensor-core kernel
         // to start beside it (the routing chain in front of it takes a few hundred microseconds
         // under contention); for a short unique attention the tensor-core items run after it, on
@@ -511,7 +511,7 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
             MOSKA_TRY(launch_shared_tc(q, k_shared, v_shared, dense ? nullptr : seg_entries, o_part,
                                        lse_part, softmax_scale, shape, ws, dense,
                                        tc_sm_share(shape, dense, unique_ms), side));
-        if (!dense || !tc)
+        if (!tc)
             MOSKA_TRY(launch_shared_small(q, k_shared, v_shared, dense ? nullptr : seg_entries, o_part,
                                           lse_part, softmax_scale, shape, ws, dense, side));
         if (beside || !tc) MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, side));

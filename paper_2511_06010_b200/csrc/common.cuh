@@ -56,8 +56,8 @@ struct TileItem {
 };
 
 struct WsHeader {
-    int32_t n_small_tiles;  // items in the small-tile list
-    int32_t n_big_tiles;    // items in the big-tile list
+    int32_t n_small_tiles;  // items in the second list: single-tile items (tensor-core shapes) or 16-row tiles
+    int32_t n_big_tiles;    // items of two 128-row query tiles
     int32_t reserved;
     int32_t n_tiny_tiles;   // items in the 8-row tile list
     int32_t pad[60];
@@ -70,7 +70,7 @@ struct WsLayout {
     int32_t small_entries;    // requests per small (16-row) tile
     int32_t tiny_entries;     // requests per 8-row tile
     int32_t big_entries;      // requests per big tile
-    int32_t big_min_entries;  // a remainder of at least this many requests still forms a big tile
+    int32_t tc;               // 1: the tensor-core kernel serves this shape (two-tile + single-tile items)
     int64_t max_small, max_big;
     size_t off_hist, off_totals, off_small, off_big, off_tiny;
     size_t group_total;  // end of what the grouping passes and shared attention use
@@ -81,11 +81,8 @@ WsLayout ws_layout(const moska_shape* s);
 
 constexpr int kRouteSmallC = 256;   // up to this many chunks the router keeps its scores in shared memory
 constexpr int kSmallTileRows = 16;  // query rows of one small tile (two 8-row MMA column blocks)
-constexpr int kBigTileRows = 128;   // query rows of one tensor-core (tcgen05) tile; a work item has two
-#ifndef MOSKA_BIG_MIN_ROWS
-#define MOSKA_BIG_MIN_ROWS 16
-#endif
-constexpr int kBigMinRows = MOSKA_BIG_MIN_ROWS;  // fewer leftover rows of a segment than this go to small tiles
+constexpr int kBigTileRows = 128;   // query rows of one tensor-core (tcgen05) tile; a work item has one or two
+constexpr int kDenseTcMinRows = 16; // dense mode: batches with fewer query rows per KV head take the streaming tiles
 
 // ---- internal launchers (one per .cu file) -----------------------------------------------------
 int launch_summaries(const uint16_t* k_shared, float* summaries, const moska_shape* s,

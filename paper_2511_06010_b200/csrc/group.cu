@@ -24,7 +24,7 @@ WsLayout ws_layout(const moska_shape* s)
     w.small_entries = kSmallTileRows / G;
     w.tiny_entries = 8 / G;  // requests whose rows fit one 8-row MMA column block (0: no such tiles)
     w.big_entries = 2 * (kBigTileRows / G);  // a tensor-core work item holds two 128-row tiles
-    w.big_min_entries = shared_tc_supported(s) ? (kBigMinRows + G - 1) / G : 0x7fffffff;
+    w.tc = shared_tc_supported(s) ? 1 : 0;
     const int64_t P = (int64_t)s->B * s->Hkv * s->k;
     const int64_t segs = P < w.n_keys ? P : w.n_keys;  // non-empty segments at most
     w.max_small = P / w.small_entries + segs;
@@ -82,15 +82,16 @@ group_count_kernel(const uint32_t* __restrict__ bitmap, int32_t* __restrict__ to
 }
 
 // Exclusive scans over the keys, one CTA: entries -> seg_offsets; tiles -> work lists.
-// A segment's requests go, in order, to tensor-core items (whole multiples of big_entries, and a
-// remainder of at least big_min_entries), then to 16-row tiles, and a last piece of at most
-// tiny_entries requests (8 rows) to the 8-row tile list.
+// Shapes the tensor-core kernel serves (tc): a segment's requests go, in order, to items of two
+// 128-row query tiles (big_entries requests; a remainder of more than one tile's requests still
+// forms one) and the rest, if any, to ONE single-tile item in the second list.  Other shapes: 16-row
+// tiles in the second list and a last piece of at most tiny_entries requests (8 rows) in the third.
 __global__ void __launch_bounds__(1024)
 group_scan_kernel(const uint32_t* __restrict__ bitmap, int words, const int32_t* __restrict__ totals,
                   int32_t* __restrict__ seg_offsets,
                   WsHeader* __restrict__ hdr, TileItem* __restrict__ small_items,
                   TileItem* __restrict__ tiny_items, TileItem* __restrict__ big_items, int n_keys,
-                  int small_entries, int tiny_entries, int big_entries, int big_min_entries)
+                  int small_entries, int tiny_entries, int big_entries, int tc)
 {
     __shared__ int4 warp_sum[32];
     __shared__ int4 carry;
@@ -111,21 +112,19 @@ group_scan_kernel(const uint32_t* __restrict__ bitmap, int words, const int32_t*
             else
                 for (int w = 0; w < words; ++w) n += __popc(bitmap[(size_t)key * words + w]);
         }
-        int n_big = n / big_entries;
-        int rem = n - n_big * big_entries;
-        if (rem >= big_min_entries) {
-            ++n_big;
-            rem = 0;
-        }
-        if (big_min_entries == 0x7fffffff) {
-            n_big = 0;
-            rem = n;
-        }
-        int n_small = rem / small_entries;
-        const int last = rem - n_small * small_entries;  // requests of the last, partial tile
-        int n_tiny = 0;
-        if (last > 0) {
-            if (last <= tiny_entries) n_tiny = 1; else ++n_small;
+        int n_big = 0, n_small = 0, n_tiny = 0;
+        int small_cap = small_entries;  // requests per item of the second list
+        if (tc) {
+            n_big = n / big_entries;
+            const int rem = n - n_big * big_entries;
+            small_cap = big_entries / 2;  // one 128-row query tile
+            if (rem > small_cap) ++n_big; else if (rem > 0) n_small = 1;
+        } else {
+            n_small = n / small_entries;
+            const int last = n - n_small * small_entries;  // requests of the last, partial tile
+            if (last > 0) {
+                if (last <= tiny_entries) n_tiny = 1; else ++n_small;
+            }
         }
         // x: entries, y: 16-row tiles, z: tensor-core items, w: 8-row tiles
         const int4 v = make_int4(n, n_small, n_big, n_tiny);
@@ -158,7 +157,7 @@ group_scan_kernel(const uint32_t* __restrict__ bitmap, int words, const int32_t*
                 e += cnt;
             }
             for (int t = 0; t < n_small; ++t) {
-                const int cnt = min(small_entries, ex.x + n - e);
+                const int cnt = min(small_cap, ex.x + n - e);
                 small_items[ex.y + t] = TileItem{key, e, cnt, 0};
                 e += cnt;
             }
@@ -258,7 +257,7 @@ int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_ent
     }
     group_scan_kernel<<<1, 1024, 0, st>>>(bitmap, lay.words, totals, seg_offsets, hdr, small_items, tiny_items, big_items,
                                           lay.n_keys, lay.small_entries, lay.tiny_entries,
-                                          lay.big_entries, lay.big_min_entries);
+                                          lay.big_entries, lay.tc);
     MOSKA_LAUNCH_CHECK("group_scan_kernel");
     group_emit_kernel<<<(lay.n_keys + 7) / 8, 256, 0, st>>>(topk_idx, bitmap, seg_offsets, seg_entries,
                                                             status, lay.n_keys, s->Hkv, s->C, s->k, lay.words);

@@ -35,10 +35,11 @@ constexpr int kD = 128;                        // head dimension this kernel is 
 constexpr int kKvTile = 128;                   // tokens per K/V tile
 constexpr int kTileBytes = 128 * kD * 2;       // one Q, K or V tile in shared memory
 constexpr int kHalfBytes = kTileBytes / 2;     // 64 head-dimension columns of a tile
+constexpr int kSubBytes = kTileBytes / 2;      // query sub-buffer for a tile of at most 64 rows
 constexpr int kStages = 4;                     // K/V ring slots
 constexpr int kThreads = 384;                  // 8 softmax warps, TMA warp, MMA warp, 2 gather warps
 constexpr int kLoadWarp = 8, kMmaWarp = 9, kGatherWarp0 = 10;
-constexpr int kSoftmaxRegs = 208, kOtherRegs = 80;  // per-thread register budgets after set-up
+constexpr int kSoftmaxRegs = 208, kOtherRegs = 96;  // per-thread register budgets after set-up
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.f;       // log2 units a row maximum may lag behind
@@ -47,7 +48,8 @@ struct __align__(1024) TcSmem {
     uint8_t q[2][kTileBytes];
     uint8_t kv[kStages][kTileBytes];
     uint64_t full[kStages], empty[kStages];
-    uint64_t q_full[2], q_free[2], s_full[2], p_full[2], o_full[2];
+    uint64_t q_full[2][2], q_free[2][2];  // [slot][sub-buffer]; a full tile signals / frees [.][0] (both)
+    uint64_t s_full[2], p_full[2], o_full[2];
     uint64_t x_full, x_free;      // split items: statistics of slot 1 published / O_1 read
     float stat_m[kBigTileRows];   // split items: running maximum and sum of slot 1's rows
     float stat_l[kBigTileRows];
@@ -59,7 +61,8 @@ struct TcParams {
     const uint16_t* q;
     const int32_t* seg_entries;
     const WsHeader* hdr;
-    const TileItem* items;
+    const TileItem* items;    // items of two query tiles (more than 128 rows)
+    const TileItem* singles;  // items of one query tile
     float* o_part;
     float* lse_part;
     int* status;
@@ -121,53 +124,116 @@ __device__ __forceinline__ float fmax3(float a, float b, float c)
     return d;
 }
 
-// One work item.  The CTA has two "slots" (t = 0, 1), each with its own S/P and O accumulator in
-// TMEM and its own softmax warp group.  An item with more than 128 rows runs its two query tiles
-// in the two slots over all K/V tiles.  An item with at most 128 rows is SPLIT: both slots hold
-// the same query tile, slot 0 takes the even and slot 1 the odd K/V tiles, and the two partial
-// softmax states are combined at the end -- so the tensor pipe always has two independent
-// dependency chains to alternate between.
-struct Item {
-    int h;            // KV head
-    int n_kv;         // K/V tiles of 128 tokens
-    int n_e[2];       // requests in query tile 0 / 1
-    int entry_begin;  // routed: first entry of the item in seg_entries
-    int b0;           // dense: first request of the item
-    int slot_dense;   // dense: partial slot (= run of chunks)
-    int split;        // 1: both slots work on query tile 0
-    int n_it[2];      // K/V tiles handled by slot 0 / 1
-    long long kv_row0;  // first token row of the item's K/V range in the [Hkv*C*L][D] store
+// One work unit of a CTA.  The CTA has two "slots" (t = 0, 1), each with its own S/P and O
+// accumulator in TMEM, its own softmax warp group and its own query buffer.  Three forms:
+//   two tiles  one item of more than 128 rows: its two query tiles run in the two slots over the
+//              same K/V tiles (one shared-memory copy serves both);
+//   pair       two different items of at most 128 rows each, one per slot, every slot over its own
+//              item's K/V tiles (which alternate in the ring) -- nothing is shared and nothing is
+//              merged, so one slot's epilogue and query gather run under the other slot's tiles;
+//   split      a single item of at most 128 rows: both slots hold the same query tile, slot 0 takes
+//              the even and slot 1 the odd K/V tiles, and the two partial softmax states are
+//              combined at the end.
+// In every form the tensor pipe has two independent dependency chains to alternate between.
+enum : int { kTwoTiles = 0, kSplit = 1, kPair = 2 };
+
+struct Unit {
+    int mode;
+    int n_kv;            // K/V tiles of 128 tokens of one item
+    int h[2];            // KV head of the item whose rows sit in slot t
+    int n_e[2];          // requests of that item's tile (split: slot 1 mirrors slot 0)
+    int entry_begin[2];  // routed: first entry of the tile in seg_entries
+    int b0[2];           // dense: first request of the tile
+    int slot_dense;      // dense: partial slot (= run of chunks)
+    int n_it[2];         // K/V tiles handled by slot 0 / 1
+    long long kv_row0[2];  // first token row of the slot's K/V range in the [Hkv*C*L][D] store
 };
 
-__device__ __forceinline__ Item decode_item(const TcParams& p, int item, int G, int per_tile)
+// Where the routed work lists end and how the single-tile items are scheduled on this grid: whole
+// rounds of pairs (two items per CTA and round), and the remaining fewer than 2 * grid items one per
+// unit in the split form, so that the last round still spreads over as many CTAs as it has items.
+struct Schedule {
+    int n_two, n_pairs, n_units;
+};
+
+__device__ __forceinline__ Schedule make_schedule(const TcParams& p)
 {
-    Item it;
+    Schedule s;
+    if (p.dense) {
+        s.n_two = p.n_items_dense;
+        s.n_pairs = 0;
+        s.n_units = p.n_items_dense;
+    } else {
+        s.n_two = p.hdr->n_big_tiles;
+        const int n1 = p.hdr->n_small_tiles;
+        s.n_pairs = (n1 / (2 * (int)gridDim.x)) * (int)gridDim.x;
+        s.n_units = s.n_two + s.n_pairs + (n1 - 2 * s.n_pairs);
+    }
+    return s;
+}
+
+__device__ __forceinline__ Unit decode_unit(const TcParams& p, const Schedule& sch, int unit, int G,
+                                            int per_tile)
+{
+    Unit it;
+    it.slot_dense = 0;
+    it.b0[0] = it.b0[1] = 0;
     if (!p.dense) {
-        const int4 raw = __ldg(reinterpret_cast<const int4*>(p.items) + item);  // TileItem
-        it.h = raw.x / p.C;
-        it.entry_begin = raw.y;
-        it.n_e[0] = min(raw.z, per_tile);
-        it.n_e[1] = min(raw.z - it.n_e[0], per_tile);
-        it.kv_row0 = (long long)raw.x * p.L;
         it.n_kv = p.L / kKvTile;
-        it.b0 = 0;
-        it.slot_dense = 0;
+        if (unit < sch.n_two) {
+            const int4 raw = __ldg(reinterpret_cast<const int4*>(p.items) + unit);  // TileItem
+            it.mode = kTwoTiles;
+            it.h[0] = it.h[1] = raw.x / p.C;
+            it.entry_begin[0] = raw.y;
+            it.entry_begin[1] = raw.y + per_tile;
+            it.n_e[0] = min(raw.z, per_tile);
+            it.n_e[1] = min(raw.z - it.n_e[0], per_tile);
+            it.kv_row0[0] = it.kv_row0[1] = (long long)raw.x * p.L;
+        } else if (unit < sch.n_two + sch.n_pairs) {
+            it.mode = kPair;
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                const int4 raw = __ldg(reinterpret_cast<const int4*>(p.singles) + 2 * (unit - sch.n_two) + t);
+                it.h[t] = raw.x / p.C;
+                it.entry_begin[t] = raw.y;
+                it.n_e[t] = min(raw.z, per_tile);
+                it.kv_row0[t] = (long long)raw.x * p.L;
+            }
+        } else {
+            const int4 raw = __ldg(reinterpret_cast<const int4*>(p.singles) + 2 * sch.n_pairs +
+                                   (unit - sch.n_two - sch.n_pairs));
+            it.mode = kSplit;
+            it.h[0] = it.h[1] = raw.x / p.C;
+            it.entry_begin[0] = it.entry_begin[1] = raw.y;
+            it.n_e[0] = it.n_e[1] = min(raw.z, per_tile);
+            it.kv_row0[0] = it.kv_row0[1] = (long long)raw.x * p.L;
+        }
     } else {
         const int b_tiles = (p.B + 2 * per_tile - 1) / (2 * per_tile);
-        const int bt = item % b_tiles;
-        it.slot_dense = (item / b_tiles) % p.shared_slots;
-        it.h = item / (b_tiles * p.shared_slots);
+        const int bt = unit % b_tiles;
+        it.slot_dense = (unit / b_tiles) % p.shared_slots;
+        it.h[0] = it.h[1] = unit / (b_tiles * p.shared_slots);
         const int run = (p.C + p.shared_slots - 1) / p.shared_slots;
         const int c0 = min(p.C, it.slot_dense * run), c1 = min(p.C, c0 + run);
-        it.b0 = bt * 2 * per_tile;
-        it.n_e[0] = min(per_tile, p.B - it.b0);
-        it.n_e[1] = max(0, min(per_tile, p.B - it.b0 - per_tile));
-        it.kv_row0 = ((long long)it.h * p.C + c0) * p.L;
+        it.b0[0] = bt * 2 * per_tile;
+        it.b0[1] = it.b0[0] + per_tile;
+        it.n_e[0] = min(per_tile, p.B - it.b0[0]);
+        it.n_e[1] = max(0, min(per_tile, p.B - it.b0[1]));
+        it.kv_row0[0] = it.kv_row0[1] = ((long long)it.h[0] * p.C + c0) * p.L;
         it.n_kv = (c1 - c0) * (p.L / kKvTile);
-        it.entry_begin = 0;
+        it.entry_begin[0] = it.entry_begin[1] = 0;
+        it.mode = kTwoTiles;
+        if (it.n_e[1] == 0 && it.n_kv >= 2) {
+            it.mode = kSplit;
+            it.n_e[1] = it.n_e[0];
+            it.b0[1] = it.b0[0];
+        }
     }
-    it.split = (it.n_e[1] == 0 && it.n_kv >= 2) ? 1 : 0;
-    if (it.split) {
+    if (it.mode == kSplit && it.n_kv < 2) {  // a single K/V tile cannot be divided: slot 0 alone
+        it.mode = kTwoTiles;
+        it.n_e[1] = 0;
+    }
+    if (it.mode == kSplit) {
         it.n_it[0] = (it.n_kv + 1) >> 1;
         it.n_it[1] = it.n_kv >> 1;
     } else {
@@ -177,22 +243,55 @@ __device__ __forceinline__ Item decode_item(const TcParams& p, int item, int G, 
     return it;
 }
 
+// a[t] for t in {0, 1} without indexing the array at run time (keeps it in registers)
+template <class T>
+__device__ __forceinline__ T pick(const T (&a)[2], int t)
+{
+    return t ? a[1] : a[0];
+}
+
+// Query buffers.  Slot u owns 32 KB: one full tile (two 64-column halves of 128 rows, 16 KB apart),
+// or two 16 KB sub-buffers for tiles of at most 64 rows (halves 8 KB apart).  The MMA always reads
+// 128 rows; behind a short tile it reads whatever follows in shared memory (the other sub-buffer,
+// the next slot's buffer, the start of the K/V ring) -- rows of the accumulator that no thread
+// looks at.  Consecutive short tiles of a slot alternate between the two sub-buffers, so the next
+// item's rows are gathered while the MMAs still read this item's.
+struct QUse {
+    bool present;  // the slot gathers a query tile of its own in this unit
+    bool small;    // at most 64 rows: one sub-buffer
+    int sub;       // sub-buffer (small), else 0
+};
+
+__device__ __forceinline__ QUse q_use(const Unit& it, int u, int G, uint32_t& n_small)
+{
+    QUse q;
+    q.present = it.n_kv > 0 && it.n_e[u] > 0 && !(it.mode == kSplit && u == 1);
+    q.small = it.n_e[u] * G <= 64;
+    q.sub = 0;
+    if (q.present && q.small) q.sub = (n_small++) & 1;
+    return q;
+}
+
 // Roles of the third warp group (after it has given registers up): TMA producer, MMA issuer and
 // the two query-gather warps.
 __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
-                                         const CUtensorMap& tm_q, const TcParams& p, int n_items, int G, int per_tile,
-                                         uint32_t tmem, int warp, int lane)
+                                         const CUtensorMap& tm_q, const TcParams& p, const Schedule& sch, int G,
+                                         int per_tile, uint32_t tmem, int warp, int lane)
 {
     volatile int* ab = &sm.abort_flag;
+    const int n_pos = p.B * p.Hkv * p.k;  // routed: valid entries of seg_entries are below this
 
     if (warp == kLoadWarp) {
-        // =========================== TMA producer: K_0, V_0, K_1, V_1, ... =======================
+        // =========================== TMA producer ================================================
+        // two tiles: K_0 V_0 K_1 V_1 ... of the item; split: the same; pair: the two items' tiles
+        // alternate, K_0 V_0 of slot 0's item, K_0 V_0 of slot 1's, K_1 V_1 of slot 0's, ...
         if (lane == 0) {
-            uint32_t ld = 0;  // loads issued so far, over all items
+            uint32_t ld = 0;  // loads issued so far, over all units
             bool ok = true;
-            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-                const Item it = decode_item(p, item, G, per_tile);
-                for (int x = 0; x < 2 * it.n_kv; ++x, ++ld) {
+            for (int unit = blockIdx.x; unit < sch.n_units && ok; unit += gridDim.x) {
+                const Unit it = decode_unit(p, sch, unit, G, per_tile);
+                const int n_loads = (it.mode == kPair ? 4 : 2) * it.n_kv;
+                for (int x = 0; x < n_loads; ++x, ++ld) {
                     const uint32_t s = ld % kStages;
                     if (ld >= kStages && !mbar_wait(&sm.empty[s], ((ld / kStages) - 1) & 1, ab)) {
                         ok = false;
@@ -200,7 +299,10 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
                     }
                     mbar_arrive_expect_tx(&sm.full[s], kTileBytes);
                     const CUtensorMap* tm = (x & 1) ? &tm_v : &tm_k;
-                    const int y = (int)(it.kv_row0 + (long long)(x >> 1) * kKvTile);
+                    const int vt = x >> 1;  // tile in ring order
+                    const int y = it.mode == kPair
+                        ? (int)(it.kv_row0[vt & 1] + (long long)(vt >> 1) * kKvTile)
+                        : (int)(it.kv_row0[0] + (long long)vt * kKvTile);
                     tma_load_2d(sm.kv[s], tm, 0, y, &sm.full[s]);
                     tma_load_2d(sm.kv[s] + kHalfBytes, tm, 64, y, &sm.full[s]);
                 }
@@ -214,18 +316,23 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
         }
         __syncwarp();
     } else if (warp >= kGatherWarp0) {
-        // =========================== query gather of tile u ======================================
+        // =========================== query gather of slot u ======================================
         // Brings the tile's query rows into the 128-byte-swizzled K-major operand layout as soon
-        // as the MMAs of the previous item have stopped reading the buffer: TMA row gathers, four
-        // rows per copy (lane l owns tile rows 4l .. 4l+3), so the copies do not queue behind the
-        // softmax groups' result stores in the load/store pipe.  Rows past the item's last one hold
+        // as the MMAs have stopped reading the (sub-)buffer: TMA row gathers, four rows per copy
+        // (lane l owns tile rows 4l .. 4l+3), so the copies do not queue behind the softmax
+        // groups' result stores in the load/store pipe.  Rows past the item's last one hold
         // stale or repeated query rows; their results are never written.
         const int u = warp - kGatherWarp0;
-        uint32_t uses = 0;
+        uint32_t n_small = 0;
+        uint32_t arrivals[2] = {0, 0};  // uses of sub-buffer 0 / 1 so far (a full tile uses both)
+        uint64_t* last_full = nullptr;  // barrier and phase of the last gather, for the abort path
+        uint32_t last_phase = 0;
+        uint32_t fills[2] = {0, 0};     // gathers signalled on q_full[u][0 / 1] so far
         bool ok = true;
-        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-            const Item it = decode_item(p, item, G, per_tile);
-            if (it.n_kv == 0 || it.n_e[u] == 0) continue;
+        for (int unit = blockIdx.x; unit < sch.n_units && ok; unit += gridDim.x) {
+            const Unit it = decode_unit(p, sch, unit, G, per_tile);
+            const QUse qu = q_use(it, u, G, n_small);
+            if (!qu.present) continue;
             int rr[4];  // global query rows of tile rows 4 * lane .. 4 * lane + 3
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
@@ -234,33 +341,43 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
                 if (i < it.n_e[u] * G) {
                     const int e = i / G, g = i % G;
                     int b;
-                    if (!p.dense)
-                        b = __ldg(p.seg_entries + it.entry_begin + u * per_tile + e) / (p.k * p.Hkv);
-                    else
-                        b = it.b0 + u * per_tile + e;
-                    rr[m] = b * p.Hq + it.h * G + g;
+                    if (!p.dense) {
+                        const int pp = __ldg(p.seg_entries + it.entry_begin[u] + e);
+                        b = (unsigned)pp < (unsigned)n_pos ? pp / (p.k * p.Hkv) : 0;
+                    } else {
+                        b = it.b0[u] + e;
+                    }
+                    rr[m] = b * p.Hq + it.h[u] * G + g;
                 }
             }
-            if (uses > 0) {
-                ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_free[u], (uses - 1) & 1, ab));
-                if (!ok) break;
+            // the MMAs that read what is about to be overwritten must have completed
+#pragma unroll
+            for (int sb = 0; sb < 2; ++sb) {
+                if (qu.small && sb != qu.sub) continue;
+                if (arrivals[sb] > 0 && ok)
+                    ok = __all_sync(0xffffffffu, mbar_wait(&sm.q_free[u][sb], (arrivals[sb] - 1) & 1, ab));
+                ++arrivals[sb];
             }
-            ++uses;
+            if (!ok) break;
+            uint64_t* bar = &sm.q_full[u][qu.sub];
+            last_full = bar;
+            last_phase = fills[qu.sub]++ & 1;
             // only the groups of four rows that hold a query row are copied; the tile rows after
             // them keep whatever an earlier item left there
             const int n_groups = (it.n_e[u] * G + 3) >> 2;
-            if (lane == 0) mbar_arrive_expect_tx(&sm.q_full[u], n_groups * 2 * (4 * 128));
+            if (lane == 0) mbar_arrive_expect_tx(bar, n_groups * 2 * (4 * 128));
             __syncwarp();
             if (lane < n_groups) {
-                uint8_t* dst = sm.q[u] + lane * (4 * 128);
-                tma_gather4_2d(dst, &tm_q, 0, rr[0], rr[1], rr[2], rr[3], &sm.q_full[u]);
-                tma_gather4_2d(dst + kHalfBytes, &tm_q, 64, rr[0], rr[1], rr[2], rr[3], &sm.q_full[u]);
+                uint8_t* dst = sm.q[u] + (qu.small ? qu.sub * kSubBytes : 0) + lane * (4 * 128);
+                const int half = qu.small ? kSubBytes / 2 : kHalfBytes;
+                tma_gather4_2d(dst, &tm_q, 0, rr[0], rr[1], rr[2], rr[3], bar);
+                tma_gather4_2d(dst + half, &tm_q, 64, rr[0], rr[1], rr[2], rr[3], bar);
             }
         }
-        if (*ab && uses > 0) {
+        if (*ab && last_full != nullptr) {
             // giving up: let the copies still in flight land before the CTA leaves
             volatile int never = 0;
-            mbar_wait(&sm.q_full[u], (uses - 1) & 1, &never);
+            mbar_wait(last_full, last_phase, &never);
         }
     } else {
         // =========================== MMA issuer ===================================================
@@ -278,13 +395,15 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
             const uint32_t lo_k = static_cast<uint32_t>(d_kmajor) + (smem_u32(sm.kv[0]) >> 4);
             const uint32_t lo_v = static_cast<uint32_t>(d_nmajor) + (smem_u32(sm.kv[0]) >> 4);
             auto desc = [](uint32_t hi, uint32_t lo) { return (static_cast<uint64_t>(hi) << 32) | lo; };
-            // S_t = Q_u K^T, K in ring slot s: 8 steps of 16 head-dimension columns
-            auto issue_qk = [&](int tq, int u, uint32_t s) {
-                const uint32_t a = lo_q + u * (kTileBytes >> 4), b = lo_k + s * (kTileBytes >> 4);
+            // S_t = Q K^T, Q at descriptor address qa with its halves qh apart, K in ring slot s:
+            // 8 steps of 16 head-dimension columns
+            auto issue_qk = [&](int tq, uint32_t qa, uint32_t qh, uint32_t s) {
+                const uint32_t b = lo_k + s * (kTileBytes >> 4);
 #pragma unroll
                 for (int ks = 0; ks < kD / 16; ++ks) {
-                    const uint32_t off = ((ks >> 2) * kHalfBytes + (ks & 3) * 32) >> 4;
-                    mma_ss(tmem + tq * 128, desc(hi_k, a + off), desc(hi_k, b + off), id_qk, ks > 0);
+                    const uint32_t sub = ((ks & 3) * 32) >> 4;
+                    mma_ss(tmem + tq * 128, desc(hi_k, qa + (ks >> 2) * qh + sub),
+                           desc(hi_k, b + (((ks >> 2) * kHalfBytes) >> 4) + sub), id_qk, ks > 0);
                 }
             };
             // O_t += P_t V, V in ring slot s: 8 steps of 16 tokens
@@ -295,45 +414,64 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
                     mma_ts(tmem + 256 + tq * 128, tmem + tq * 128 + ks * 8,
                            desc(hi_n, b + ks * (2048 >> 4)), id_pv, acc || ks > 0);
             };
-            uint32_t ld0 = 0;               // ring position of the item's first load
-            uint32_t qc[2] = {0, 0}, pc[2] = {0, 0};
-            int q_reads[2] = {0, 0};        // score MMAs of the item that still have to read q[u]
-            auto issue_scores = [&](const Item& it, int tq, uint32_t s) {
-                const int u = it.split ? 0 : tq;
-                issue_qk(tq, u, s);
-                tc_commit(&sm.s_full[tq]);
-                if (--q_reads[u] == 0) tc_commit(&sm.q_free[u]);  // the gather warp may refill q[u]
-            };
+            uint32_t ld0 = 0;               // ring position of the unit's first load
+            uint32_t pc[2] = {0, 0};
+            uint32_t n_small[2] = {0, 0}, fills[2][2] = {{0, 0}, {0, 0}};
+            int q_reads[2] = {0, 0};        // score MMAs of the unit that still have to read q[u]
             bool ok = true;
-            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-                const Item it = decode_item(p, item, G, per_tile);
-                // K/V tile of slot tq's x-th step, and whether that slot is the tile's last reader
-                auto tile_of = [&](int tq, int x) { return it.split ? 2 * x + tq : x; };
-                auto last_reader = [&](int tq) { return it.split || it.n_it[1] == 0 || tq == 1; };
+            for (int unit = blockIdx.x; unit < sch.n_units && ok; unit += gridDim.x) {
+                const Unit it = decode_unit(p, sch, unit, G, per_tile);
+                QUse qu[2];
+                uint32_t qa[2], qh[2];
+                for (int u = 0; u < 2; ++u) {
+                    qu[u] = q_use(it, u, G, n_small[u]);
+                    qa[u] = lo_q + ((u * kTileBytes + (qu[u].small ? qu[u].sub * kSubBytes : 0)) >> 4);
+                    qh[u] = (qu[u].small ? kSubBytes / 2 : kHalfBytes) >> 4;
+                }
+                // ring position of the K tile of slot tq's x-th step (its V tile is the next one),
+                // and whether that slot is the tile's last reader
+                auto k_load = [&](int tq, int x) {
+                    return ld0 + 2 * (it.mode == kTwoTiles ? x : 2 * x + tq);
+                };
+                auto last_reader = [&](int tq) {
+                    return it.mode != kTwoTiles || it.n_it[1] == 0 || tq == 1;
+                };
                 auto wait_load = [&](uint32_t g) {
                     return mbar_wait(&sm.full[g % kStages], (g / kStages) & 1, ab);
                 };
-                q_reads[0] = it.n_kv;
-                q_reads[1] = it.n_e[1] > 0 ? it.n_kv : 0;
+                auto issue_scores = [&](int tq, uint32_t s) {
+                    const int u = it.mode == kSplit ? 0 : tq;
+                    issue_qk(tq, qa[u], qh[u], s);
+                    tc_commit(&sm.s_full[tq]);
+                    if (--q_reads[u] == 0) {  // the gather warp may refill the (sub-)buffer
+                        if (qu[u].small) {
+                            tc_commit(&sm.q_free[u][qu[u].sub]);
+                        } else {
+                            tc_commit(&sm.q_free[u][0]);
+                            tc_commit(&sm.q_free[u][1]);
+                        }
+                    }
+                };
+                q_reads[0] = it.mode == kSplit ? it.n_kv : it.n_it[0];
+                q_reads[1] = it.mode == kSplit ? 0 : it.n_it[1];
                 for (int u = 0; u < 2 && ok; ++u) {
-                    if (it.n_kv == 0 || it.n_e[u] == 0) continue;
-                    ok = mbar_wait(&sm.q_full[u], qc[u] & 1, ab);
-                    ++qc[u];
+                    if (!qu[u].present) continue;
+                    ok = mbar_wait(&sm.q_full[u][qu[u].sub], fills[u][qu[u].sub]++ & 1, ab);
                 }
                 // first scores of both slots
                 for (int tq = 0; tq < 2 && ok; ++tq) {
                     if (it.n_it[tq] == 0) continue;
-                    const uint32_t g = ld0 + 2 * tile_of(tq, 0);
+                    const uint32_t g = k_load(tq, 0);
                     ok = wait_load(g);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    issue_scores(it, tq, g % kStages);
+                    issue_scores(tq, g % kStages);
                     if (last_reader(tq)) tc_commit(&sm.empty[g % kStages]);
                 }
                 for (int x = 0; x < it.n_it[0] && ok; ++x) {
                     for (int tq = 0; tq < 2 && ok; ++tq) {
                         if (x >= it.n_it[tq]) continue;
-                        const uint32_t gv = ld0 + 2 * tile_of(tq, x) + 1;
+                        const uint32_t gv = k_load(tq, x) + 1;
                         ok = wait_load(gv) && mbar_wait(&sm.p_full[tq], pc[tq] & 1, ab);
                         if (!ok) break;
                         ++pc[tq];
@@ -341,23 +479,22 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
                         issue_pv(tq, gv % kStages, x > 0);
                         if (last_reader(tq)) tc_commit(&sm.empty[gv % kStages]);
                         if (x + 1 < it.n_it[tq]) {
-                            const uint32_t gk = ld0 + 2 * tile_of(tq, x + 1);
+                            const uint32_t gk = k_load(tq, x + 1);
                             ok = wait_load(gk);
                             if (!ok) break;
                             tc_fence_after_sync();
-                            issue_scores(it, tq, gk % kStages);
+                            issue_scores(tq, gk % kStages);
                             if (last_reader(tq)) tc_commit(&sm.empty[gk % kStages]);
                         } else {
                             tc_commit(&sm.o_full[tq]);
                         }
                     }
                 }
-                ld0 += 2 * it.n_kv;
+                ld0 += (it.mode == kPair ? 4 : 2) * it.n_kv;
             }
         }
         __syncwarp();
     }
-
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -370,8 +507,8 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = p.Hq / p.Hkv;
     const int per_tile = kBigTileRows / G;  // requests per query tile
-    const int n_items = p.dense ? p.n_items_dense : p.hdr->n_big_tiles;
-    if ((int)blockIdx.x >= n_items) return;
+    const Schedule sch = make_schedule(p);
+    if ((int)blockIdx.x >= sch.n_units) return;
 
     // ---- set-up: barriers, tensor memory --------------------------------------------------------
     if (tid == 0) {
@@ -380,8 +517,10 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             mbar_init(&sm.empty[s], 1);
         }
         for (int u = 0; u < 2; ++u) {
-            mbar_init(&sm.q_full[u], 1);
-            mbar_init(&sm.q_free[u], 1);
+            for (int sb = 0; sb < 2; ++sb) {
+                mbar_init(&sm.q_full[u][sb], 1);
+                mbar_init(&sm.q_free[u][sb], 1);
+            }
             mbar_init(&sm.s_full[u], 1);
             mbar_init(&sm.p_full[u], 128);
             mbar_init(&sm.o_full[u], 1);
@@ -417,30 +556,39 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         const uint32_t t_o = tmem + lane_sel + 256 + t * 128;  // O_t
         const uint32_t t_o_other = tmem + lane_sel + 256 + (1 - t) * 128;
         const float sl2 = p.scale * kLog2e;
-        uint32_t sc = 0, oc[2] = {0, 0}, xc = 0;  // barrier phases completed before this item
+        const int n_pos = p.B * p.Hkv * p.k;
+        uint32_t sc = 0, oc[2] = {0, 0}, xc = 0;  // barrier phases completed before this unit
         bool alive = true;
-        for (int item = blockIdx.x; item < n_items && alive; item += gridDim.x) {
-            const Item it = decode_item(p, item, G, per_tile);
-            const int n_it = it.n_it[t];
-            const int src = it.split ? 0 : t;  // query tile whose rows sit on this group's lanes
+        for (int unit = blockIdx.x; unit < sch.n_units && alive; unit += gridDim.x) {
+            const Unit it = decode_unit(p, sch, unit, G, per_tile);
+            const int n_it = pick(it.n_it, t);
+            const bool split = it.mode == kSplit;
             const uint32_t ph_o[2] = {oc[0] & 1u, oc[1] & 1u}, ph_x = xc & 1u;
             oc[0] += it.n_it[0] > 0;
             oc[1] += it.n_it[1] > 0;
-            xc += it.split;
+            xc += split;
+            const int n_rows = pick(it.n_e, t) * G;
+            // a warp none of whose rows exists skips the arithmetic (every row of the products
+            // depends on its own query row only), but keeps every barrier in step
+            const bool warp_live = (warp & 3) * 32 < n_rows;
             long long my_r = -1;
             int my_slot = 0;
-            if (i < it.n_e[src] * G) {
+            if (i < n_rows) {
                 const int e = i / G, g = i % G;
-                int b;
+                int b = -1;
                 if (!p.dense) {
-                    const int pp = __ldg(p.seg_entries + it.entry_begin + src * per_tile + e);
-                    my_slot = pp % p.k;
-                    b = pp / (p.k * p.Hkv);
+                    const int pp = __ldg(p.seg_entries + pick(it.entry_begin, t) + e);
+                    if ((unsigned)pp < (unsigned)n_pos) {
+                        my_slot = pp % p.k;
+                        b = pp / (p.k * p.Hkv);
+                    } else {
+                        atomicMin(p.status, (int)MOSKA_ERR_INVALID_ARG);  // not a position of this batch
+                    }
                 } else {
                     my_slot = it.slot_dense;
-                    b = it.b0 + src * per_tile + e;
+                    b = pick(it.b0, t) + e;
                 }
-                my_r = (long long)b * p.Hq + it.h * G + g;
+                if (b >= 0) my_r = (long long)b * p.Hq + pick(it.h, t) * G + g;
             }
             if (it.n_kv == 0) {  // dense mode: a trailing run without chunks
                 if (my_r >= 0) {
@@ -455,78 +603,81 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 alive = __all_sync(0xffffffffu, mbar_wait(&sm.s_full[t], sc & 1, ab));
                 if (!alive) break;
                 ++sc;
-                tc_fence_after_sync();
-                // the row's 128 scores: four loads in flight, one wait
-                uint32_t r[4][32];
+                if (warp_live) {
+                    tc_fence_after_sync();
+                    // the row's 128 scores: four loads in flight, one wait
+                    uint32_t r[4][32];
 #pragma unroll
-                for (int c = 0; c < 4; ++c) tmem_ld32(t_s + c * 32, r[c]);
-                tmem_ld_wait();
-                // eight independent maximum chains of three-input maxima, then a tree
-                float mxs[8];
+                    for (int c = 0; c < 4; ++c) tmem_ld32(t_s + c * 32, r[c]);
+                    tmem_ld_wait();
+                    // eight independent maximum chains of three-input maxima, then a tree
+                    float mxs[8];
 #pragma unroll
-                for (int x = 0; x < 8; ++x)
-                    mxs[x] = fmaxf(__uint_as_float(r[0][2 * x]), __uint_as_float(r[0][2 * x + 1]));
+                    for (int x = 0; x < 8; ++x)
+                        mxs[x] = fmaxf(__uint_as_float(r[0][2 * x]), __uint_as_float(r[0][2 * x + 1]));
 #pragma unroll
-                for (int x = 8; x < 16; ++x)
-                    mxs[x & 7] = fmax3(mxs[x & 7], __uint_as_float(r[0][2 * x]), __uint_as_float(r[0][2 * x + 1]));
+                    for (int x = 8; x < 16; ++x)
+                        mxs[x & 7] = fmax3(mxs[x & 7], __uint_as_float(r[0][2 * x]), __uint_as_float(r[0][2 * x + 1]));
 #pragma unroll
-                for (int c = 1; c < 4; ++c)
+                    for (int c = 1; c < 4; ++c)
 #pragma unroll
-                    for (int x = 0; x < 16; ++x)
-                        mxs[x & 7] = fmax3(mxs[x & 7], __uint_as_float(r[c][2 * x]), __uint_as_float(r[c][2 * x + 1]));
-                const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
-                                       fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
-                if (j == 0) {
-                    m_ref = mx;
-                } else {
-                    const bool need = (mx - m_ref) * sl2 > kRescaleThreshold;
-                    if (__any_sync(0xffffffffu, need)) {
-                        // every MMA issued before S_t(j), PV_t(j-1) included, has completed
-                        const float alpha = need ? fast_exp2((m_ref - mx) * sl2) : 1.f;
-                        if (need) m_ref = mx;
-                        l_sum *= alpha;
+                        for (int x = 0; x < 16; ++x)
+                            mxs[x & 7] = fmax3(mxs[x & 7], __uint_as_float(r[c][2 * x]), __uint_as_float(r[c][2 * x + 1]));
+                    const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
+                                           fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
+                    if (j == 0) {
+                        m_ref = mx;
+                    } else {
+                        // rows that do not exist hold arbitrary bits: they never ask for a rescale
+                        const bool need = i < n_rows && (mx - m_ref) * sl2 > kRescaleThreshold;
+                        if (__any_sync(0xffffffffu, need)) {
+                            // every MMA issued before S_t(j), PV_t(j-1) included, has completed
+                            const float alpha = need ? fast_exp2((m_ref - mx) * sl2) : 1.f;
+                            if (need) m_ref = mx;
+                            l_sum *= alpha;
 #pragma unroll 1
-                        for (int c = 0; c < 4; ++c) {
-                            uint32_t o_acc[32];
-                            tmem_ld32(t_o + c * 32, o_acc);
-                            tmem_ld_wait();
+                            for (int c = 0; c < 4; ++c) {
+                                uint32_t o_acc[32];
+                                tmem_ld32(t_o + c * 32, o_acc);
+                                tmem_ld_wait();
 #pragma unroll
-                            for (int x = 0; x < 32; ++x)
-                                o_acc[x] = __float_as_uint(__uint_as_float(o_acc[x]) * alpha);
-                            tmem_st32(t_o + c * 32, o_acc);
+                                for (int x = 0; x < 32; ++x)
+                                    o_acc[x] = __float_as_uint(__uint_as_float(o_acc[x]) * alpha);
+                                tmem_st32(t_o + c * 32, o_acc);
+                            }
                         }
                     }
-                }
-                // P = exp2((S - m_ref) * scale * log2 e) as bf16, written over the columns of S
-                const float2 sl2_2 = make_float2(sl2, sl2);
-                const float2 nmb_2 = make_float2(-m_ref * sl2, -m_ref * sl2);
-                float2 ls[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};  // partial row sums
+                    // P = exp2((S - m_ref) * scale * log2 e) as bf16, written over the columns of S
+                    const float2 sl2_2 = make_float2(sl2, sl2);
+                    const float2 nmb_2 = make_float2(-m_ref * sl2, -m_ref * sl2);
+                    float2 ls[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};  // partial row sums
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    uint32_t pk[16];
+                    for (int c = 0; c < 4; ++c) {
+                        uint32_t pk[16];
 #pragma unroll
-                    for (int x = 0; x < 16; ++x) {
-                        const float2 e = ffma2(make_float2(__uint_as_float(r[c][2 * x]),
-                                                           __uint_as_float(r[c][2 * x + 1])),
-                                               sl2_2, nmb_2);
-                        float2 pr;
-                        pr.x = fast_exp2(e.x);
-                        pr.y = fast_exp2(e.y);
-                        ls[x & 1] = fadd2(ls[x & 1], pr);
-                        __nv_bfloat162 b2 = __floats2bfloat162_rn(pr.x, pr.y);
-                        pk[x] = *reinterpret_cast<uint32_t*>(&b2);
+                        for (int x = 0; x < 16; ++x) {
+                            const float2 e = ffma2(make_float2(__uint_as_float(r[c][2 * x]),
+                                                               __uint_as_float(r[c][2 * x + 1])),
+                                                   sl2_2, nmb_2);
+                            float2 pr;
+                            pr.x = fast_exp2(e.x);
+                            pr.y = fast_exp2(e.y);
+                            ls[x & 1] = fadd2(ls[x & 1], pr);
+                            __nv_bfloat162 b2 = __floats2bfloat162_rn(pr.x, pr.y);
+                            pk[x] = *reinterpret_cast<uint32_t*>(&b2);
+                        }
+                        tmem_st16(t_s + c * 16, pk);
                     }
-                    tmem_st16(t_s + c * 16, pk);
+                    l_sum += (ls[0].x + ls[0].y) + (ls[1].x + ls[1].y);
+                    tmem_st_wait();
                 }
-                l_sum += (ls[0].x + ls[0].y) + (ls[1].x + ls[1].y);
-                tmem_st_wait();
                 tc_fence_before_sync();
                 mbar_arrive(&sm.p_full[t]);
             }
             if (!alive) break;
 
             // ---- epilogue: normalised partial output and log-sum-exp of the row -----------------
-            if (it.split && t == 1) {
+            if (split && t == 1) {
                 // publish this slot's statistics; slot 0's group combines and writes
                 sm.stat_m[i] = m_ref;
                 sm.stat_l[i] = l_sum;
@@ -534,11 +685,11 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 alive = __all_sync(0xffffffffu, mbar_wait(&sm.x_free, ph_x, ab));
                 continue;
             }
-            if (n_it == 0) continue;  // slot 1 of an item with a single tile and a single K/V tile
+            if (n_it == 0) continue;  // slot 1 of a unit with a single tile and a single K/V tile
             alive = __all_sync(0xffffffffu, mbar_wait(&sm.o_full[t], ph_o[t], ab));
             if (!alive) break;
             float a_mine = 1.f, a_other = 0.f, m_all = m_ref, den = l_sum;
-            if (it.split) {
+            if (split) {
                 alive = __all_sync(0xffffffffu, mbar_wait(&sm.o_full[1], ph_o[1], ab)) &&
                         __all_sync(0xffffffffu, mbar_wait(&sm.x_full, ph_x, ab));
                 if (!alive) break;
@@ -548,16 +699,16 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 a_other = fast_exp2((m1 - m_all) * sl2);
                 den = a_mine * l_sum + a_other * l1;
             }
-            tc_fence_after_sync();
-            const float inv = 1.f / den;
-            a_mine *= inv;
-            a_other *= inv;
-            float4* o = my_r >= 0
-                ? reinterpret_cast<float4*>(p.o_part + (my_r * p.n_slots + my_slot) * kD)
-                : nullptr;
-            // the whole accumulator row: four loads in flight, one wait (two rounds when a second
-            // accumulator has to be folded in)
-            {
+            if (warp_live) {
+                tc_fence_after_sync();
+                const float inv = 1.f / den;
+                a_mine *= inv;
+                a_other *= inv;
+                float4* o = my_r >= 0
+                    ? reinterpret_cast<float4*>(p.o_part + (my_r * p.n_slots + my_slot) * kD)
+                    : nullptr;
+                // the whole accumulator row: four loads in flight, one wait (two rounds when a
+                // second accumulator has to be folded in)
                 uint32_t r[4][32];
 #pragma unroll
                 for (int c = 0; c < 4; ++c) tmem_ld32(t_o + c * 32, r[c]);
@@ -566,7 +717,7 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 for (int c = 0; c < 4; ++c)
 #pragma unroll
                     for (int x = 0; x < 32; ++x) r[c][x] = __float_as_uint(__uint_as_float(r[c][x]) * a_mine);
-                if (it.split) {
+                if (split) {
 #pragma unroll
                     for (int hv = 0; hv < 2; ++hv) {
                         uint32_t r2[2][32];
@@ -589,17 +740,17 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         for (int x = 0; x < 4; ++x)
                             st_global_v8(reinterpret_cast<float*>(o) + c * 32 + x * 8,
                                          reinterpret_cast<const float*>(&r[c][8 * x]));
+                    p.lse_part[my_r * p.n_slots + my_slot] = m_all * p.scale + logf(den);
                 }
             }
-            if (my_r >= 0) p.lse_part[my_r * p.n_slots + my_slot] = m_all * p.scale + logf(den);
-            if (it.split) {
+            if (split) {
                 tc_fence_before_sync();
                 mbar_arrive(&sm.x_free);  // O_1 and the statistics may be overwritten
             }
         }
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
-        other_roles(sm, tm_k, tm_v, tm_q, p, n_items, G, per_tile, tmem, warp, lane);
+        other_roles(sm, tm_k, tm_v, tm_q, p, sch, G, per_tile, tmem, warp, lane);
     }
 
     // ---- teardown -------------------------------------------------------------------------------
@@ -684,9 +835,10 @@ int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t
         p.n_items_dense = (int)grid;
     } else {
         const WsLayout lay = ws_layout(s);
-        grid = lay.max_big;
+        grid = lay.max_big + lay.max_small;
         p.hdr = reinterpret_cast<const WsHeader*>(ws);
         p.items = reinterpret_cast<const TileItem*>(static_cast<const char*>(ws) + lay.off_big);
+        p.singles = reinterpret_cast<const TileItem*>(static_cast<const char*>(ws) + lay.off_small);
     }
     if (grid == 0) return MOSKA_OK;
     if (grid > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "shared attention grid too large");
