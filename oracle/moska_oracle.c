@@ -62,6 +62,48 @@ void oracle_chunk_summaries(const uint16_t* k_shared, double* summaries, int Hkv
 }
 
 /*
+ * Second training-free chunk embedding behind the same summaries buffer (Section II-B and III-B
+ * cite two routers; the first pools a chunk's keys uniformly, which is the mean above; the
+ * second weights a chunk's tokens by an attention pass inside the chunk).  The reading taken
+ * here: the chunk's mean key kbar probes the chunk's own keys,
+ *     w_t = softmax_t( scale * <kbar, k_t> ),   summary = sum_t w_t k_t,
+ * i.e. one softmax-attention row with query kbar and the chunk's keys as both keys and values.
+ * scale = 0 gives uniform weights, hence the mean.
+ *   k_shared [Hkv][C][L][D] bf16 bits  ->  summaries [Hkv][C][D] double
+ */
+void oracle_chunk_summaries_attn(const uint16_t* k_shared, double* summaries, double scale,
+                                 int Hkv, int C, int L, int D)
+{
+#pragma omp parallel for schedule(static)
+    for (long hc = 0; hc < (long)Hkv * C; ++hc) {
+        double* kbar = (double*)malloc(sizeof(double) * D);
+        double* s = (double*)malloc(sizeof(double) * L);
+        for (int d = 0; d < D; ++d) {
+            double acc = 0.0;
+            for (int t = 0; t < L; ++t) acc += bf16_to_double(k_shared[(hc * L + t) * D + d]);
+            kbar[d] = acc / (double)L;
+        }
+        double smax = -INFINITY;
+        for (int t = 0; t < L; ++t) {
+            double acc = 0.0;
+            for (int d = 0; d < D; ++d) acc += kbar[d] * bf16_to_double(k_shared[(hc * L + t) * D + d]);
+            s[t] = scale * acc;
+            if (s[t] > smax) smax = s[t];
+        }
+        double den = 0.0;
+        for (int t = 0; t < L; ++t) den += exp(s[t] - smax);
+        for (int d = 0; d < D; ++d) {
+            double acc = 0.0;
+            for (int t = 0; t < L; ++t)
+                acc += exp(s[t] - smax) * bf16_to_double(k_shared[(hc * L + t) * D + d]);
+            summaries[hc * D + d] = acc / den;
+        }
+        free(kbar);
+        free(s);
+    }
+}
+
+/*
  * Router (Section III-B): score[b][h][c] = <sum_g q[b][h*G+g], summaries[h][c]>; the k chunks
  * of largest score are kept, exact ties going to the lower chunk index; the selected indices
  * are returned in ascending chunk order.  Selection is exhaustive: k passes, each taking the

@@ -80,6 +80,15 @@ def chunk_summaries(k_shared) -> np.ndarray:
     return out
 
 
+def chunk_summaries_attn(k_shared, scale: float) -> np.ndarray:
+    """Attention-pooled chunk embedding: softmax(scale * <mean key, k_t>)-weighted mean of the keys."""
+    Hkv, C, L, D = k_shared.shape
+    kb = _bits(k_shared)
+    out = np.empty((Hkv, C, D), dtype=np.float64)
+    _load().oracle_chunk_summaries_attn(_p(kb), _p(out), ctypes.c_double(scale), Hkv, C, L, D)
+    return out
+
+
 def route(q, summaries, k: int, return_all: bool = False):
     """-> (topk_idx int32 [B][Hkv][k] ascending, topk_score f64 [B][Hkv][k][, scores_all])."""
     B, Hq, D = q.shape

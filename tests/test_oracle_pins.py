@@ -96,6 +96,55 @@ def test_summaries_match_numpy_mean_and_indexing():
     assert abs(s[1, 2, 3] - sum(float(ks[1, 2, t, 3]) for t in range(8)) / 8) < 1e-15
 
 
+def test_attention_pooled_summaries_pins():
+    """The second chunk embedding: softmax(scale <mean key, k_t>)-weighted mean of the keys.
+    Pinned by (1) the library's attention routine with the mean key as the query and the chunk's
+    keys as keys AND values, (2) plain loops, (3) scale = 0 -> the arithmetic mean, (4) identical
+    keys -> that key, (5) one key far along the mean's direction takes all the weight, (6) the
+    order of the tokens inside a chunk does not matter, a change of one chunk leaves the others."""
+    g = torch.Generator().manual_seed(3)
+    Hkv, C, L, D = 2, 3, 8, 4
+    ks = torch.randn(Hkv, C, L, D, generator=g).to(torch.bfloat16)
+    scale = 0.7
+    s = O.chunk_summaries_attn(ks, scale)
+    assert s.shape == (Hkv, C, D)
+    K = ks.to(torch.float64)
+    kbar = K.mean(dim=2, keepdim=True)                                  # [Hkv][C][1][D]
+    ref = torch.nn.functional.scaled_dot_product_attention(kbar, K, K, scale=scale)[:, :, 0]
+    np.testing.assert_allclose(s, ref.numpy(), rtol=0, atol=1e-13)
+    # plain loops for one chunk: a swapped head/chunk index or a dropped max-subtraction shows
+    h, c = 1, 2
+    kk = wide(ks)[h, c]
+    mean = [sum(kk[t][d] for t in range(L)) / L for d in range(D)]
+    sc = [scale * sum(mean[d] * kk[t][d] for d in range(D)) for t in range(L)]
+    z = sum(math.exp(x) for x in sc)
+    brute = [sum(math.exp(sc[t]) / z * kk[t][d] for t in range(L)) for d in range(D)]
+    np.testing.assert_allclose(s[h, c], brute, rtol=0, atol=1e-13)
+    # scale 0: uniform weights = the mean embedding
+    np.testing.assert_allclose(O.chunk_summaries_attn(ks, 0.0), O.chunk_summaries(ks), rtol=0, atol=1e-15)
+    # identical keys
+    key = torch.randn(D, generator=g).to(torch.bfloat16)
+    same = key.repeat(1, 1, L, 1).clone()
+    np.testing.assert_allclose(O.chunk_summaries_attn(same, 3.0)[0, 0], wide(key), rtol=0, atol=1e-15)
+    # a dominant key: 7 keys e_0, one key 64 e_0 -> mean ~ 8.9 e_0, scores 8.9 vs 568: all weight on it
+    dom = torch.zeros(1, 1, L, D)
+    dom[..., 0] = 1.0
+    dom[0, 0, 5, 0] = 64.0
+    out = O.chunk_summaries_attn(dom.to(torch.bfloat16), 1.0)[0, 0]
+    np.testing.assert_allclose(out, [64.0, 0, 0, 0], rtol=0, atol=1e-12)
+    # token order inside a chunk is irrelevant; other chunks are untouched by a change in one
+    perm = torch.randperm(L, generator=g)
+    ks2 = ks.clone()
+    ks2[0, 1] = ks[0, 1][perm]
+    s2 = O.chunk_summaries_attn(ks2, scale)
+    np.testing.assert_allclose(s2, s, rtol=0, atol=1e-14)
+    ks3 = ks.clone()
+    ks3[1, 0] = -ks[1, 0]
+    s3 = O.chunk_summaries_attn(ks3, scale)
+    assert np.array_equal(np.delete(s3.reshape(Hkv * C, D), 3, axis=0), np.delete(s.reshape(Hkv * C, D), 3, axis=0))
+    assert not np.allclose(s3[1, 0], s[1, 0])
+
+
 # ---------------------------------------------------------------- routing
 def test_route_scores_and_exhaustive_topk():
     p = tiny_problem(2, B=4, Hq=6, Hkv=2, D=8, C=7, L=4, k=3)
