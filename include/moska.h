@@ -137,6 +137,19 @@ int moska_build_chunk_summaries(const uint16_t* k_shared, float* summaries,
                                 const moska_shape* shape, moska_stream stream);
 
 /*
+ * A second training-free chunk embedding for the same `summaries` buffer (Section II-B and III-B
+ * cite two lightweight routers: one pools a chunk's keys uniformly -- the mean above -- the other
+ * weights a chunk's tokens by an attention pass inside the chunk).  Here the chunk's mean key
+ * kbar probes the chunk's own keys:
+ *     w_t = softmax_t(probe_scale * <kbar, k_t>),   summaries[h][c] = sum_t w_t k_t,
+ * so tokens aligned with the chunk's centre count more and outliers less; probe_scale = 0 gives
+ * the mean.  Everything downstream (moska_route and on) is unchanged.  Offline step; fp32.
+ *   probe_scale  finite, >= 0 (1/sqrt(D) is the natural choice); L <= 10240
+ */
+int moska_build_chunk_summaries_attn(const uint16_t* k_shared, float* summaries, float probe_scale,
+                                     const moska_shape* shape, moska_stream stream);
+
+/*
  * Router (Section III-B): relevance of chunk c for (request b, KV head h) is the inner product
  * of the pooled query  qbar[b][h] = sum_{g<G} q[b][h*G+g]  with summaries[h][c]; the k chunks
  * with the largest score are selected, exact ties going to the lower chunk index.

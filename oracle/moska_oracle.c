@@ -391,3 +391,46 @@ void oracle_attend_unique_fp8(const uint16_t* q, const uint8_t* k8, const uint8_
         free(s);
     }
 }
+
+/*
+ * Shared KV Attention over an FP8 shared store (Section III-A with the KV precision of Section
+ * IV).  Storage: E4M3 codes [Hkv][C][L][D] for keys and for values and ONE scale per (KV head,
+ * chunk) for each, so token t of chunk c of head h has key  k_scale[h][c] * e4m3(k8[h][c][t][:])
+ * and value  v_scale[h][c] * e4m3(v8[h][c][t][:]).  Staged form as oracle_shared_partials: one
+ * partial per (row, routed chunk j), attention of the row over the L tokens of that chunk alone.
+ *   ->  o_part [B][Hq][k][D], lse_part [B][Hq][k]
+ */
+void oracle_shared_partials_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v8,
+                                const float* k_scale, const float* v_scale,
+                                const int32_t* topk_idx, double* o_part, double* lse_part,
+                                double scale, int B, int Hq, int Hkv, int D, int C, int L, int k)
+{
+    const int G = Hq / Hkv;
+#pragma omp parallel for schedule(dynamic, 1)
+    for (long rj = 0; rj < (long)B * Hq * k; ++rj) {
+        const long r = rj / k;
+        const int j = (int)(rj % k);
+        const int b = (int)(r / Hq), hq = (int)(r % Hq), h = hq / G;
+        const long hc = (long)h * C + topk_idx[((long)b * Hkv + h) * k + j];
+        const double ksc = (double)k_scale[hc], vsc = (double)v_scale[hc];
+        double* o = o_part + rj * D;
+        double* s = (double*)malloc(sizeof(double) * L);
+        double m = -INFINITY;
+        for (int d = 0; d < D; ++d) o[d] = 0.0;
+        for (int t = 0; t < L; ++t) {
+            double acc = 0.0;
+            for (int d = 0; d < D; ++d)
+                acc += bf16_to_double(q[r * D + d]) * (ksc * oracle_e4m3_value(k8[(hc * L + t) * D + d]));
+            s[t] = scale * acc;
+            if (s[t] > m) m = s[t];
+        }
+        double z = 0.0;
+        for (int t = 0; t < L; ++t) z += exp(s[t] - m);
+        lse_part[rj] = m + log(z);
+        for (int t = 0; t < L; ++t) {
+            const double p = exp(s[t] - lse_part[rj]);
+            for (int d = 0; d < D; ++d) o[d] += p * (vsc * oracle_e4m3_value(v8[(hc * L + t) * D + d]));
+        }
+        free(s);
+    }
+}

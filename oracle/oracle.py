@@ -187,3 +187,30 @@ def attend_unique_fp8(q, k8, v8, k_scale, v_scale, kv_start, kv_len, scale: floa
     _load().oracle_attend_unique_fp8(_p(qb), _p(kk), _p(vv), _p(ks), _p(vs), _p(st), _p(ln), _p(out),
                                      _p(lse), ctypes.c_double(scale), B, Hq, Hkv, D)
     return out, lse
+
+
+def shared_partials_fp8(q, k8, v8, k_scale, v_scale, topk_idx, scale: float):
+    """Per-(row, routed chunk) partials over an FP8 shared store (codes [Hkv][C][L][D], one scale
+    per (KV head, chunk) for K and for V) -> (o_part f64 [B][Hq][k][D], lse_part f64 [B][Hq][k])."""
+    B, Hq, D = q.shape
+    Hkv, C, L, _ = k8.shape
+    idx = _i32(topk_idx)
+    k = idx.shape[2]
+
+    def _u8(t):
+        if isinstance(t, torch.Tensor):
+            t = t.detach().cpu().numpy()
+        return np.ascontiguousarray(t, dtype=np.uint8)
+
+    def _f32(t):
+        if isinstance(t, torch.Tensor):
+            t = t.detach().cpu().numpy()
+        return np.ascontiguousarray(t, dtype=np.float32)
+
+    o = np.empty((B, Hq, k, D), dtype=np.float64)
+    lse = np.empty((B, Hq, k), dtype=np.float64)
+    qb, kk, vv, ks, vs = _bits(q), _u8(k8), _u8(v8), _f32(k_scale), _f32(v_scale)
+    assert ks.shape == (Hkv, C) and vs.shape == (Hkv, C)
+    _load().oracle_shared_partials_fp8(_p(qb), _p(kk), _p(vv), _p(ks), _p(vs), _p(idx), _p(o), _p(lse),
+                                       ctypes.c_double(scale), B, Hq, Hkv, D, C, L, k)
+    return o, lse

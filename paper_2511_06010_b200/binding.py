@@ -49,6 +49,7 @@ EXPORTS = {
     "moska_default_unique_splits": (_i, [ctypes.c_int32] * 3),
     "moska_default_unique_splits_fp8": (_i, [ctypes.c_int32] * 3),
     "moska_build_chunk_summaries": (_i, [_vp, _vp, _sp, _vp]),
+    "moska_build_chunk_summaries_attn": (_i, [_vp, _vp, _f, _sp, _vp]),
     "moska_route": (_i, [_vp, _vp, _vp, _vp, _sp, _vp, _sz, _vp]),
     "moska_group_by_chunk": (_i, [_vp, _vp, _vp, _sp, _vp, _sz, _vp]),
     "moska_group_by_chunk_noalloc": (_i, [_vp, _vp, _vp, _sp, _vp]),
@@ -136,6 +137,12 @@ def default_unique_splits_fp8(B: int, Hkv: int, max_len: int) -> int:
 def build_chunk_summaries(k_shared, summaries, s, stream=None) -> None:
     _check(_lib.moska_build_chunk_summaries(_ptr(k_shared), _ptr(summaries), ctypes.byref(s),
                                             _stream(stream)), "moska_build_chunk_summaries")
+
+
+def build_chunk_summaries_attn(k_shared, summaries, probe_scale, s, stream=None) -> None:
+    _check(_lib.moska_build_chunk_summaries_attn(_ptr(k_shared), _ptr(summaries), probe_scale,
+                                                 ctypes.byref(s), _stream(stream)),
+           "moska_build_chunk_summaries_attn")
 
 
 def route(q, summaries, topk_idx, topk_score, s, ws=None, stream=None) -> None:

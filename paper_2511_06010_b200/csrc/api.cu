@@ -168,6 +168,19 @@ int moska_build_chunk_summaries(const uint16_t* k_shared, float* summaries,
     return launch_summaries(k_shared, summaries, shape, (cudaStream_t)stream);
 }
 
+int moska_build_chunk_summaries_attn(const uint16_t* k_shared, float* summaries, float probe_scale,
+                                     const moska_shape* shape, moska_stream stream)
+{
+    MOSKA_API_RANGE();
+    MOSKA_TRY(check_shape(shape, false));
+    REQUIRE_PTR(k_shared, 16);
+    REQUIRE_PTR(summaries, 16);
+    if (!(probe_scale >= 0.f) || !std::isfinite(probe_scale))
+        return fail(MOSKA_ERR_INVALID_ARG, "probe_scale must be finite and >= 0");
+    MOSKA_TRY(check_device());
+    return launch_summaries_attn(k_shared, summaries, probe_scale, shape, (cudaStream_t)stream);
+}
+
 namespace {
 // SMs the persistent tensor-core kernel gets when it runs beside unique attention: both kernels'
 // work is estimated (tensor-core items from the shape, unique attention from the token hint at

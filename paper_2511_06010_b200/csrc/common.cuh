@@ -87,6 +87,8 @@ constexpr int kDenseTcMinRows = 16; // dense mode: batches with fewer query rows
 // ---- internal launchers (one per .cu file) -----------------------------------------------------
 int launch_summaries(const uint16_t* k_shared, float* summaries, const moska_shape* s,
                      cudaStream_t st);
+int launch_summaries_attn(const uint16_t* k_shared, float* summaries, float probe_scale,
+                          const moska_shape* s, cudaStream_t st);
 int launch_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
                  const moska_shape* s, void* ws, bool mark_groups, cudaStream_t st);
 int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,

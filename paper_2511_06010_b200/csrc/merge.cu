@@ -103,7 +103,134 @@ summaries_kernel(const uint16_t* __restrict__ k_shared, float* __restrict__ summ
     }
 }
 
+// One CTA per (KV head, chunk): attention-pooled chunk embedding.  The chunk's mean key probes
+// the chunk's own keys, w_t = softmax_t(scale * <mean, k_t>), embedding = sum_t w_t k_t; all in
+// fp32, every sum in a fixed order.  The chunk (L * D * 2 bytes) is read three times, the second
+// and third time from L2.  Dynamic shared memory: L floats (the scores).
+template <int D>
+__global__ void __launch_bounds__(256)
+summaries_attn_kernel(const uint16_t* __restrict__ k_shared, float* __restrict__ summaries, int L,
+                      float scale)
+{
+    constexpr int LANES = D / 8;          // threads covering one token row with 16-byte loads
+    constexpr int GROUPS = 256 / LANES;   // token rows in flight per pass
+    extern __shared__ float score[];      // [L]
+    __shared__ float red[GROUPS][D];
+    __shared__ float kbar[D];
+    __shared__ float wred[8];
+    __shared__ float stat[2];
+    const int col = threadIdx.x % LANES, grp = threadIdx.x / LANES;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint16_t* base = k_shared + (long long)blockIdx.x * L * D + col * 8;
+    auto load8 = [&](int t, float (&x)[8]) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(base + (long long)t * D));
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            x[2 * i] = __uint_as_float(w[i] << 16);
+            x[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+        }
+    };
+    // column sums over the tokens, each thread its 8 columns of every GROUPS-th token, then over
+    // the groups in ascending order
+    auto reduce_columns = [&](const float (&acc)[8], float divide_by, float* dst) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) red[grp][col * 8 + i] = acc[i];
+        __syncthreads();
+        if (threadIdx.x < D) {
+            float s = 0.f;
+            for (int gI = 0; gI < GROUPS; ++gI) s += red[gI][threadIdx.x];
+            dst[threadIdx.x] = s / divide_by;
+        }
+        __syncthreads();
+    };
+    // ---- pass 1: the mean key
+    float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+    for (int t = grp; t < L; t += GROUPS) {
+        float x[8];
+        load8(t, x);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] += x[i];
+    }
+    reduce_columns(acc, (float)L, kbar);
+    // ---- pass 2: scores, their maximum and the sum of the exponentials
+    float kb[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) kb[i] = kbar[col * 8 + i];
+    for (int t0 = 0; t0 < L; t0 += GROUPS) {  // every thread takes part in the shuffles
+        const int t = t0 + grp;
+        float d = 0.f;
+        if (t < L) {
+            float x[8];
+            load8(t, x);
+#pragma unroll
+            for (int i = 0; i < 8; ++i) d = fmaf(kb[i], x[i], d);
+        }
+#pragma unroll
+        for (int off = LANES / 2; off > 0; off >>= 1) d += __shfl_xor_sync(0xffffffffu, d, off);
+        if (col == 0 && t < L) score[t] = scale * d;
+    }
+    __syncthreads();
+    float m = -INFINITY;
+    for (int t = threadIdx.x; t < L; t += 256) m = fmaxf(m, score[t]);
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, off));
+    if (lane == 0) wred[warp] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float mm = wred[0];
+        for (int w = 1; w < 8; ++w) mm = fmaxf(mm, wred[w]);
+        stat[0] = mm;
+    }
+    __syncthreads();
+    const float smax = stat[0];
+    float z = 0.f;
+    for (int t = threadIdx.x; t < L; t += 256) {
+        const float e = expf(score[t] - smax);
+        score[t] = e;  // the unnormalised weight
+        z += e;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) z += __shfl_xor_sync(0xffffffffu, z, off);
+    __syncthreads();  // every wred[] of the maximum has been read
+    if (lane == 0) wred[warp] = z;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float zz = 0.f;
+        for (int w = 0; w < 8; ++w) zz += wred[w];
+        stat[1] = zz;
+    }
+    __syncthreads();
+    // ---- pass 3: the weighted column sums
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    for (int t = grp; t < L; t += GROUPS) {
+        float x[8];
+        load8(t, x);
+        const float w = score[t];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = fmaf(w, x[i], acc[i]);
+    }
+    reduce_columns(acc, stat[1], summaries + (long long)blockIdx.x * D);
+}
+
 }  // namespace
+
+int launch_summaries_attn(const uint16_t* k_shared, float* summaries, float probe_scale,
+                          const moska_shape* s, cudaStream_t st)
+{
+    const long long grid = (long long)s->Hkv * s->C;
+    if (grid == 0) return MOSKA_OK;
+    const size_t smem = sizeof(float) * (size_t)s->L;
+    if (smem > 40 * 1024)
+        return fail(MOSKA_ERR_UNSUPPORTED, "attention-pooled summaries are built for L <= 10240");
+    if (s->D == 128)
+        summaries_attn_kernel<128><<<(unsigned)grid, 256, smem, st>>>(k_shared, summaries, s->L, probe_scale);
+    else
+        summaries_attn_kernel<64><<<(unsigned)grid, 256, smem, st>>>(k_shared, summaries, s->L, probe_scale);
+    MOSKA_LAUNCH_CHECK("summaries_attn_kernel");
+    return MOSKA_OK;
+}
 
 int launch_merge(const float* o_part, const float* lse_part, uint16_t* out, float* out_f32,
                  float* lse_out, const moska_shape* s, cudaStream_t st)

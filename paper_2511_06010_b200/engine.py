@@ -50,8 +50,14 @@ class MoskaLayer:
         self.overlap_routing = True
 
     # -- offline ---------------------------------------------------------------------------------
-    def build_summaries(self, k_shared):
-        M.build_chunk_summaries(k_shared, self.summaries, self.shape)
+    def build_summaries(self, k_shared, attention_pooled=False, probe_scale=None):
+        """Chunk embeddings for the router: the mean key, or (attention_pooled) the mean key's
+        softmax-weighted pooling of the chunk's keys."""
+        if attention_pooled:
+            M.build_chunk_summaries_attn(k_shared, self.summaries,
+                                         self.scale if probe_scale is None else probe_scale, self.shape)
+        else:
+            M.build_chunk_summaries(k_shared, self.summaries, self.shape)
         return self.summaries
 
     # -- the individual stages (used by the per-stage parity tests and per-kernel timing) --------

@@ -211,3 +211,36 @@ def quantize_unique_store_fp8(un: UniqueStore, release: bool = False) -> UniqueS
     if release:
         un.v_unique = None
     return UniqueStoreFp8(k8, v8, ks, vs)
+
+
+@dataclasses.dataclass
+class SharedStoreFp8:
+    k8: torch.Tensor        # uint8 [Hkv][C][L][D]  FP8 E4M3 codes of the shared keys
+    v8: torch.Tensor        # uint8 [Hkv][C][L][D]  FP8 E4M3 codes of the shared values
+    k_scale: torch.Tensor   # fp32  [Hkv][C]        key = k_scale[h][c] * e4m3(k8)
+    v_scale: torch.Tensor   # fp32  [Hkv][C]
+
+
+def quantize_shared_store_fp8(sh: SharedStore) -> SharedStoreFp8:
+    """Storage-format conversion of a shared KV store to FP8 E4M3 with ONE scale per (KV head,
+    chunk) for the keys and one for the values: scale = max|x| over the chunk / 448, codes by
+    torch's round-to-nearest cast.  Input preparation only: the FP8 store is what both the CUDA
+    path and the oracle are given (chunk embeddings for the router are built from whichever store
+    the caller keeps in bf16; the benchmark builds them before it drops the bf16 copy)."""
+    def q8(x):
+        Hkv, C = x.shape[:2]
+        codes = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+        scales = torch.empty(Hkv, C, dtype=torch.float32, device=x.device)
+        step = max(1, (1 << 24) // (x.shape[2] * x.shape[3]))
+        for h in range(Hkv):
+            for c0 in range(0, C, step):
+                xs = x[h, c0:c0 + step].float()
+                amax = xs.abs().amax(dim=(-1, -2))
+                scale = torch.where(amax > 0, amax / 448.0, torch.ones_like(amax))
+                codes[h, c0:c0 + step] = (xs / scale[:, None, None]).to(torch.float8_e4m3fn).view(torch.uint8)
+                scales[h, c0:c0 + step] = scale
+        return codes, scales
+
+    k8, ks = q8(sh.k_shared)
+    v8, vs = q8(sh.v_shared)
+    return SharedStoreFp8(k8, v8, ks, vs)

@@ -639,3 +639,78 @@ def test_many_small_segments_run_as_pairs_on_the_tensor_core_kernel():
                    zipf_s=1.2, seed=62)
     run_case(w, n_unique_splits=1, check_baseline=False)
     run_case(w, n_unique_splits=1, check_baseline=False, two_streams=True, unique_tokens=10**9)
+
+
+def test_attention_pooled_chunk_embeddings_and_routing_with_them():
+    """The second chunk embedding (mean key probing the chunk's keys, softmax-weighted pooling)
+    against the oracle, for D = 64 and 128, several chunk lengths and probe scales (0 = the mean);
+    then the router on those embeddings against the oracle's routing on its own, and a whole step
+    routed by them against the definition."""
+    M, MoskaLayer = _mods()
+    for D, Hq, Hkv, C, L, k, ps in ((128, 8, 2, 40, 512, 4, None), (64, 4, 1, 9, 128, 2, 0.5),
+                                   (128, 8, 2, 300, 256, 7, 0.0), (128, 16, 2, 12, 640, 3, 0.3)):
+        w = W.Workload("attnsum", B=24, Hq=Hq, Hkv=Hkv, D=D, C=C, L=L, k=k, unique_len=50, seed=71 + C)
+        sh = W.make_shared_store(w, "cuda")
+        un = W.make_unique_store(w, "cuda")
+        q = W.make_queries(w, sh, 0, "cuda")
+        layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, 50)
+        scale = layer.scale if ps is None else ps
+        layer.build_summaries(sh.k_shared, attention_pooled=True, probe_scale=ps)
+        ref = O.chunk_summaries_attn(sh.k_shared.cpu(), scale)
+        got = layer.summaries.cpu().numpy().astype(np.float64)
+        # fp32 sums of 128..640 terms of magnitude ~1 and fp32 exponentials: a few 1e-6
+        np.testing.assert_allclose(got, ref, rtol=0, atol=2e-5)
+        if ps == 0.0:
+            np.testing.assert_allclose(got, O.chunk_summaries(sh.k_shared.cpu()), rtol=0, atol=4e-6)
+        layer.route(q)
+        ref_idx, _, ref_all = O.route(q.cpu(), ref, w.k, return_all=True)
+        gpu_idx = layer.topk_idx.cpu().numpy()
+        PU.check_routing(gpu_idx, ref_idx, ref_all)
+        out = layer.step(q, sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, un.kv_start, un.kv_len)
+        torch.cuda.synchronize()
+        gpu_idx = layer.topk_idx.cpu().numpy()
+        want, _ = O.attend_direct(q.cpu(), sh.k_shared.cpu(), sh.v_shared.cpu(), un.k_unique.cpu(),
+                                  un.v_unique.cpu(), un.kv_start.cpu(), un.kv_len.cpu(), gpu_idx,
+                                  layer.scale)
+        PU.check_attention(out.float().cpu().numpy(), want, "step routed by attention-pooled embeddings")
+        assert M.device_status() == 0
+
+
+def test_kv_head_shards_of_one_batch_reassemble_to_the_oracle():
+    """One batch split by KV head over N ranks (every rank: Hkv / N heads of the shared and the
+    private store, those heads' queries, no exchange): the N shards, run one after another on this
+    GPU through the same engine a rank uses, concatenated along the head axis, equal the oracle on
+    the whole problem; routing and grouping of a shard equal the whole problem's for its heads."""
+    from paper_2511_06010_b200 import distributed as DD
+
+    M, MoskaLayer = _mods()
+    lens = np.array([300, 1, 0, 1000, 64, 17, 129, 511, 700, 77], dtype=np.int64)
+    w = W.Workload("kvshard", B=len(lens), Hq=16, Hkv=4, D=128, C=24, L=256, k=5, unique_len=0, seed=81)
+    sh = W.make_shared_store(w, "cuda")
+    un = W.make_unique_store(w, "cuda", lens)
+    q = W.make_queries(w, sh, 0, "cuda")
+    summ = O.chunk_summaries(sh.k_shared.cpu())
+    ref_idx, _, ref_all = O.route(q.cpu(), summ, w.k, return_all=True)
+    for world in (2, 4):
+        outs, idxs = [], []
+        for rank in range(world):
+            h0, h1 = DD.kv_head_shard(w.Hkv, rank, world)
+            ws = W.kv_head_shard(w, rank, world)
+            assert (ws.Hkv, ws.Hq) == (h1 - h0, (h1 - h0) * w.G)
+            q_r, ks_r, vs_r, ku_r, vu_r = DD.slice_kv_heads(h0, h1, w.G, q, sh.k_shared, sh.v_shared,
+                                                            un.k_unique, un.v_unique)
+            layer = MoskaLayer(ws.B, ws.Hq, ws.Hkv, ws.D, ws.C, ws.L, ws.k, int(lens.max()),
+                               n_unique_splits=2)
+            layer.build_summaries(ks_r)
+            out = layer.step(q_r, ks_r, vs_r, ku_r, vu_r, un.kv_start, un.kv_len, two_streams=(rank % 2 == 1))
+            torch.cuda.synchronize()
+            outs.append(out.clone())
+            idxs.append(layer.topk_idx.cpu().numpy())
+        out = torch.cat(outs, dim=1)                       # heads of rank 0, then rank 1, ...
+        gpu_idx = np.concatenate(idxs, axis=1)
+        assert PU.check_routing(gpu_idx, ref_idx, ref_all) == 0
+        ref, _ = O.attend_direct(q.cpu(), sh.k_shared.cpu(), sh.v_shared.cpu(), un.k_unique.cpu(),
+                                 un.v_unique.cpu(), un.kv_start.cpu().numpy(), un.kv_len.cpu().numpy(),
+                                 gpu_idx, 1.0 / math.sqrt(w.D))
+        PU.check_attention(out.float().cpu().numpy(), ref, f"{world} KV-head shards reassembled")
+    assert M.device_status() == 0

@@ -78,3 +78,62 @@ def test_fp8_attention_against_a_brute_force_loop_with_scales():
             assert abs(lse[b, hq] - ref_lse) < 1e-12
     # the quantiser really is a storage conversion: dequantised values are close to the originals
     assert float((kd.float() - k.float()).abs().max()) < 0.07 * float(k.float().abs().max())
+
+
+def _small_shared(seed=5, B=3, Hq=4, Hkv=2, D=16, C=4, L=8, k=2):
+    g = torch.Generator().manual_seed(seed)
+    q = torch.randn(B, Hq, D, generator=g).to(torch.bfloat16)
+    ks = (torch.randn(Hkv, C, L, D, generator=g) * torch.rand(Hkv, C, 1, 1, generator=g) * 3).to(torch.bfloat16)
+    vs = (torch.randn(Hkv, C, L, D, generator=g) * (0.2 + torch.rand(Hkv, C, 1, 1, generator=g))).to(torch.bfloat16)
+    topk = np.stack([np.stack([np.sort(np.random.default_rng(seed + 7 * b + h).choice(C, k, replace=False))
+                               for h in range(Hkv)]) for b in range(B)]).astype(np.int32)
+    return q, ks, vs, topk
+
+
+def test_fp8_shared_partials_equal_bf16_partials_on_a_store_both_formats_hold_exactly():
+    """Codes on the E4M3 grid with per-chunk scales that are powers of two: every stored value is
+    exact in bf16 too, so the FP8 staged partials must equal the bf16 oracle's (pinned elsewhere
+    against brute force and the library's attention routine).  A scale applied to the wrong chunk
+    or head, or a K scale used for V, changes the result."""
+    q, ks, vs, topk = _small_shared()
+    Hkv, C = ks.shape[:2]
+    k8 = ks.float().clamp(-448, 448).to(torch.float8_e4m3fn)
+    v8 = vs.float().clamp(-448, 448).to(torch.float8_e4m3fn)
+    rng = np.random.default_rng(1)
+    ksc = (2.0 ** rng.integers(-3, 3, size=(Hkv, C))).astype(np.float32)
+    vsc = (2.0 ** rng.integers(-3, 3, size=(Hkv, C))).astype(np.float32)
+    assert len(np.unique(ksc)) > 2 and not np.array_equal(ksc, vsc)
+    kb = (k8.float() * torch.from_numpy(ksc)[:, :, None, None]).to(torch.bfloat16)
+    vb = (v8.float() * torch.from_numpy(vsc)[:, :, None, None]).to(torch.bfloat16)
+    assert torch.equal(kb.float(), k8.float() * torch.from_numpy(ksc)[:, :, None, None])
+    o8, l8 = O.shared_partials_fp8(q, k8.view(torch.uint8), v8.view(torch.uint8), ksc, vsc, topk, 0.25)
+    ob, lb = O.shared_partials(q, kb, vb, topk, 0.25)
+    np.testing.assert_allclose(o8, ob, rtol=0, atol=1e-13)
+    np.testing.assert_allclose(l8, lb, rtol=0, atol=1e-13)
+
+
+def test_fp8_shared_partials_against_a_brute_force_loop_with_quantiser_scales():
+    q, ks, vs, topk = _small_shared(seed=9)
+    f8 = W.quantize_shared_store_fp8(W.SharedStore(ks, vs, None))
+    assert f8.k_scale.shape == ks.shape[:2] and f8.k8.dtype == torch.uint8
+    scale = 1.0 / math.sqrt(q.shape[-1])
+    o, lse = O.shared_partials_fp8(q, f8.k8, f8.v8, f8.k_scale, f8.v_scale, topk, scale)
+    kd = f8.k8.view(torch.float8_e4m3fn).to(torch.float64) * f8.k_scale[:, :, None, None].to(torch.float64)
+    vd = f8.v8.view(torch.float8_e4m3fn).to(torch.float64) * f8.v_scale[:, :, None, None].to(torch.float64)
+    B, Hq, D = q.shape
+    G = Hq // ks.shape[0]
+    L = ks.shape[2]
+    for b in range(B):
+        for hq in range(Hq):
+            h = hq // G
+            for j, c in enumerate(topk[b, h]):
+                qq = q[b, hq].to(torch.float64)
+                s = torch.tensor([scale * float(qq @ kd[h, c, t]) for t in range(L)], dtype=torch.float64)
+                ref_lse = float(torch.logsumexp(s, 0))
+                p = torch.exp(s - ref_lse)
+                ref = sum(p[t] * vd[h, c, t] for t in range(L))
+                np.testing.assert_allclose(o[b, hq, j], ref.numpy(), rtol=0, atol=1e-12)
+                assert abs(lse[b, hq, j] - ref_lse) < 1e-12
+    # the quantiser is a storage conversion: every chunk uses the full code range, values stay close
+    assert int(f8.k8.view(torch.float8_e4m3fn).float().abs().amax(dim=(-1, -2)).min()) == 448
+    assert float((kd.float() - ks.float()).abs().max()) < 0.07 * float(ks.float().abs().max())
