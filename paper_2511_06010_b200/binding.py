@@ -13,7 +13,8 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "csrc", "libmoska.so")
+# MOSKA_LIB names another build of the library (same ABI) to load instead of the in-tree one.
+LIB_PATH = os.environ.get("MOSKA_LIB") or os.path.join(_HERE, "csrc", "libmoska.so")
 
 if not os.path.exists(LIB_PATH):
     raise ImportError(

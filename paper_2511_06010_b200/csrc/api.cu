@@ -207,6 +207,9 @@ int tc_sm_share(const moska_shape* s, bool dense, double unique_ms)
     return x;
 }
 
+#ifndef MOSKA_BESIDE_MS
+#define MOSKA_BESIDE_MS 0.8
+#endif
 // The event pair that orders the side stream of a two-stream step after / before the main
 // stream.  Events belong to the device they were created on, so there is one pair per (host
 // thread, device ordinal), created on first use with that device current and kept.
@@ -519,7 +522,7 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
         // all SMs.
         const double unique_ms = (double)shape->unique_tokens * shape->Hkv *
                                  (kv.fp8 ? 2.0 * shape->D + 8.0 : 4.0 * shape->D) / 7.0e9;
-        const bool beside = tc && (dense || unique_ms >= 0.8);
+        const bool beside = tc && (dense || unique_ms >= MOSKA_BESIDE_MS);
         if (tc && beside)
             MOSKA_TRY(launch_shared_tc(q, k_shared, v_shared, dense ? nullptr : seg_entries, o_part,
                                        lse_part, softmax_scale, shape, ws, dense,

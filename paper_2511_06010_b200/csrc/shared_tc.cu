@@ -36,10 +36,19 @@ constexpr int kKvTile = 128;                   // tokens per K/V tile
 constexpr int kTileBytes = 128 * kD * 2;       // one Q, K or V tile in shared memory
 constexpr int kHalfBytes = kTileBytes / 2;     // 64 head-dimension columns of a tile
 constexpr int kSubBytes = kTileBytes / 2;      // query sub-buffer for a tile of at most 64 rows
-constexpr int kStages = 4;                     // K/V ring slots
+#ifndef MOSKA_TC_STAGES
+#define MOSKA_TC_STAGES 4
+#endif
+constexpr int kStages = MOSKA_TC_STAGES;       // K/V ring slots (5 fill the 227 KB of an SM exactly)
 constexpr int kThreads = 384;                  // 8 softmax warps, TMA warp, MMA warp, 2 gather warps
 constexpr int kLoadWarp = 8, kMmaWarp = 9, kGatherWarp0 = 10;
-constexpr int kSoftmaxRegs = 208, kOtherRegs = 96;  // per-thread register budgets after set-up
+// Per-thread register budgets after set-up.  The CTA is launched with kLaunchRegs per thread (the
+// 64 K registers of an SM over 384 threads, rounded down to a multiple of 8); what the four other
+// warps give back must cover what the eight softmax warps ask for, or their request never returns.
+constexpr int kLaunchRegs = 168, kSoftmaxRegs = 208, kOtherRegs = 88;
+static_assert(4 * (kLaunchRegs - kOtherRegs) >= 8 * (kSoftmaxRegs - kLaunchRegs),
+              "setmaxnreg: the released registers do not cover the requested ones");
+static_assert(kSoftmaxRegs % 8 == 0 && kOtherRegs % 8 == 0, "setmaxnreg takes multiples of 8");
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.f;       // log2 units a row maximum may lag behind
@@ -56,6 +65,8 @@ struct __align__(1024) TcSmem {
     uint32_t tmem_base;
     int abort_flag;
 };
+
+static_assert(sizeof(TcSmem) + 1024 <= 232448, "the CTA's shared memory exceeds the 227 KB an SM offers");
 
 struct TcParams {
     const uint16_t* q;
