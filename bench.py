@@ -596,7 +596,7 @@ def measure(args, w_full, rank, world, dev, headline: bool):
     rows_merge_bytes = w.B * w.Hq * ((S.shared_slots + S.n_unique_splits) * (w.D + 1) * 4 + w.D * 2)
     # kernels of one step: route (scoring + selection beyond 256 chunks), 2-3 grouping passes, unique,
     # shared, merge
-    n_shared_launches = 1 if (w.D == 128) else 2   # one tensor-core kernel, or 16-row and 8-row tiles
+    n_shared_launches = 2   # the tensor-core kernel and the 8-row streaming tiles, or 16-row and 8-row tiles
     n_launch = 3 if w.dense else (1 + (w.C > 256)) + (3 if w.B > 64 else 2) + 1 + n_shared_launches + 1
     hbm_bytes = work["unique_bytes"] + work["shared_bytes"] + rows_merge_bytes
     amort = P / max(1, touched)

@@ -326,14 +326,14 @@ int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_
             return launch_shared_tc(q, k_shared, v_shared, nullptr, o_part, lse_part, softmax_scale,
                                     shape, ws, true, 0, st);
         return launch_shared_small(q, k_shared, v_shared, nullptr, o_part, lse_part, softmax_scale,
-                                   shape, ws, true, st);
+                                   shape, ws, true, false, st);
     }
     // routed: the grouping pass cut every segment into work items for the kernel that serves the shape
     if (tc)
-        return launch_shared_tc(q, k_shared, v_shared, seg_entries, o_part, lse_part, softmax_scale,
-                                shape, ws, false, 0, st);
+        MOSKA_TRY(launch_shared_tc(q, k_shared, v_shared, seg_entries, o_part, lse_part, softmax_scale,
+                                   shape, ws, false, 0, st));
     return launch_shared_small(q, k_shared, v_shared, seg_entries, o_part, lse_part, softmax_scale,
-                               shape, ws, false, st);
+                               shape, ws, false, tc, st);
 }
 
 int moska_device_status(int32_t* status_host)
@@ -527,9 +527,11 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
             MOSKA_TRY(launch_shared_tc(q, k_shared, v_shared, dense ? nullptr : seg_entries, o_part,
                                        lse_part, softmax_scale, shape, ws, dense,
                                        tc_sm_share(shape, dense, unique_ms), side));
-        if (!tc)
+        // the streaming tiles (every tile of a shape the tensor-core kernel does not serve, else the
+        // 8-row tiles of routed mode) always run beside unique attention
+        if (!tc || !dense)
             MOSKA_TRY(launch_shared_small(q, k_shared, v_shared, dense ? nullptr : seg_entries, o_part,
-                                          lse_part, softmax_scale, shape, ws, dense, side));
+                                          lse_part, softmax_scale, shape, ws, dense, tc, side));
         if (beside || !tc) MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, side));
         MOSKA_CUDA_TRY(cudaEventRecord(ev_join, side));
         MOSKA_CUDA_TRY(cudaStreamWaitEvent(st, ev_join, 0));

@@ -97,7 +97,7 @@ int launch_group_noalloc(const int32_t* topk_idx, int32_t* seg_offsets, int32_t*
                          const moska_shape* s, cudaStream_t st);
 int launch_shared_small(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
                         const int32_t* seg_entries, float* o_part, float* lse_part, float scale,
-                        const moska_shape* s, void* ws, bool dense, cudaStream_t st);
+                        const moska_shape* s, void* ws, bool dense, bool tiny_list_only, cudaStream_t st);
 // Tensor-core (tcgen05) Shared KV Attention over the big-tile work list (routed) or over
 // (KV head, run of chunks, 256 / G requests) items (dense).
 bool shared_tc_supported(const moska_shape* s);

@@ -84,8 +84,10 @@ group_count_kernel(const uint32_t* __restrict__ bitmap, int32_t* __restrict__ to
 // Exclusive scans over the keys, one CTA: entries -> seg_offsets; tiles -> work lists.
 // Shapes the tensor-core kernel serves (tc): a segment's requests go, in order, to items of two
 // 128-row query tiles (big_entries requests; a remainder of more than one tile's requests still
-// forms one) and the rest, if any, to ONE single-tile item in the second list.  Other shapes: 16-row
-// tiles in the second list and a last piece of at most tiny_entries requests (8 rows) in the third.
+// forms one) and the rest, if any, to ONE item: a single-tile item in the second list, or, if it
+// has at most tiny_entries requests (8 rows), an 8-row tile in the third (the streaming kernel:
+// for one or two requests on a chunk nothing beats reading it straight through).  Other shapes:
+// 16-row tiles in the second list and a last piece of at most tiny_entries requests in the third.
 __global__ void __launch_bounds__(1024)
 group_scan_kernel(const uint32_t* __restrict__ bitmap, int words, const int32_t* __restrict__ totals,
                   int32_t* __restrict__ seg_offsets,
@@ -118,7 +120,9 @@ group_scan_kernel(const uint32_t* __restrict__ bitmap, int words, const int32_t*
             n_big = n / big_entries;
             const int rem = n - n_big * big_entries;
             small_cap = big_entries / 2;  // one 128-row query tile
-            if (rem > small_cap) ++n_big; else if (rem > 0) n_small = 1;
+            if (rem > small_cap) ++n_big;
+            else if (rem > tiny_entries) n_small = 1;
+            else if (rem > 0) n_tiny = 1;  // one 8-row column block: the streaming kernel's list
         } else {
             n_small = n / small_entries;
             const int last = n - n_small * small_entries;  // requests of the last, partial tile

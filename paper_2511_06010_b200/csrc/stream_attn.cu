@@ -323,7 +323,7 @@ int launch_gemv_baseline(const uint16_t* q, const uint16_t* k_shared, const uint
 
 int launch_shared_small(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
                         const int32_t* seg_entries, float* o_part, float* lse_part, float scale,
-                        const moska_shape* s, void* ws, bool dense, cudaStream_t st)
+                        const moska_shape* s, void* ws, bool dense, bool tiny_list_only, cudaStream_t st)
 {
     const int n_slots = s->shared_slots + s->n_unique_splits;
     const int G = s->Hq / s->Hkv;
@@ -360,10 +360,12 @@ int launch_shared_small(const uint16_t* q, const uint16_t* k_shared, const uint1
             q, k_shared, v_shared, seg_entries, hdr, ITEMS, o_part, lse_part, scale, s->B, s->Hq,      \
             s->Hkv, s->C, s->L, s->k, s->shared_slots, n_slots, dense ? 1 : 0, WORD);                  \
     } while (0)
-    if (s->D == 128) {
-        MOSKA_LAUNCH_SMALL(128, 2, items, kSmallWord);
-    } else {
-        MOSKA_LAUNCH_SMALL(64, 2, items, kSmallWord);
+    if (!tiny_list_only) {  // (routed shapes of the tensor-core kernel: the second list is not ours)
+        if (s->D == 128) {
+            MOSKA_LAUNCH_SMALL(128, 2, items, kSmallWord);
+        } else {
+            MOSKA_LAUNCH_SMALL(64, 2, items, kSmallWord);
+        }
     }
     if (!dense && tiny_items != nullptr) {
         MOSKA_LAUNCH_CHECK("shared_small_kernel");
