@@ -57,12 +57,18 @@ NCU_TRAFFIC_BYTES = {
     ("unique_staged_kernel", "cfg1_llama8b_b64"): 1.0817e9,
     # profiles/unique_fp8_kernel_cfg1.md: 554.3 MB read + 7.2 MB written
     ("unique_fp8_kernel", "cfg1_llama8b_b64"): 5.615e8,
-    # profiles/shared_tc_kernel_cfg3.md: 559.2 MB read + 139.8 MB written
-    ("shared_tc_kernel", "cfg3_dense_b512"): 6.995e8,
+    # profiles/shared_tc_kernel_cfg3.md: 569.5 MB read + 128.8 MB written
+    ("shared_tc_kernel", "cfg3_dense_b512"): 6.983e8,
+}
+# DRAM bytes the per-request GEMV baseline really reads per launch (ncu), where captured
+GEMV_DRAM_BYTES = {
+    # profiles/gemv_baseline_dram_cfg1.md: 725.7 MB read + 7.3 MB written (algorithmic: 1073.7 MB)
+    "cfg1_llama8b_b64": 7.33e8,
 }
 NCU_TRAFFIC_RATIO = {
-    # unique_staged_kernel: 1.0817 GB measured for 1.0785 GB algorithmic on workload 1
-    "unique_staged_kernel": (1.0817e9 / 1.0785e9, "scaled from the workload-1 capture by bytes"),
+    # profiles/unique_staged_kernel_cfg4_b64.md: 4.7050 GB measured for 4.7009 GB algorithmic on a
+    # 64-request cut of workload 4 (the full workload is too large to capture with counters)
+    "unique_staged_kernel": (4.7050e9 / 4.7009e9, "scaled by bytes from the capture of a 64-request cut of workload 4"),
 }
 
 
@@ -651,6 +657,9 @@ def measure(args, w_full, rank, world, dev, headline: bool):
             # algorithmic bytes of the baseline (every routed chunk once per request and KV head);
             # where they fit the 126 MB L2 part of them never reaches DRAM
             "algorithmic_gbs": work["gemv_bytes"] / (gemv_ms * 1e-3) / 1e9,
+            "algorithmic_bytes": work["gemv_bytes"],
+            "dram_bytes_ncu": GEMV_DRAM_BYTES.get(w_full.name),
+            "shared_attention_bytes": work["shared_bytes"],
             # both kernels alone on the GPU (in the step part of shared attention overlaps unique)
             "shared_speedup": gemv_ms / iso["shared"] if iso["shared"] > 0 else None,
             "amortisation_factor": amort,

@@ -622,12 +622,13 @@ def test_grouping_reports_lists_that_break_its_precondition():
     assert M.device_status() == 0
 
 
-def test_many_small_segments_run_as_pairs_on_the_tensor_core_kernel():
-    """Hundreds of (KV head, chunk) segments of a few rows each: more single-tile items than twice
-    the number of CTAs, so the kernel runs them two per CTA (one per slot, each over its own
-    chunk) and the rest of the last round one per CTA.  Chunks of one, two and four K/V tiles;
-    tiles of at most 64 rows (two alternating query sub-buffers) mixed with tiles of 65 to 128
-    rows (whole buffer) and items of two tiles; also on a share of the SMs (more rounds)."""
+def test_many_small_segments_pairs_on_the_tensor_core_kernel_and_streamed_8_row_tiles():
+    """Hundreds of (KV head, chunk) segments of a few rows each: segments of at most 8 rows go to the
+    streaming tiles, and there are more single-tile items than twice the number of CTAs, so the
+    tensor-core kernel runs them two per CTA (one per slot, each over its own chunk) and the rest
+    of the last round one per CTA.  Chunks of one, two and four K/V tiles; tiles of at most 64 rows
+    (two alternating query sub-buffers) mixed with tiles of 65 to 128 rows (whole buffer) and items
+    of two tiles; also on a share of the SMs (more rounds)."""
     # G = 4, uniform targets: segments of 1-6 requests (4-24 rows)
     for L in (128, 256, 512):
         w = W.Workload(f"pairs_L{L}", B=64, Hq=8, Hkv=2, D=128, C=256, L=L, k=8, unique_len=40, seed=61)
