@@ -234,6 +234,26 @@ int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_
                       moska_stream stream);
 
 /*
+ * Shared KV Attention over a shared store kept in FP8 (E4M3), the KV precision the paper's
+ * evaluation assumes (Section IV) applied to the batched product of Section III-A.  Token t of chunk
+ * c of KV head h has key k_scale[h][c] * e4m3(k8[h][c][t][:]) and value v_scale[h][c] *
+ * e4m3(v8[h][c][t][:]): ONE scale per (KV head, chunk) and tensor, so the key scale joins the softmax
+ * scale and the value scale the final normalisation.  The code tiles arrive by TMA (half the bytes
+ * of the bf16 store), are widened exactly to f16 in shared memory and multiplied on the tensor cores
+ * with f16 Q and P and fp32 accumulation.  Routed mode only (topk_idx, seg_offsets, seg_entries as
+ * for moska_shared_attn, none NULL), D = 128; every segment runs on the tensor-core kernel.
+ *   k8_shared, v8_shared  uint8 [Hkv][C][L][D]  OCP FP8 E4M3 codes (128-byte aligned)
+ *   k_scale, v_scale      float [Hkv][C]        positive
+ * Chunk embeddings for the router are built from whichever copy of the keys the caller has in
+ * bf16 (moska_build_chunk_summaries*); they are an offline step.
+ */
+int moska_shared_attn_fp8(const uint16_t* q, const uint8_t* k8_shared, const uint8_t* v8_shared,
+                          const float* k_scale, const float* v_scale, const int32_t* topk_idx,
+                          const int32_t* seg_offsets, const int32_t* seg_entries, float* o_part,
+                          float* lse_part, float softmax_scale, const moska_shape* shape, void* ws,
+                          size_t ws_bytes, moska_stream stream);
+
+/*
  * Unique KV Attention (Section III-A: per-request attention over private KV, a memory-bound
  * GEMV-like pass).  Split-K over the request's tokens: each of the n_unique_splits slots holds
  * the partial result over a disjoint token range (which range is an implementation detail);
@@ -333,6 +353,20 @@ int moska_decode_step_fp8kv(const uint16_t* q, const float* summaries, const uin
                             float* lse_part, uint16_t* out, float* lse_out, float softmax_scale,
                             const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream,
                             moska_stream side_stream, moska_profiler* prof);
+
+/*
+ * moska_decode_step with the SHARED store in FP8 (laid out as for moska_shared_attn_fp8); the
+ * private store stays bf16.  Same schedule, buffers, outputs and error behaviour; routed mode only
+ * (summaries must not be NULL), D = 128.
+ */
+int moska_decode_step_fp8shared(const uint16_t* q, const float* summaries, const uint8_t* k8_shared,
+                                const uint8_t* v8_shared, const float* k_scale_shared,
+                                const float* v_scale_shared, const uint16_t* k_unique,
+                                const uint16_t* v_unique, const int64_t* kv_start, const int32_t* kv_len,
+                                int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
+                                float* o_part, float* lse_part, uint16_t* out, float* lse_out,
+                                float softmax_scale, const moska_shape* shape, void* ws, size_t ws_bytes,
+                                moska_stream stream, moska_stream side_stream, moska_profiler* prof);
 
 /*
  * moska_decode_step for a caller whose step inputs live in HOST memory: copies q_host (bf16

@@ -55,12 +55,14 @@ EXPORTS = {
     "moska_group_by_chunk": (_i, [_vp, _vp, _vp, _sp, _vp, _sz, _vp]),
     "moska_group_by_chunk_noalloc": (_i, [_vp, _vp, _vp, _sp, _vp]),
     "moska_shared_attn": (_i, [_vp] * 8 + [_f, _sp, _vp, _sz, _vp]),
+    "moska_shared_attn_fp8": (_i, [_vp] * 10 + [_f, _sp, _vp, _sz, _vp]),
     "moska_unique_attn": (_i, [_vp] * 7 + [_f, _sp, _vp]),
     "moska_unique_attn_fp8": (_i, [_vp] * 9 + [_f, _sp, _vp]),
     "moska_merge": (_i, [_vp] * 5 + [_sp, _vp]),
     "moska_gemv_baseline": (_i, [_vp] * 6 + [_f, _sp, _vp]),
     "moska_decode_step": (_i, [_vp] * 15 + [_f, _sp, _vp, _sz, _vp, _vp, _vp]),
     "moska_decode_step_fp8kv": (_i, [_vp] * 17 + [_f, _sp, _vp, _sz, _vp, _vp, _vp]),
+    "moska_decode_step_fp8shared": (_i, [_vp] * 17 + [_f, _sp, _vp, _sz, _vp, _vp, _vp]),
     "moska_decode_step_host": (_i, [_vp] * 16 + [_f, _sp, _vp, _sz, _vp, _vp, _vp]),
     "moska_profiler_create": (_i, [ctypes.POINTER(_vp), ctypes.c_int32]),
     "moska_profiler_destroy": (None, [_vp]),
@@ -176,6 +178,15 @@ def shared_attn(q, k_shared, v_shared, topk_idx, seg_offsets, seg_entries, o_par
                                   ws_bytes, _stream(stream)), "moska_shared_attn")
 
 
+def shared_attn_fp8(q, k8_shared, v8_shared, k_scale, v_scale, topk_idx, seg_offsets, seg_entries, o_part,
+                    lse_part, softmax_scale, s, ws, stream=None) -> None:
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(_lib.moska_shared_attn_fp8(_ptr(q), _ptr(k8_shared), _ptr(v8_shared), _ptr(k_scale), _ptr(v_scale),
+                                      _ptr(topk_idx), _ptr(seg_offsets), _ptr(seg_entries), _ptr(o_part),
+                                      _ptr(lse_part), softmax_scale, ctypes.byref(s), _ptr(ws), ws_bytes,
+                                      _stream(stream)), "moska_shared_attn_fp8")
+
+
 def unique_attn(q, k_unique, v_unique, kv_start, kv_len, o_part, lse_part, softmax_scale, s,
                 stream=None) -> None:
     _check(_lib.moska_unique_attn(_ptr(q), _ptr(k_unique), _ptr(v_unique), _ptr(kv_start),
@@ -225,6 +236,18 @@ def decode_step_fp8kv(q, summaries, k_shared, v_shared, k8_unique, v8_unique, k_
         _ptr(seg_offsets), _ptr(seg_entries), _ptr(o_part), _ptr(lse_part), _ptr(out),
         _ptr(lse_out), softmax_scale, ctypes.byref(s), _ptr(ws), ws_bytes, _stream(stream),
         None if side_stream is None else _stream(side_stream), prof), "moska_decode_step_fp8kv")
+
+
+def decode_step_fp8shared(q, summaries, k8_shared, v8_shared, k_scale_shared, v_scale_shared, k_unique,
+                          v_unique, kv_start, kv_len, topk_idx, seg_offsets, seg_entries, o_part, lse_part, out,
+                          lse_out, softmax_scale, s, ws, stream=None, side_stream=None, prof=None) -> None:
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(_lib.moska_decode_step_fp8shared(
+        _ptr(q), _ptr(summaries), _ptr(k8_shared), _ptr(v8_shared), _ptr(k_scale_shared),
+        _ptr(v_scale_shared), _ptr(k_unique), _ptr(v_unique), _ptr(kv_start), _ptr(kv_len), _ptr(topk_idx),
+        _ptr(seg_offsets), _ptr(seg_entries), _ptr(o_part), _ptr(lse_part), _ptr(out), _ptr(lse_out),
+        softmax_scale, ctypes.byref(s), _ptr(ws), ws_bytes, _stream(stream),
+        None if side_stream is None else _stream(side_stream), prof), "moska_decode_step_fp8shared")
 
 
 def decode_step_host(q_host, q_dev, summaries, k_shared, v_shared, k_unique, v_unique, kv_start,

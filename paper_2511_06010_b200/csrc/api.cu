@@ -336,6 +336,35 @@ int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_
                                shape, ws, false, tc, st);
 }
 
+int moska_shared_attn_fp8(const uint16_t* q, const uint8_t* k8_shared, const uint8_t* v8_shared,
+                          const float* k_scale, const float* v_scale, const int32_t* topk_idx,
+                          const int32_t* seg_offsets, const int32_t* seg_entries, float* o_part,
+                          float* lse_part, float softmax_scale, const moska_shape* shape, void* ws,
+                          size_t ws_bytes, moska_stream stream)
+{
+    MOSKA_API_RANGE();
+    MOSKA_TRY(check_shape(shape, true));
+    if (!shared_tc_supported(shape))
+        return fail(MOSKA_ERR_UNSUPPORTED, "the FP8 shared store is built for D = 128");
+    REQUIRE_PTR(q, 16);
+    REQUIRE_PTR(k8_shared, 128);
+    REQUIRE_PTR(v8_shared, 128);
+    REQUIRE_PTR(k_scale, 4);
+    REQUIRE_PTR(v_scale, 4);
+    REQUIRE_PTR(o_part, 32);
+    REQUIRE_PTR(lse_part, 4);
+    if (topk_idx == nullptr || seg_offsets == nullptr || seg_entries == nullptr)
+        return fail(MOSKA_ERR_UNSUPPORTED, "the FP8 shared store is built for routed mode (no dense mode)");
+    if (shape->shared_slots != shape->k)
+        return fail(MOSKA_ERR_INVALID_ARG, "routed mode needs shared_slots == k");
+    if (ws == nullptr || !aligned(ws, 256) || ws_bytes < ws_layout(shape).total)
+        return fail(MOSKA_ERR_WORKSPACE, "workspace missing, misaligned or smaller than %zu bytes",
+                    ws_layout(shape).total);
+    MOSKA_TRY(check_device());
+    return launch_shared_tc_fp8(q, k8_shared, v8_shared, k_scale, v_scale, seg_entries, o_part, lse_part,
+                                softmax_scale, shape, ws, 0, (cudaStream_t)stream);
+}
+
 int moska_device_status(int32_t* status_host)
 {
     if (status_host == nullptr) return fail(MOSKA_ERR_INVALID_ARG, "status_host is NULL");
@@ -452,8 +481,16 @@ int unique_impl(const uint16_t* q, const UniqueKv& kv, const int64_t* kv_start, 
                              st);
 }
 
+// The shared store in FP8 (codes + one scale per (KV head, chunk)), when the step uses one.
+struct SharedF8 {
+    const uint8_t* k8 = nullptr;
+    const uint8_t* v8 = nullptr;
+    const float* k_scale = nullptr;
+    const float* v_scale = nullptr;
+};
+
 int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* k_shared,
-                     const uint16_t* v_shared, const UniqueKv& kv, const int64_t* kv_start,
+                     const uint16_t* v_shared, const SharedF8* f8, const UniqueKv& kv, const int64_t* kv_start,
                      const int32_t* kv_len, int32_t* topk_idx, int32_t* seg_offsets,
                      int32_t* seg_entries, float* o_part, float* lse_part, uint16_t* out,
                      float* lse_out, float softmax_scale, const moska_shape* shape, void* ws,
@@ -462,6 +499,16 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
 {
     const bool dense = summaries == nullptr;
     cudaStream_t st = (cudaStream_t)stream, side = (cudaStream_t)side_stream;
+    if (f8 != nullptr && dense)
+        return fail(MOSKA_ERR_UNSUPPORTED, "the FP8 shared store is built for routed mode (no dense mode)");
+    // the tensor-core kernel over whichever shared store the step has
+    auto shared_tc = [&](bool dense_mode, int max_ctas, cudaStream_t s_) {
+        if (f8 != nullptr)
+            return launch_shared_tc_fp8(q, f8->k8, f8->v8, f8->k_scale, f8->v_scale, seg_entries, o_part,
+                                        lse_part, softmax_scale, shape, ws, max_ctas, s_);
+        return launch_shared_tc(q, k_shared, v_shared, dense_mode ? nullptr : seg_entries, o_part, lse_part,
+                                softmax_scale, shape, ws, dense_mode, max_ctas, s_);
+    };
     if (side == nullptr) {
         // one stream: route, group, unique, shared, merge
         if (!dense) {
@@ -477,9 +524,13 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
         MOSKA_TRY(unique_impl(q, kv, kv_start, kv_len, o_part, lse_part, softmax_scale, shape, st));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 1, st));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 0, st));
-        MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, dense ? nullptr : topk_idx,
-                                    dense ? nullptr : seg_offsets, dense ? nullptr : seg_entries,
-                                    o_part, lse_part, softmax_scale, shape, ws, ws_bytes, st));
+        if (f8 != nullptr)
+            MOSKA_TRY(moska_shared_attn_fp8(q, f8->k8, f8->v8, f8->k_scale, f8->v_scale, topk_idx, seg_offsets,
+                                            seg_entries, o_part, lse_part, softmax_scale, shape, ws, ws_bytes, st));
+        else
+            MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, dense ? nullptr : topk_idx,
+                                        dense ? nullptr : seg_offsets, dense ? nullptr : seg_entries,
+                                        o_part, lse_part, softmax_scale, shape, ws, ws_bytes, st));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, st));
     } else {
         // Two streams.  Unique attention (HBM-bound, thousands of short-lived CTAs) is enqueued
@@ -492,8 +543,17 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
         cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
         MOSKA_TRY(fork_join_events(&ev_fork, &ev_join));
         MOSKA_TRY(check_shape(shape, !dense));
-        REQUIRE_PTR(k_shared, 128);
-        REQUIRE_PTR(v_shared, 128);
+        if (f8 != nullptr) {
+            if (!shared_tc_supported(shape))
+                return fail(MOSKA_ERR_UNSUPPORTED, "the FP8 shared store is built for D = 128");
+            REQUIRE_PTR(f8->k8, 128);
+            REQUIRE_PTR(f8->v8, 128);
+            REQUIRE_PTR(f8->k_scale, 4);
+            REQUIRE_PTR(f8->v_scale, 4);
+        } else {
+            REQUIRE_PTR(k_shared, 128);
+            REQUIRE_PTR(v_shared, 128);
+        }
         REQUIRE_PTR(o_part, 32);
         REQUIRE_PTR(lse_part, 4);
         if (dense && shape->shared_slots > shape->C)
@@ -523,21 +583,18 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
         const double unique_ms = (double)shape->unique_tokens * shape->Hkv *
                                  (kv.fp8 ? 2.0 * shape->D + 8.0 : 4.0 * shape->D) / 7.0e9;
         const bool beside = tc && (dense || unique_ms >= MOSKA_BESIDE_MS);
-        if (tc && beside)
-            MOSKA_TRY(launch_shared_tc(q, k_shared, v_shared, dense ? nullptr : seg_entries, o_part,
-                                       lse_part, softmax_scale, shape, ws, dense,
-                                       tc_sm_share(shape, dense, unique_ms), side));
+        if (tc && beside) MOSKA_TRY(shared_tc(dense, tc_sm_share(shape, dense, unique_ms), side));
         // the streaming tiles (every tile of a shape the tensor-core kernel does not serve, else the
-        // 8-row tiles of routed mode) always run beside unique attention
-        if (!tc || !dense)
+        // 8-row tiles of routed mode) always run beside unique attention; with the FP8 store the
+        // tensor-core kernel takes those items as well
+        if ((!tc || !dense) && f8 == nullptr)
             MOSKA_TRY(launch_shared_small(q, k_shared, v_shared, dense ? nullptr : seg_entries, o_part,
                                           lse_part, softmax_scale, shape, ws, dense, tc, side));
         if (beside || !tc) MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, side));
         MOSKA_CUDA_TRY(cudaEventRecord(ev_join, side));
         MOSKA_CUDA_TRY(cudaStreamWaitEvent(st, ev_join, 0));
         if (tc && !beside) {
-            MOSKA_TRY(launch_shared_tc(q, k_shared, v_shared, seg_entries, o_part, lse_part,
-                                       softmax_scale, shape, ws, false, 0, st));
+            MOSKA_TRY(shared_tc(false, 0, st));
             MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, st));
         }
     }
@@ -561,9 +618,34 @@ int moska_decode_step(const uint16_t* q, const float* summaries, const uint16_t*
     UniqueKv kv;
     kv.k = k_unique;
     kv.v = v_unique;
-    return decode_step_impl(q, summaries, k_shared, v_shared, kv, kv_start, kv_len, topk_idx,
+    return decode_step_impl(q, summaries, k_shared, v_shared, nullptr, kv, kv_start, kv_len, topk_idx,
                             seg_offsets, seg_entries, o_part, lse_part, out, lse_out, softmax_scale,
                             shape, ws, ws_bytes, stream, side_stream, prof);
+}
+
+int moska_decode_step_fp8shared(const uint16_t* q, const float* summaries, const uint8_t* k8_shared,
+                                const uint8_t* v8_shared, const float* k_scale_shared,
+                                const float* v_scale_shared, const uint16_t* k_unique,
+                                const uint16_t* v_unique, const int64_t* kv_start, const int32_t* kv_len,
+                                int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
+                                float* o_part, float* lse_part, uint16_t* out, float* lse_out,
+                                float softmax_scale, const moska_shape* shape, void* ws, size_t ws_bytes,
+                                moska_stream stream, moska_stream side_stream, moska_profiler* prof)
+{
+    MOSKA_API_RANGE();
+    if (summaries == nullptr)
+        return fail(MOSKA_ERR_UNSUPPORTED, "the FP8 shared store is built for routed mode (no dense mode)");
+    UniqueKv kv;
+    kv.k = k_unique;
+    kv.v = v_unique;
+    SharedF8 f8;
+    f8.k8 = k8_shared;
+    f8.v8 = v8_shared;
+    f8.k_scale = k_scale_shared;
+    f8.v_scale = v_scale_shared;
+    return decode_step_impl(q, summaries, nullptr, nullptr, &f8, kv, kv_start, kv_len, topk_idx, seg_offsets,
+                            seg_entries, o_part, lse_part, out, lse_out, softmax_scale, shape, ws, ws_bytes,
+                            stream, side_stream, prof);
 }
 
 int moska_decode_step_fp8kv(const uint16_t* q, const float* summaries, const uint16_t* k_shared,
@@ -582,7 +664,7 @@ int moska_decode_step_fp8kv(const uint16_t* q, const float* summaries, const uin
     kv.k_scale = k_scale;
     kv.v_scale = v_scale;
     kv.fp8 = true;
-    return decode_step_impl(q, summaries, k_shared, v_shared, kv, kv_start, kv_len, topk_idx,
+    return decode_step_impl(q, summaries, k_shared, v_shared, nullptr, kv, kv_start, kv_len, topk_idx,
                             seg_offsets, seg_entries, o_part, lse_part, out, lse_out, softmax_scale,
                             shape, ws, ws_bytes, stream, side_stream, prof);
 }

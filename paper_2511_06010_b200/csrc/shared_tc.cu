@@ -21,6 +21,7 @@
 // division by the row sum.  TMEM: S_0, S_1, O_0, O_1 of 128 columns each = all 512 columns.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include <mutex>
 
@@ -40,6 +41,11 @@ constexpr int kSubBytes = kTileBytes / 2;      // query sub-buffer for a tile of
 #define MOSKA_TC_STAGES 4
 #endif
 constexpr int kStages = MOSKA_TC_STAGES;       // K/V ring slots (5 fill the 227 KB of an SM exactly)
+// FP8 shared store: the tiles arrive as E4M3 codes (16 KB) in a ring of their own and are widened
+// to f16 operand tiles by the two gather warps; fewer operand slots leave room for the codes.
+constexpr int kCodeBytes = 128 * kD;           // one K or V tile of codes
+constexpr int kCodeStages = 4;
+constexpr int kOpStagesF8 = 3;
 constexpr int kThreads = 384;                  // 8 softmax warps, TMA warp, MMA warp, 2 gather warps
 constexpr int kLoadWarp = 8, kMmaWarp = 9, kGatherWarp0 = 10;
 // Per-thread register budgets after set-up.  The CTA is launched with kLaunchRegs per thread (the
@@ -53,7 +59,13 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 constexpr float kRescaleThreshold = 8.f;       // log2 units a row maximum may lag behind
 
-struct __align__(1024) TcSmem {
+// F: the shared store is FP8 (see above); otherwise bf16 tiles come straight from TMA.
+template <bool F>
+struct TcSmemT;
+
+template <>
+struct __align__(1024) TcSmemT<false> {
+    static constexpr int kOp = kStages;  // operand (K/V) ring slots
     uint8_t q[2][kTileBytes];
     uint8_t kv[kStages][kTileBytes];
     uint64_t full[kStages], empty[kStages];
@@ -66,7 +78,26 @@ struct __align__(1024) TcSmem {
     int abort_flag;
 };
 
-static_assert(sizeof(TcSmem) + 1024 <= 232448, "the CTA's shared memory exceeds the 227 KB an SM offers");
+template <>
+struct __align__(1024) TcSmemT<true> {
+    static constexpr int kOp = kOpStagesF8;
+    uint8_t q[2][kTileBytes];
+    uint8_t kv[kOpStagesF8][kTileBytes];     // f16 operand tiles written by the gather warps
+    uint8_t codes[kCodeStages][kCodeBytes];  // E4M3 code tiles written by TMA
+    uint64_t full[kOpStagesF8], empty[kOpStagesF8];
+    uint64_t code_full[kCodeStages], code_empty[kCodeStages];
+    uint64_t q_full[2][2], q_free[2][2];
+    uint64_t q_ready[2][2];       // the gathered rows have been converted to f16
+    uint64_t s_full[2], p_full[2], o_full[2];
+    uint64_t x_full, x_free;
+    float stat_m[kBigTileRows];
+    float stat_l[kBigTileRows];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+static_assert(sizeof(TcSmemT<false>) + 1024 <= 232448 && sizeof(TcSmemT<true>) + 1024 <= 232448,
+              "the CTA's shared memory exceeds the 227 KB an SM offers");
 
 struct TcParams {
     const uint16_t* q;
@@ -74,6 +105,9 @@ struct TcParams {
     const WsHeader* hdr;
     const TileItem* items;    // items of two query tiles (more than 128 rows)
     const TileItem* singles;  // items of one query tile
+    const TileItem* tiny;     // FP8 store: the 8-row items as well (further single-tile items)
+    const float* k_scale;     // FP8 store: scale per (KV head, chunk) of the keys / values
+    const float* v_scale;
     float* o_part;
     float* lse_part;
     int* status;
@@ -158,6 +192,7 @@ struct Unit {
     int slot_dense;      // dense: partial slot (= run of chunks)
     int n_it[2];         // K/V tiles handled by slot 0 / 1
     long long kv_row0[2];  // first token row of the slot's K/V range in the [Hkv*C*L][D] store
+    int key[2];            // routed: h * C + chunk of the slot's item (index of its scales)
 };
 
 // Where the routed work lists end and how the single-tile items are scheduled on this grid: whole
@@ -176,11 +211,19 @@ __device__ __forceinline__ Schedule make_schedule(const TcParams& p)
         s.n_units = p.n_items_dense;
     } else {
         s.n_two = p.hdr->n_big_tiles;
-        const int n1 = p.hdr->n_small_tiles;
+        const int n1 = p.hdr->n_small_tiles + (p.tiny != nullptr ? p.hdr->n_tiny_tiles : 0);
         s.n_pairs = (n1 / (2 * (int)gridDim.x)) * (int)gridDim.x;
         s.n_units = s.n_two + s.n_pairs + (n1 - 2 * s.n_pairs);
     }
     return s;
+}
+
+// i-th single-tile item: the second work list, then (FP8 store) the third
+__device__ __forceinline__ int4 single_item(const TcParams& p, int i)
+{
+    const int n_small = p.hdr->n_small_tiles;
+    const TileItem* src = i < n_small ? p.singles + i : p.tiny + (i - n_small);
+    return __ldg(reinterpret_cast<const int4*>(src));
 }
 
 __device__ __forceinline__ Unit decode_unit(const TcParams& p, const Schedule& sch, int unit, int G,
@@ -188,6 +231,7 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& p, const Schedule& s
 {
     Unit it;
     it.slot_dense = 0;
+    it.key[0] = it.key[1] = 0;
     it.b0[0] = it.b0[1] = 0;
     if (!p.dense) {
         it.n_kv = p.L / kKvTile;
@@ -200,19 +244,21 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& p, const Schedule& s
             it.n_e[0] = min(raw.z, per_tile);
             it.n_e[1] = min(raw.z - it.n_e[0], per_tile);
             it.kv_row0[0] = it.kv_row0[1] = (long long)raw.x * p.L;
+            it.key[0] = it.key[1] = raw.x;
         } else if (unit < sch.n_two + sch.n_pairs) {
             it.mode = kPair;
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
-                const int4 raw = __ldg(reinterpret_cast<const int4*>(p.singles) + 2 * (unit - sch.n_two) + t);
+                const int4 raw = single_item(p, 2 * (unit - sch.n_two) + t);
                 it.h[t] = raw.x / p.C;
                 it.entry_begin[t] = raw.y;
                 it.n_e[t] = min(raw.z, per_tile);
                 it.kv_row0[t] = (long long)raw.x * p.L;
+                it.key[t] = raw.x;
             }
         } else {
-            const int4 raw = __ldg(reinterpret_cast<const int4*>(p.singles) + 2 * sch.n_pairs +
-                                   (unit - sch.n_two - sch.n_pairs));
+            const int4 raw = single_item(p, 2 * sch.n_pairs + (unit - sch.n_two - sch.n_pairs));
+            it.key[0] = it.key[1] = raw.x;
             it.mode = kSplit;
             it.h[0] = it.h[1] = raw.x / p.C;
             it.entry_begin[0] = it.entry_begin[1] = raw.y;
@@ -285,10 +331,28 @@ __device__ __forceinline__ QUse q_use(const Unit& it, int u, int G, uint32_t& n_
 
 // Roles of the third warp group (after it has given registers up): TMA producer, MMA issuer and
 // the two query-gather warps.
-__device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
+// Two E4M3 codes (low byte -> low half) widened to two f16 values; exact.
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_codes)
+{
+    uint32_t r;
+    const unsigned short v = static_cast<unsigned short>(two_codes);
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(r) : "h"(v));
+    return r;
+}
+
+// Two bf16 values (one 32-bit word) to two f16 values, round to nearest.
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w)
+{
+    const __half2 h = __floats2half2_rn(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
+
+template <bool F>
+__device__ __forceinline__ void other_roles(TcSmemT<F>& sm, const CUtensorMap& tm_k, const CUtensorMap& tm_v,
                                          const CUtensorMap& tm_q, const TcParams& p, const Schedule& sch, int G,
                                          int per_tile, uint32_t tmem, int warp, int lane)
 {
+    constexpr int kOp = TcSmemT<F>::kOp;
     volatile int* ab = &sm.abort_flag;
     const int n_pos = p.B * p.Hkv * p.k;  // routed: valid entries of seg_entries are below this
 
@@ -303,26 +367,43 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
                 const Unit it = decode_unit(p, sch, unit, G, per_tile);
                 const int n_loads = (it.mode == kPair ? 4 : 2) * it.n_kv;
                 for (int x = 0; x < n_loads; ++x, ++ld) {
-                    const uint32_t s = ld % kStages;
-                    if (ld >= kStages && !mbar_wait(&sm.empty[s], ((ld / kStages) - 1) & 1, ab)) {
-                        ok = false;
-                        break;
-                    }
-                    mbar_arrive_expect_tx(&sm.full[s], kTileBytes);
                     const CUtensorMap* tm = (x & 1) ? &tm_v : &tm_k;
                     const int vt = x >> 1;  // tile in ring order
                     const int y = it.mode == kPair
                         ? (int)(it.kv_row0[vt & 1] + (long long)(vt >> 1) * kKvTile)
                         : (int)(it.kv_row0[0] + (long long)vt * kKvTile);
-                    tma_load_2d(sm.kv[s], tm, 0, y, &sm.full[s]);
-                    tma_load_2d(sm.kv[s] + kHalfBytes, tm, 64, y, &sm.full[s]);
+                    if constexpr (F) {
+                        // one box of 128 code rows x 128 bytes into the code ring
+                        const uint32_t s = ld % kCodeStages;
+                        if (ld >= kCodeStages &&
+                            !mbar_wait(&sm.code_empty[s], ((ld / kCodeStages) - 1) & 1, ab)) {
+                            ok = false;
+                            break;
+                        }
+                        mbar_arrive_expect_tx(&sm.code_full[s], kCodeBytes);
+                        tma_load_2d(sm.codes[s], tm, 0, y, &sm.code_full[s]);
+                    } else {
+                        const uint32_t s = ld % kOp;
+                        if (ld >= kOp && !mbar_wait(&sm.empty[s], ((ld / kOp) - 1) & 1, ab)) {
+                            ok = false;
+                            break;
+                        }
+                        mbar_arrive_expect_tx(&sm.full[s], kTileBytes);
+                        tma_load_2d(sm.kv[s], tm, 0, y, &sm.full[s]);
+                        tma_load_2d(sm.kv[s] + kHalfBytes, tm, 64, y, &sm.full[s]);
+                    }
                 }
             }
             if (*ab) {
                 // giving up: let the copies still in flight land before the CTA leaves
                 volatile int never = 0;
-                for (uint32_t x = ld > kStages ? ld - kStages : 0; x < ld; ++x)
-                    mbar_wait(&sm.full[x % kStages], (x / kStages) & 1, &never);
+                if constexpr (F) {
+                    for (uint32_t x = ld > kCodeStages ? ld - kCodeStages : 0; x < ld; ++x)
+                        mbar_wait(&sm.code_full[x % kCodeStages], (x / kCodeStages) & 1, &never);
+                } else {
+                    for (uint32_t x = ld > kOp ? ld - kOp : 0; x < ld; ++x)
+                        mbar_wait(&sm.full[x % kOp], (x / kOp) & 1, &never);
+                }
             }
         }
         __syncwarp();
@@ -333,17 +414,65 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
         // (lane l owns tile rows 4l .. 4l+3), so the copies do not queue behind the softmax
         // groups' result stores in the load/store pipe.  Rows past the item's last one hold
         // stale or repeated query rows; their results are never written.
+        // FP8 store: the same warp then converts the gathered rows to f16 in place and, together with
+        // the other gather warp (64 token rows each), widens the unit's code tiles into the operand
+        // ring.
         const int u = warp - kGatherWarp0;
         uint32_t n_small = 0;
         uint32_t arrivals[2] = {0, 0};  // uses of sub-buffer 0 / 1 so far (a full tile uses both)
         uint64_t* last_full = nullptr;  // barrier and phase of the last gather, for the abort path
         uint32_t last_phase = 0;
         uint32_t fills[2] = {0, 0};     // gathers signalled on q_full[u][0 / 1] so far
+        uint32_t cv = 0;                // FP8 store: code tiles widened so far, over all units
         bool ok = true;
+        // FP8 store: widens this warp's half (64 token rows) of every code tile of the unit
+        auto widen_unit = [&](const Unit& it) {
+            if constexpr (F) {
+                const int n_loads = (it.mode == kPair ? 4 : 2) * it.n_kv;
+                for (int x = 0; x < n_loads && ok; ++x, ++cv) {
+                    const uint32_t cs = cv % kCodeStages, os = cv % kOp;
+                    bool w = mbar_wait(&sm.code_full[cs], (cv / kCodeStages) & 1, ab);
+                    if (w && cv >= kOp) w = mbar_wait(&sm.empty[os], ((cv / kOp) - 1) & 1, ab);
+                    ok = __all_sync(0xffffffffu, w);
+                    if (!ok) break;
+                    const uint8_t* src = sm.codes[cs];
+                    uint8_t* dst = sm.kv[os];
+#pragma unroll 4
+                    for (int i = 0; i < 16; ++i) {
+                        const int idx = i * 32 + lane;
+                        const int row = u * 64 + (idx >> 3), j = idx & 7;  // 16 codes: dims 16j .. 16j+15
+                        const uint4 c = *reinterpret_cast<const uint4*>(src + row * 128 + ((j ^ (row & 7)) << 4));
+                        uint4 lo, hi;
+                        lo.x = e4m3x2_to_f16x2(c.x);
+                        lo.y = e4m3x2_to_f16x2(c.x >> 16);
+                        lo.z = e4m3x2_to_f16x2(c.y);
+                        lo.w = e4m3x2_to_f16x2(c.y >> 16);
+                        hi.x = e4m3x2_to_f16x2(c.z);
+                        hi.y = e4m3x2_to_f16x2(c.z >> 16);
+                        hi.z = e4m3x2_to_f16x2(c.w);
+                        hi.w = e4m3x2_to_f16x2(c.w >> 16);
+                        // the 16 values are pieces 2 (j % 4) and 2 (j % 4) + 1 of the row's half j / 4
+                        uint8_t* drow = dst + (j >> 2) * kHalfBytes + row * 128;
+                        const int c0 = 2 * (j & 3);
+                        *reinterpret_cast<uint4*>(drow + ((c0 ^ (row & 7)) << 4)) = lo;
+                        *reinterpret_cast<uint4*>(drow + (((c0 + 1) ^ (row & 7)) << 4)) = hi;
+                    }
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        mbar_arrive(&sm.full[os]);
+                        mbar_arrive(&sm.code_empty[cs]);
+                    }
+                }
+            }
+        };
         for (int unit = blockIdx.x; unit < sch.n_units && ok; unit += gridDim.x) {
             const Unit it = decode_unit(p, sch, unit, G, per_tile);
             const QUse qu = q_use(it, u, G, n_small);
-            if (!qu.present) continue;
+            if (!qu.present) {
+                widen_unit(it);
+                continue;
+            }
             int rr[4];  // global query rows of tile rows 4 * lane .. 4 * lane + 3
 #pragma unroll
             for (int m = 0; m < 4; ++m) {
@@ -384,6 +513,29 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
                 tma_gather4_2d(dst, &tm_q, 0, rr[0], rr[1], rr[2], rr[3], bar);
                 tma_gather4_2d(dst + half, &tm_q, 64, rr[0], rr[1], rr[2], rr[3], bar);
             }
+            if constexpr (F) {
+                // the rows have landed: bf16 -> f16 in place (the copied groups only), then tell
+                // the MMA warp
+                ok = __all_sync(0xffffffffu, mbar_wait(bar, last_phase, ab));
+                if (!ok) break;
+                uint8_t* base = sm.q[u] + (qu.small ? qu.sub * kSubBytes : 0);
+                const int half = qu.small ? kSubBytes / 2 : kHalfBytes;
+                const int n_pieces = n_groups * 4 * 8;  // 16-byte pieces per half
+                for (int i = lane; i < 2 * n_pieces; i += 32) {
+                    uint4* ptr = reinterpret_cast<uint4*>(base + (i >= n_pieces ? half : 0) +
+                                                          (i % n_pieces) * 16);
+                    uint4 v = *ptr;
+                    v.x = bf16x2_to_f16x2(v.x);
+                    v.y = bf16x2_to_f16x2(v.y);
+                    v.z = bf16x2_to_f16x2(v.z);
+                    v.w = bf16x2_to_f16x2(v.w);
+                    *ptr = v;
+                }
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.q_ready[u][qu.sub]);
+                widen_unit(it);
+            }
         }
         if (*ab && last_full != nullptr) {
             // giving up: let the copies still in flight land before the CTA leaves
@@ -393,8 +545,9 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
     } else {
         // =========================== MMA issuer ===================================================
         if (lane == 0) {
-            const uint32_t id_qk = idesc_bf16_f32(128, kKvTile, false);
-            const uint32_t id_pv = idesc_bf16_f32(128, kD, true);
+            // bf16 operands, or (FP8 store) f16 operands: Q and P are then f16 as well
+            const uint32_t id_qk = F ? idesc_f16_f32(128, kKvTile, false) : idesc_bf16_f32(128, kKvTile, false);
+            const uint32_t id_pv = F ? idesc_f16_f32(128, kD, true) : idesc_bf16_f32(128, kD, true);
             // Operand descriptors differ only in their start-address field (low word, units of 16
             // bytes): build the constant parts once and add tile offsets per instruction, so that
             // issuing an MMA costs a handful of integer instructions.
@@ -448,7 +601,7 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
                     return it.mode != kTwoTiles || it.n_it[1] == 0 || tq == 1;
                 };
                 auto wait_load = [&](uint32_t g) {
-                    return mbar_wait(&sm.full[g % kStages], (g / kStages) & 1, ab);
+                    return mbar_wait(&sm.full[g % kOp], (g / kOp) & 1, ab);
                 };
                 auto issue_scores = [&](int tq, uint32_t s) {
                     const int u = it.mode == kSplit ? 0 : tq;
@@ -467,7 +620,9 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
                 q_reads[1] = it.mode == kSplit ? 0 : it.n_it[1];
                 for (int u = 0; u < 2 && ok; ++u) {
                     if (!qu[u].present) continue;
-                    ok = mbar_wait(&sm.q_full[u][qu[u].sub], fills[u][qu[u].sub]++ & 1, ab);
+                    uint64_t* bar;
+                    if constexpr (F) bar = &sm.q_ready[u][qu[u].sub]; else bar = &sm.q_full[u][qu[u].sub];
+                    ok = mbar_wait(bar, fills[u][qu[u].sub]++ & 1, ab);
                 }
                 // first scores of both slots
                 for (int tq = 0; tq < 2 && ok; ++tq) {
@@ -476,8 +631,8 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
                     ok = wait_load(g);
                     if (!ok) break;
                     tc_fence_after_sync();
-                    issue_scores(tq, g % kStages);
-                    if (last_reader(tq)) tc_commit(&sm.empty[g % kStages]);
+                    issue_scores(tq, g % kOp);
+                    if (last_reader(tq)) tc_commit(&sm.empty[g % kOp]);
                 }
                 for (int x = 0; x < it.n_it[0] && ok; ++x) {
                     for (int tq = 0; tq < 2 && ok; ++tq) {
@@ -487,15 +642,15 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
                         if (!ok) break;
                         ++pc[tq];
                         tc_fence_after_sync();
-                        issue_pv(tq, gv % kStages, x > 0);
-                        if (last_reader(tq)) tc_commit(&sm.empty[gv % kStages]);
+                        issue_pv(tq, gv % kOp, x > 0);
+                        if (last_reader(tq)) tc_commit(&sm.empty[gv % kOp]);
                         if (x + 1 < it.n_it[tq]) {
                             const uint32_t gk = k_load(tq, x + 1);
                             ok = wait_load(gk);
                             if (!ok) break;
                             tc_fence_after_sync();
-                            issue_scores(tq, gk % kStages);
-                            if (last_reader(tq)) tc_commit(&sm.empty[gk % kStages]);
+                            issue_scores(tq, gk % kOp);
+                            if (last_reader(tq)) tc_commit(&sm.empty[gk % kOp]);
                         } else {
                             tc_commit(&sm.o_full[tq]);
                         }
@@ -508,13 +663,15 @@ __device__ __forceinline__ void other_roles(TcSmem& sm, const CUtensorMap& tm_k,
     }
 }
 
+template <bool F>
 __global__ void __launch_bounds__(kThreads, 1)
 shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
                  const __grid_constant__ CUtensorMap tm_q, const TcParams p)
 {
     extern __shared__ uint8_t smem_raw[];
-    TcSmem& sm = *reinterpret_cast<TcSmem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
-                                            ~static_cast<uintptr_t>(1023));
+    TcSmemT<F>& sm = *reinterpret_cast<TcSmemT<F>*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                                    ~static_cast<uintptr_t>(1023));
+    constexpr int kOp = TcSmemT<F>::kOp;
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int G = p.Hq / p.Hkv;
     const int per_tile = kBigTileRows / G;  // requests per query tile
@@ -523,9 +680,17 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 
     // ---- set-up: barriers, tensor memory --------------------------------------------------------
     if (tid == 0) {
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(&sm.full[s], 1);
+        for (int s = 0; s < kOp; ++s) {
+            mbar_init(&sm.full[s], F ? 2 : 1);  // FP8 store: one arrival per widening warp
             mbar_init(&sm.empty[s], 1);
+        }
+        if constexpr (F) {
+            for (int s = 0; s < kCodeStages; ++s) {
+                mbar_init(&sm.code_full[s], 1);
+                mbar_init(&sm.code_empty[s], 2);
+            }
+            for (int u = 0; u < 2; ++u)
+                for (int sb = 0; sb < 2; ++sb) mbar_init(&sm.q_ready[u][sb], 1);
         }
         for (int u = 0; u < 2; ++u) {
             for (int sb = 0; sb < 2; ++sb) {
@@ -566,7 +731,6 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         const uint32_t t_s = tmem + lane_sel + t * 128;        // S_t, and P_t over its columns
         const uint32_t t_o = tmem + lane_sel + 256 + t * 128;  // O_t
         const uint32_t t_o_other = tmem + lane_sel + 256 + (1 - t) * 128;
-        const float sl2 = p.scale * kLog2e;
         const int n_pos = p.B * p.Hkv * p.k;
         uint32_t sc = 0, oc[2] = {0, 0}, xc = 0;  // barrier phases completed before this unit
         bool alive = true;
@@ -578,6 +742,11 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             oc[0] += it.n_it[0] > 0;
             oc[1] += it.n_it[1] > 0;
             xc += split;
+            // FP8 store: the chunk's key scale joins the softmax scale, its value scale the final
+            // normalisation (routed mode: one chunk per item)
+            const float ksc = F ? __ldg(p.k_scale + pick(it.key, t)) : 1.f;
+            const float vsc = F ? __ldg(p.v_scale + pick(it.key, t)) : 1.f;
+            const float sl2 = p.scale * kLog2e * ksc;
             const int n_rows = pick(it.n_e, t) * G;
             // a warp none of whose rows exists skips the arithmetic (every row of the products
             // depends on its own query row only), but keeps every barrier in step
@@ -674,8 +843,13 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                             pr.x = fast_exp2(e.x);
                             pr.y = fast_exp2(e.y);
                             ls[x & 1] = fadd2(ls[x & 1], pr);
-                            __nv_bfloat162 b2 = __floats2bfloat162_rn(pr.x, pr.y);
-                            pk[x] = *reinterpret_cast<uint32_t*>(&b2);
+                            if constexpr (F) {
+                                const __half2 h2 = __floats2half2_rn(pr.x, pr.y);
+                                pk[x] = *reinterpret_cast<const uint32_t*>(&h2);
+                            } else {
+                                const __nv_bfloat162 b2 = __floats2bfloat162_rn(pr.x, pr.y);
+                                pk[x] = *reinterpret_cast<const uint32_t*>(&b2);
+                            }
                         }
                         tmem_st16(t_s + c * 16, pk);
                     }
@@ -712,7 +886,7 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             }
             if (warp_live) {
                 tc_fence_after_sync();
-                const float inv = 1.f / den;
+                const float inv = vsc / den;
                 a_mine *= inv;
                 a_other *= inv;
                 float4* o = my_r >= 0
@@ -751,7 +925,7 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         for (int x = 0; x < 4; ++x)
                             st_global_v8(reinterpret_cast<float*>(o) + c * 32 + x * 8,
                                          reinterpret_cast<const float*>(&r[c][8 * x]));
-                    p.lse_part[my_r * p.n_slots + my_slot] = m_all * p.scale + logf(den);
+                    p.lse_part[my_r * p.n_slots + my_slot] = m_all * (p.scale * ksc) + logf(den);
                 }
             }
             if (split) {
@@ -761,7 +935,7 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
         }
     } else {
         asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kOtherRegs));
-        other_roles(sm, tm_k, tm_v, tm_q, p, sch, G, per_tile, tmem, warp, lane);
+        other_roles<F>(sm, tm_k, tm_v, tm_q, p, sch, G, per_tile, tmem, warp, lane);
     }
 
     // ---- teardown -------------------------------------------------------------------------------
@@ -833,10 +1007,32 @@ int make_q_map(CUtensorMap* tm, const uint16_t* base, long long rows)
 
 bool shared_tc_supported(const moska_shape* s) { return s->D == kD && s->L % kKvTile == 0; }
 
-int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
-                     const int32_t* seg_entries, float* o_part, float* lse_part, float scale,
-                     const moska_shape* s, void* ws, bool dense, int max_ctas, cudaStream_t st)
+namespace {
+
+// [rows][128] matrix of E4M3 codes, loaded in boxes of 128 rows x 128 bytes with the 128-byte swizzle.
+int make_code_map(CUtensorMap* tm, const uint8_t* base, long long rows)
 {
+    EncodeTiledFn enc = nullptr;
+    MOSKA_TRY_STATUS(encoder(&enc));
+    const cuuint64_t dims[2] = {(cuuint64_t)kD, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)kD};
+    const cuuint32_t box[2] = {(cuuint32_t)kD, (cuuint32_t)kKvTile};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = enc(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<uint8_t*>(base), dims, strides,
+                           box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return fail(MOSKA_ERR_CUDA, "cuTensorMapEncodeTiled failed for FP8 codes (%d)", (int)r);
+    return MOSKA_OK;
+}
+
+// Common part of the two launchers.  k8 / v8 != nullptr selects the FP8 shared store (routed mode
+// only; every single-tile item, the 8-row ones included, runs on this kernel then).
+int launch_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared, const uint8_t* k8,
+              const uint8_t* v8, const float* k_scale, const float* v_scale, const int32_t* seg_entries,
+              float* o_part, float* lse_part, float scale, const moska_shape* s, void* ws, bool dense,
+              int max_ctas, cudaStream_t st)
+{
+    const bool fp8 = k8 != nullptr;
     const int G = s->Hq / s->Hkv;
     const int per_cta = 2 * (kBigTileRows / G);
     long long grid;  // upper bound of the number of work items
@@ -850,6 +1046,7 @@ int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t
         p.hdr = reinterpret_cast<const WsHeader*>(ws);
         p.items = reinterpret_cast<const TileItem*>(static_cast<const char*>(ws) + lay.off_big);
         p.singles = reinterpret_cast<const TileItem*>(static_cast<const char*>(ws) + lay.off_small);
+        if (fp8) p.tiny = reinterpret_cast<const TileItem*>(static_cast<const char*>(ws) + lay.off_tiny);
     }
     if (grid == 0) return MOSKA_OK;
     if (grid > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "shared attention grid too large");
@@ -862,13 +1059,20 @@ int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t
     const long long kv_rows = (long long)s->Hkv * s->C * s->L;
     if (kv_rows > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "shared store exceeds 2^31 tokens");
     CUtensorMap tm_k, tm_v, tm_q;
-    MOSKA_TRY_STATUS(make_kv_map(&tm_k, k_shared, kv_rows));
-    MOSKA_TRY_STATUS(make_kv_map(&tm_v, v_shared, kv_rows));
+    if (fp8) {
+        MOSKA_TRY_STATUS(make_code_map(&tm_k, k8, kv_rows));
+        MOSKA_TRY_STATUS(make_code_map(&tm_v, v8, kv_rows));
+    } else {
+        MOSKA_TRY_STATUS(make_kv_map(&tm_k, k_shared, kv_rows));
+        MOSKA_TRY_STATUS(make_kv_map(&tm_v, v_shared, kv_rows));
+    }
     MOSKA_TRY_STATUS(make_q_map(&tm_q, q, (long long)s->B * s->Hq));
     int* status = nullptr;
     MOSKA_TRY_STATUS(status_word(&status));
     p.q = q;
     p.seg_entries = seg_entries;
+    p.k_scale = k_scale;
+    p.v_scale = v_scale;
     p.o_part = o_part;
     p.lse_part = lse_part;
     p.status = status;
@@ -882,11 +1086,35 @@ int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t
     p.shared_slots = s->shared_slots;
     p.n_slots = s->shared_slots + s->n_unique_splits;
     p.dense = dense ? 1 : 0;
-    const int smem = (int)sizeof(TcSmem) + 1024;
-    MOSKA_CUDA_TRY(cudaFuncSetAttribute(shared_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    shared_tc_kernel<<<(unsigned)grid, kThreads, smem, st>>>(tm_k, tm_v, tm_q, p);
+    if (fp8) {
+        const int smem = (int)sizeof(TcSmemT<true>) + 1024;
+        MOSKA_CUDA_TRY(cudaFuncSetAttribute(shared_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        shared_tc_kernel<true><<<(unsigned)grid, kThreads, smem, st>>>(tm_k, tm_v, tm_q, p);
+    } else {
+        const int smem = (int)sizeof(TcSmemT<false>) + 1024;
+        MOSKA_CUDA_TRY(cudaFuncSetAttribute(shared_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        shared_tc_kernel<false><<<(unsigned)grid, kThreads, smem, st>>>(tm_k, tm_v, tm_q, p);
+    }
     MOSKA_LAUNCH_CHECK("shared_tc_kernel");
     return MOSKA_OK;
+}
+
+}  // namespace
+
+int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
+                     const int32_t* seg_entries, float* o_part, float* lse_part, float scale,
+                     const moska_shape* s, void* ws, bool dense, int max_ctas, cudaStream_t st)
+{
+    return launch_tc(q, k_shared, v_shared, nullptr, nullptr, nullptr, nullptr, seg_entries, o_part, lse_part,
+                     scale, s, ws, dense, max_ctas, st);
+}
+
+int launch_shared_tc_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v8, const float* k_scale,
+                         const float* v_scale, const int32_t* seg_entries, float* o_part, float* lse_part,
+                         float scale, const moska_shape* s, void* ws, int max_ctas, cudaStream_t st)
+{
+    return launch_tc(q, nullptr, nullptr, k8, v8, k_scale, v_scale, seg_entries, o_part, lse_part, scale, s,
+                     ws, false, max_ctas, st);
 }
 
 // Measured on B200: an item costs about 6 us of fill, drain and epilogue plus 2.2 us per K/V

@@ -196,6 +196,12 @@ __host__ __device__ constexpr uint32_t idesc_bf16_f32(int M, int N, bool b_mn_ma
            | (static_cast<uint32_t>(M >> 4) << 24);   // M / 16
 }
 
+// The same with f16 A and B.
+__host__ __device__ constexpr uint32_t idesc_f16_f32(int M, int N, bool b_mn_major)
+{
+    return idesc_bf16_f32(M, N, b_mn_major) & ~((1u << 7) | (1u << 10));
+}
+
 // D[tmem] (+)= A[smem] * B[smem]; issued by ONE thread.
 __device__ __forceinline__ void mma_ss(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
                                        uint32_t idesc, bool accumulate)

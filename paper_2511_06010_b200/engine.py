@@ -71,6 +71,11 @@ class MoskaLayer:
         M.shared_attn(q, k_shared, v_shared, self.topk_idx, self.seg_offsets, self.seg_entries,
                       self.o_part, self.lse_part, self.scale, self.shape, self.ws)
 
+    def shared_fp8(self, q, sf8):
+        """Shared KV Attention over an FP8 shared store (`sf8`: codes and per-chunk scales)."""
+        M.shared_attn_fp8(q, sf8.k8, sf8.v8, sf8.k_scale, sf8.v_scale, self.topk_idx, self.seg_offsets,
+                          self.seg_entries, self.o_part, self.lse_part, self.scale, self.shape, self.ws)
+
     def gemv_baseline(self, q, k_shared, v_shared):
         M.gemv_baseline(q, k_shared, v_shared, self.topk_idx, self.o_part, self.lse_part,
                         self.scale, self.shape)
@@ -112,6 +117,19 @@ class MoskaLayer:
                             self.seg_offsets, self.seg_entries, self.o_part, self.lse_part,
                             self.out, self.lse_out, self.scale, self.shape, self.ws, None,
                             self.side_stream if two_streams else None, prof)
+        return self.out
+
+    def step_fp8shared(self, q, sf8, k_unique, v_unique, kv_start, kv_len, two_streams=False, prof=None,
+                       unique_tokens=0):
+        """One decode step with the SHARED store in FP8 (`sf8`: codes and per-chunk scales)."""
+        self.shape.unique_tokens = int(unique_tokens)
+        two_streams = two_streams and self.overlap_routing
+        if two_streams and self.side_stream is None:
+            self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
+        M.decode_step_fp8shared(q, self.summaries, sf8.k8, sf8.v8, sf8.k_scale, sf8.v_scale, k_unique,
+                                v_unique, kv_start, kv_len, self.topk_idx, self.seg_offsets, self.seg_entries,
+                                self.o_part, self.lse_part, self.out, self.lse_out, self.scale, self.shape,
+                                self.ws, None, self.side_stream if two_streams else None, prof)
         return self.out
 
     def bind_step_host(self, q_host, q_dev, out_host, k_shared, v_shared, k_unique, v_unique,

@@ -1,0 +1,87 @@
+"""GPU parity of Shared KV Attention over an FP8 (E4M3, one scale per (KV head, chunk)) shared store:
+the tensor-core kernel fed with code tiles, against the fp64 oracle that decodes the same codes from
+the format's definition.  Tolerances are those of the bf16 path (tests/parity_utils.py)."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import oracle as O
+from paper_2511_06010_b200 import workloads as W
+from tests import parity_utils as PU
+
+pytestmark = pytest.mark.gpu
+
+
+def _mods():
+    from paper_2511_06010_b200 import binding as M
+    from paper_2511_06010_b200.engine import MoskaLayer
+
+    return M, MoskaLayer
+
+
+def _case(w, lengths=None, n_unique_splits=2, sample=None, two_streams=False, unique_tokens=0):
+    M, MoskaLayer = _mods()
+    sh = W.make_shared_store(w, "cuda")
+    un = W.make_unique_store(w, "cuda", lengths)
+    q = W.make_queries(w, sh, 0, "cuda")
+    f8 = W.quantize_shared_store_fp8(sh)
+    max_len = int(un.kv_len.max().item()) if w.B else 1
+    layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, max_len, n_unique_splits=n_unique_splits)
+    layer.build_summaries(sh.k_shared)        # offline, from the bf16 copy of the keys
+    layer.route(q)
+    layer.group()
+    sample = np.arange(w.B) if sample is None else np.asarray(sample)
+    topk = layer.topk_idx.cpu().numpy()
+    # staged oracle on the same codes: one partial per (row, routed chunk)
+    o_ref, l_ref = O.shared_partials_fp8(q[sample].cpu(), f8.k8.cpu(), f8.v8.cpu(), f8.k_scale.cpu(),
+                                         f8.v_scale.cpu(), topk[sample], layer.scale)
+    layer.o_part.fill_(float("nan"))
+    layer.lse_part.fill_(float("nan"))
+    layer.shared_fp8(q, f8)
+    torch.cuda.synchronize()
+    n_sh = layer.shape.shared_slots
+    PU.check_lse(layer.lse_part[sample][:, :, :n_sh].cpu().numpy(), l_ref, "fp8 shared lse")
+    PU.check_attention(layer.o_part[sample][:, :, :n_sh].cpu().numpy(), o_ref, "fp8 shared partial o")
+    assert torch.isfinite(layer.o_part[:, :, :n_sh]).all(), "a shared slot was left unwritten"
+    # the whole step: shared partials of the oracle merged with its unique partial
+    out = layer.step_fp8shared(q, f8, un.k_unique, un.v_unique, un.kv_start, un.kv_len,
+                               two_streams=two_streams, unique_tokens=unique_tokens)
+    torch.cuda.synchronize()
+    dummy = torch.zeros(w.Hkv, 1, 128, w.D, dtype=torch.bfloat16)
+    lens = un.kv_len.cpu().numpy()[sample]
+    starts = un.kv_start.cpu().numpy()[sample]
+    o_un, l_un = O.attend_direct(q[sample].cpu(), dummy, dummy, un.k_unique.cpu(), un.v_unique.cpu(), starts, lens,
+                                 np.zeros((len(sample), w.Hkv, 1), dtype=np.int32), layer.scale, use_shared=False)
+    o_all = np.concatenate([o_ref, o_un[:, :, None, :]], axis=2)
+    l_all = np.concatenate([l_ref, l_un[:, :, None]], axis=2)
+    want, want_lse = O.merge(o_all, l_all)
+    PU.check_attention(out[sample].float().cpu().numpy(), want, "fp8-shared decode step out")
+    PU.check_lse(layer.lse_out[sample].cpu().numpy(), want_lse, "fp8-shared decode step lse")
+    assert M.device_status() == 0
+
+
+def test_fp8_shared_small_and_large_segments_every_element():
+    """Segments of one request up to hundreds of rows (8-row items, single-tile items as pairs and
+    split, two-tile items), chunks of one to five K/V tiles, G = 4 and 8, ragged private contexts."""
+    lens = np.array([0, 1, 100, 257, 64, 33, 700, 15], dtype=np.int64)
+    for Hq, Hkv, B, C, L, k in ((8, 2, 12, 32, 512, 4), (8, 2, 96, 4, 256, 2), (16, 2, 70, 3, 128, 2),
+                                (8, 2, 200, 4, 640, 2), (8, 2, 64, 256, 256, 8)):
+        w = W.Workload("f8sh", B=B, Hq=Hq, Hkv=Hkv, D=128, C=C, L=L, k=k, unique_len=0, seed=91 + B)
+        _case(w, lengths=np.resize(lens, B))
+
+
+def test_fp8_shared_full_cfg1_sampled_two_streams():
+    w = W.CONFIGS[1]
+    _case(w, sample=[0, 7, 21, 40, 63], n_unique_splits=None, two_streams=True,
+          unique_tokens=w.B * w.unique_len)
+
+
+def test_fp8_shared_rejects_what_it_does_not_serve():
+    M, MoskaLayer = _mods()
+    layer = MoskaLayer(4, 4, 1, 64, 8, 128, 2, 16)          # D = 64
+    f8 = W.SharedStoreFp8(*(torch.zeros(1, device="cuda") for _ in range(4)))
+    with pytest.raises(M.MoskaError) as e:
+        layer.shared_fp8(torch.zeros(4, 4, 64, dtype=torch.bfloat16, device="cuda"), f8)
+    assert e.value.status == M.ERR_UNSUPPORTED
