@@ -351,6 +351,9 @@ def measure(args, w_full, rank, world, dev, headline: bool):
             raise SystemExit("--unique-kv fp8 needs head dimension 128")
         f8 = W.quantize_unique_store_fp8(un, release=True)
         torch.cuda.empty_cache()
+    sfp8 = args.shared_kv == "fp8"
+    if sfp8 and (w.D != 128 or w.dense or fp8 or T > 1):
+        raise SystemExit("--shared-kv fp8 needs head dimension 128, routed mode, the bf16 private store and q_len 1")
     n_q = max(1, w.steps)
     qs = [W.make_queries(w, sh, s, dev) for s in range(n_q)]
     kv_lens = [(un.kv_len + s).to(torch.int32) for s in range(n_q)]
@@ -360,6 +363,11 @@ def measure(args, w_full, rank, world, dev, headline: bool):
     S = layer.shape
     if not w.dense:
         layer.build_summaries(sh.k_shared)
+    sf8 = None
+    if sfp8:
+        # the shared store in FP8 E4M3 with one scale per (KV head, chunk); the chunk embeddings were
+        # built from the bf16 keys (offline step); the bf16 copy is kept only for the per-request baseline
+        sf8 = W.quantize_shared_store_fp8(sh)
     torch.cuda.synchronize()
 
     two_streams = (not args.one_stream) and layer.overlap_routing
@@ -374,7 +382,10 @@ def measure(args, w_full, rank, world, dev, headline: bool):
 
     def step(i, prof=None):
         s = i % n_q
-        if fp8:
+        if sfp8:
+            layer.step_fp8shared(qs[s], sf8, un.k_unique, un.v_unique, un.kv_start, kv_lens[s],
+                                 two_streams=two_streams, prof=prof, unique_tokens=tokens[s])
+        elif fp8:
             layer.step_fp8kv(qs[s], sh.k_shared, sh.v_shared, f8, un.kv_start, kv_lens[s],
                              two_streams=two_streams, prof=prof, unique_tokens=tokens[s])
         else:
@@ -385,11 +396,15 @@ def measure(args, w_full, rank, world, dev, headline: bool):
 
     def step_host(i):
         s = i % n_q
-        if fp8:
-            # no host-buffer entry point for the FP8 store: the same copies around the device call
+        if fp8 or sfp8:
+            # no host-buffer entry point for the FP8 stores: the same copies around the device call
             q_dev.copy_(q_host[s], non_blocking=True)
-            out = layer.step_fp8kv(q_dev, sh.k_shared, sh.v_shared, f8, un.kv_start, kv_lens[s],
-                                   two_streams=two_streams, unique_tokens=tokens[s])
+            if sfp8:
+                out = layer.step_fp8shared(q_dev, sf8, un.k_unique, un.v_unique, un.kv_start, kv_lens[s],
+                                           two_streams=two_streams, unique_tokens=tokens[s])
+            else:
+                out = layer.step_fp8kv(q_dev, sh.k_shared, sh.v_shared, f8, un.kv_start, kv_lens[s],
+                                       two_streams=two_streams, unique_tokens=tokens[s])
             out_host.copy_(out, non_blocking=True)
             torch.cuda.current_stream().synchronize()
         else:
@@ -438,6 +453,8 @@ def measure(args, w_full, rank, world, dev, headline: bool):
     work = algorithmic_work(w, lens, S.n_unique_splits, S.shared_slots, touched)
     if fp8:  # one byte per element and two fp32 scales per (token, KV head) instead of bf16 K and V
         work["unique_bytes"] -= int(lens.sum()) * w.Hkv * (2 * w.D - 8)
+    if sfp8:  # one byte per element of every touched chunk (the two scales per chunk are negligible)
+        work["shared_bytes"] -= touched * 2 * w.D * w.L
     t_flops = work["shared_flops"] / (peaks["bf16_tflops_sustained"] * 1e12)
     t_bytes = work["shared_bytes"] / (peaks["hbm_gbs"] * 1e9)
     t_unique = work["unique_bytes"] / (peaks["hbm_gbs"] * 1e9)
@@ -551,7 +568,10 @@ def measure(args, w_full, rank, world, dev, headline: bool):
     if not w.dense:
         iso["route"] = time_events(lambda: layer.route(qs[0]), iters, flush)
         iso["group"] = time_events(lambda: layer.group(), iters, flush)
-    iso["shared"] = time_events(lambda: layer.shared(qs[0], sh.k_shared, sh.v_shared), iters, flush)
+    if sfp8:
+        iso["shared"] = time_events(lambda: layer.shared_fp8(qs[0], sf8), iters, flush)
+    else:
+        iso["shared"] = time_events(lambda: layer.shared(qs[0], sh.k_shared, sh.v_shared), iters, flush)
     iso["unique"] = time_events(unique_alone, iters, flush)
     iso["merge"] = time_events(lambda: layer.merge(), iters, flush)
     shared_ms, unique_ms = stage_ms["shared"], stage_ms["unique"]
@@ -594,7 +614,7 @@ def measure(args, w_full, rank, world, dev, headline: bool):
 
     # ---- CPU baseline: the oracle as it stands on the host cores, bounded sample (N = 1 only)
     cpu = None
-    if world == 1 and not args.no_cpu_baseline and not fp8 and T == 1:
+    if world == 1 and not args.no_cpu_baseline and not fp8 and not sfp8 and T == 1:
         cpu = cpu_baseline(w, sh, un, qs[0], kv_lens[0], args.cpu_sample,
                            args.cpu_seconds if headline else args.cpu_seconds / 2)
 
@@ -602,7 +622,9 @@ def measure(args, w_full, rank, world, dev, headline: bool):
     rows_merge_bytes = w.B * w.Hq * ((S.shared_slots + S.n_unique_splits) * (w.D + 1) * 4 + w.D * 2)
     # kernels of one step: route (scoring + selection beyond 256 chunks), 2-3 grouping passes, unique,
     # shared, merge
-    n_shared_launches = 2   # the tensor-core kernel and the 8-row streaming tiles, or 16-row and 8-row tiles
+    # the tensor-core kernel and the 8-row streaming tiles (FP8 store: the tensor-core kernel alone), or
+    # 16-row and 8-row tiles
+    n_shared_launches = 1 if sfp8 else 2
     n_launch = 3 if w.dense else (1 + (w.C > 256)) + (3 if w.B > 64 else 2) + 1 + n_shared_launches + 1
     hbm_bytes = work["unique_bytes"] + work["shared_bytes"] + rows_merge_bytes
     amort = P / max(1, touched)
@@ -616,6 +638,7 @@ def measure(args, w_full, rank, world, dev, headline: bool):
             "unique_tokens_mean": float(lens.mean()), "n_unique_splits": S.n_unique_splits,
             "shared_slots": S.shared_slots, "streams": 2 if two_streams else 1,
             "unique_kv": "fp8_e4m3 + fp32 scale per (token, kv head)" if fp8 else "bf16",
+            "shared_kv": "fp8_e4m3 + fp32 scale per (kv head, chunk)" if sfp8 else "bf16",
             "q_len": T, "requests": w.B // T,
             "l2": ("flushed between steps" if flush is not None
                    else f"inputs exceed L2 ({input_bytes / 2**20:.0f} MiB of K/V per step)"),
@@ -807,6 +830,9 @@ def main():
     ap.add_argument("--unique-splits", type=int, default=None, help="override the split-K count of unique attention")
     ap.add_argument("--unique-kv", default="bf16", choices=["bf16", "fp8"],
                     help="storage of the private KV (fp8: E4M3 codes with per-token scales; no CPU baseline)")
+    ap.add_argument("--shared-kv", default="bf16", choices=["bf16", "fp8"],
+                    help="storage of the shared KV (fp8: E4M3 codes with one scale per (KV head, chunk); routed "
+                         "workloads; no CPU baseline)")
     ap.add_argument("--q-len", type=int, default=1,
                     help="query tokens per request (batch rows = requests x q_len; queries/s counts rows; no CPU baseline)")
     ap.add_argument("--no-baseline", action="store_true")
