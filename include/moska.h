@@ -57,7 +57,8 @@ typedef enum moska_status {
     MOSKA_ERR_UNSUPPORTED = -2, /* D not in {64,128}, G > 8, L % 128 != 0, device is not sm_100 */
     MOSKA_ERR_WORKSPACE   = -3, /* workspace missing or smaller than moska_workspace_bytes()    */
     MOSKA_ERR_CUDA        = -4, /* a CUDA runtime call or kernel launch failed                  */
-    MOSKA_ERR_TIMEOUT     = -5  /* device side: a bounded wait inside a kernel ran out          */
+    MOSKA_ERR_TIMEOUT     = -5, /* device side: a bounded wait inside a kernel ran out          */
+    MOSKA_ERR_CORRUPT     = -6  /* device side, debug build: workspace guard words overwritten  */
 } moska_status;
 
 /* Problem shape of one decode step of one layer. */
@@ -108,8 +109,9 @@ const char* moska_last_error(void);
  * bounded waits (TMA or MMA completion).  MOSKA_ERR_INVALID_ARG: a grouping call (either entry
  * point) met a chunk index outside [0, C) or a (request, KV head) list that is not strictly
  * ascending, or shared attention met an entry of seg_entries outside [0, B*Hkv*k).  In every
- * case the outputs of the steps since the last read are not valid.  The most negative code
- * raised since the last read is the one reported. */
+ * case the outputs of the steps since the last read are not valid.  MOSKA_ERR_CORRUPT (debug
+ * build only): guard words of the workspace were overwritten or a work list would have overflowed.
+ * The most negative code raised since the last read is the one reported. */
 int moska_device_status(int32_t* status_host);
 
 /* n_slots = shared_slots + n_unique_splits; negative status if the shape is invalid. Host only. */
@@ -212,6 +214,22 @@ int moska_group_by_chunk(const int32_t* topk_idx, int32_t* seg_offsets, int32_t*
 int moska_group_by_chunk_noalloc(const int32_t* topk_idx, int32_t* seg_offsets,
                                  int32_t* seg_entries, const moska_shape* shape,
                                  moska_stream stream);
+
+/*
+ * Debug aid (no counterpart in the paper).  A library compiled with -DMOSKA_DEBUG_GUARDS
+ * (`python -m paper_2511_06010_b200.build --debug` -> csrc/libmoska_debug.so) leaves 256 guard
+ * bytes behind every region of the workspace (moska_workspace_bytes grows accordingly), fills them
+ * and the regions' alignment padding with a pattern at the start of moska_route /
+ * moska_group_by_chunk, compares them at the end of the grouping, and checks every work-list write
+ * against the list's capacity.  This call compares the guard words once more, at any later point
+ * (after shared attention, after the step): a mismatch raises MOSKA_ERR_CORRUPT in the device
+ * status word (moska_device_status).  Nothing traps; a write beyond a list's capacity is skipped.
+ *   ws, ws_bytes   the workspace the grouping call was given (device pointer, 256-byte aligned)
+ * Returns MOSKA_ERR_UNSUPPORTED in a library built without the guard words (the regular build:
+ * its workspace layout has no room for them and its kernels carry no checks).
+ */
+int moska_debug_check_workspace(void* ws, size_t ws_bytes, const moska_shape* shape,
+                                moska_stream stream);
 
 /*
  * Shared KV Attention (Section III-A, Fig. 2a): for every non-empty segment (h, c) the query rows
@@ -372,6 +390,12 @@ int moska_decode_step_fp8shared(const uint16_t* q, const float* summaries, const
  * moska_decode_step for a caller whose step inputs live in HOST memory: copies q_host (bf16
  * [B][Hq][D], ideally pinned) into q_dev, runs the step, copies `out` back into out_host (bf16
  * [B][Hq][D]) and waits for the stream.  The KV stores and all scratch stay on the device.
+ * q_host must be 16-byte aligned.  With a side stream and buffers of 4 MiB or more the copies
+ * leave the critical path: a PAGE-LOCKED q_host is copied on the side stream in front of the
+ * router while unique attention reads its query rows straight from host memory, and the result
+ * is merged in four row ranges, each copied to out_host on the side stream while the next one is
+ * merged.  Pageable buffers and small ones take one copy before and one after the step.  Both
+ * host buffers belong to the call until it returns.
  */
 int moska_decode_step_host(const uint16_t* q_host, uint16_t* q_dev, const float* summaries,
                            const uint16_t* k_shared, const uint16_t* v_shared,

@@ -37,6 +37,7 @@ class MoskaError(RuntimeError):
 
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5
+ERR_CORRUPT = -6
 
 _vp, _sz, _f, _i = ctypes.c_void_p, ctypes.c_size_t, ctypes.c_float, ctypes.c_int
 _sp = ctypes.POINTER(MoskaShape)
@@ -54,6 +55,7 @@ EXPORTS = {
     "moska_route": (_i, [_vp, _vp, _vp, _vp, _sp, _vp, _sz, _vp]),
     "moska_group_by_chunk": (_i, [_vp, _vp, _vp, _sp, _vp, _sz, _vp]),
     "moska_group_by_chunk_noalloc": (_i, [_vp, _vp, _vp, _sp, _vp]),
+    "moska_debug_check_workspace": (_i, [_vp, _sz, _sp, _vp]),
     "moska_shared_attn": (_i, [_vp] * 8 + [_f, _sp, _vp, _sz, _vp]),
     "moska_shared_attn_fp8": (_i, [_vp] * 10 + [_f, _sp, _vp, _sz, _vp]),
     "moska_unique_attn": (_i, [_vp] * 7 + [_f, _sp, _vp]),
@@ -167,6 +169,13 @@ def group_by_chunk_noalloc(topk_idx, seg_offsets, seg_entries, s, stream=None) -
     _check(_lib.moska_group_by_chunk_noalloc(_ptr(topk_idx), _ptr(seg_offsets), _ptr(seg_entries),
                                              ctypes.byref(s), _stream(stream)),
            "moska_group_by_chunk_noalloc")
+
+
+def debug_check_workspace(ws, s, stream=None) -> None:
+    """Debug build of the library only: compares the workspace's guard words (a mismatch shows as
+    ERR_CORRUPT in device_status()); the regular build raises ERR_UNSUPPORTED."""
+    _check(_lib.moska_debug_check_workspace(_ptr(ws), ws.numel() * ws.element_size(), ctypes.byref(s),
+                                            _stream(stream)), "moska_debug_check_workspace")
 
 
 def shared_attn(q, k_shared, v_shared, topk_idx, seg_offsets, seg_entries, o_part, lse_part,

@@ -2,7 +2,9 @@
 
 Every .cu file is compiled to an object of its own (in parallel, only when it or a header is
 newer than the object) under csrc/_build/, then linked.  Run as
-`python -m paper_2511_06010_b200.build [--force] [-v]` or call `build()`.
+`python -m paper_2511_06010_b200.build [--force] [-v] [--debug]` or call `build()`.
+`--debug` / `build(debug=True)` builds csrc/libmoska_debug.so instead: the same sources with
+-DMOSKA_DEBUG_GUARDS (guard words around the workspace regions, capacity checks on the work lists).
 """
 from __future__ import annotations
 
@@ -17,6 +19,7 @@ CSRC = os.path.join(HERE, "csrc")
 OBJ_DIR = os.path.join(CSRC, "_build")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(CSRC, "libmoska.so")
+LIB_DEBUG = os.path.join(CSRC, "libmoska_debug.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a",
@@ -40,23 +43,26 @@ def _newer(deps, target) -> bool:
     return any(os.path.getmtime(p) > t for p in deps)
 
 
-def _stale() -> bool:
-    return _newer(sources() + _headers(), LIB)
+def _stale(lib: str = LIB) -> bool:
+    return _newer(sources() + _headers(), lib)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and not _stale():
-        return LIB
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    lib = LIB_DEBUG if debug else LIB
+    if not force and not _stale(lib):
+        return lib
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     os.makedirs(OBJ_DIR, exist_ok=True)
     headers = _headers()
+    extra = ["-DMOSKA_DEBUG_GUARDS"] if debug else []
+    suffix = ".debug.o" if debug else ".o"
     jobs = []
     objects = []
     for src in sources():
-        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + ".o")
+        obj = os.path.join(OBJ_DIR, os.path.basename(src)[:-3] + suffix)
         objects.append(obj)
         if force or _newer([src] + headers, obj):
-            cmd = [nvcc, *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-c", src, "-o", obj]
+            cmd = [nvcc, *NVCC_FLAGS, *extra, "-I", INCLUDE, "-I", CSRC, "-c", src, "-o", obj]
             if verbose:
                 cmd[1:1] = ["-Xptxas", "-v"]
             jobs.append(cmd)
@@ -67,13 +73,14 @@ def build(force: bool = False, verbose: bool = False) -> str:
             sys.stderr.write(r.stdout + r.stderr)
         if r.returncode != 0:
             raise subprocess.CalledProcessError(r.returncode, cmd)
-    stale_objects = set(os.listdir(OBJ_DIR)) - {os.path.basename(o) for o in objects}
-    for name in stale_objects:  # objects of source files that no longer exist
-        os.remove(os.path.join(OBJ_DIR, name))
+    known = {os.path.basename(s)[:-3] for s in sources()}
+    for name in os.listdir(OBJ_DIR):  # objects of source files that no longer exist
+        if name.split(".")[0] not in known:
+            os.remove(os.path.join(OBJ_DIR, name))
     subprocess.check_call([nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-shared",
-                           "-o", LIB, *objects])
-    return LIB
+                           "-o", lib, *objects])
+    return lib
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

@@ -291,6 +291,24 @@ int moska_group_by_chunk_noalloc(const int32_t* topk_idx, int32_t* seg_offsets,
     return launch_group_noalloc(topk_idx, seg_offsets, seg_entries, shape, (cudaStream_t)stream);
 }
 
+int moska_debug_check_workspace(void* ws, size_t ws_bytes, const moska_shape* shape,
+                                moska_stream stream)
+{
+    MOSKA_API_RANGE();
+    MOSKA_TRY(check_shape(shape, true));
+#ifdef MOSKA_DEBUG_GUARDS
+    if (ws == nullptr || !aligned(ws, 256) || ws_bytes < ws_layout(shape).total)
+        return fail(MOSKA_ERR_WORKSPACE, "workspace missing, misaligned or smaller than %zu bytes",
+                    ws_layout(shape).total);
+    MOSKA_TRY(check_device());
+    return launch_ws_guards(ws, ws_layout(shape), true, (cudaStream_t)stream);
+#else
+    (void)ws; (void)ws_bytes; (void)stream;
+    return fail(MOSKA_ERR_UNSUPPORTED, "this build of the library has no workspace guard words "
+                                       "(compile with -DMOSKA_DEBUG_GUARDS)");
+#endif
+}
+
 int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,
                       const int32_t* topk_idx, const int32_t* seg_offsets,
                       const int32_t* seg_entries, float* o_part, float* lse_part,
@@ -489,16 +507,48 @@ struct SharedF8 {
     const float* v_scale = nullptr;
 };
 
+// moska_decode_step_host: results of at least this many bytes leave the device in pieces, each
+// copied while the next one is merged
+#ifndef MOSKA_HOST_PIECES
+#define MOSKA_HOST_PIECES 4
+#endif
+#ifndef MOSKA_HOST_Q_DIRECT
+#define MOSKA_HOST_Q_DIRECT 1
+#endif
+constexpr size_t kHostPiecesMinBytes = 4u << 20;
+constexpr int kHostPieces = MOSKA_HOST_PIECES;
+
 int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* k_shared,
                      const uint16_t* v_shared, const SharedF8* f8, const UniqueKv& kv, const int64_t* kv_start,
                      const int32_t* kv_len, int32_t* topk_idx, int32_t* seg_offsets,
                      int32_t* seg_entries, float* o_part, float* lse_part, uint16_t* out,
                      float* lse_out, float softmax_scale, const moska_shape* shape, void* ws,
                      size_t ws_bytes, moska_stream stream, moska_stream side_stream,
-                     moska_profiler* prof)
+                     moska_profiler* prof, uint16_t* out_host = nullptr,
+                     const uint16_t* q_host = nullptr)
 {
     const bool dense = summaries == nullptr;
     cudaStream_t st = (cudaStream_t)stream, side = (cudaStream_t)side_stream;
+    // q_host (moska_decode_step_host): the queries still have to be copied into q.  With two
+    // streams and a page-locked source the copy runs on the side stream in front of the router
+    // while unique attention, first on `stream`, reads its query rows straight from host memory.
+    const size_t q_bytes = sizeof(uint16_t) * (size_t)shape->B * shape->Hq * shape->D;
+    const uint16_t* q_unique = q;
+    bool copy_on_side = false;
+    if (q_host != nullptr) {
+#if MOSKA_HOST_Q_DIRECT
+        cudaPointerAttributes attr{};
+        if (side != nullptr && q_bytes >= kHostPiecesMinBytes &&
+            cudaPointerGetAttributes(&attr, q_host) == cudaSuccess && attr.type == cudaMemoryTypeHost &&
+            attr.devicePointer != nullptr) {
+            q_unique = static_cast<const uint16_t*>(attr.devicePointer);
+            copy_on_side = true;
+        }
+        (void)cudaGetLastError();
+#endif
+        if (!copy_on_side)
+            MOSKA_CUDA_TRY(cudaMemcpyAsync(const_cast<uint16_t*>(q), q_host, q_bytes, cudaMemcpyHostToDevice, st));
+    }
     if (f8 != nullptr && dense)
         return fail(MOSKA_ERR_UNSUPPORTED, "the FP8 shared store is built for routed mode (no dense mode)");
     // the tensor-core kernel over whichever shared store the step has
@@ -562,8 +612,10 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
             return fail(MOSKA_ERR_INVALID_ARG, "routed mode needs shared_slots == k");
         MOSKA_CUDA_TRY(cudaEventRecord(ev_fork, st));
         MOSKA_CUDA_TRY(cudaStreamWaitEvent(side, ev_fork, 0));
+        if (copy_on_side)
+            MOSKA_CUDA_TRY(cudaMemcpyAsync(const_cast<uint16_t*>(q), q_host, q_bytes, cudaMemcpyHostToDevice, side));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 0, st));
-        MOSKA_TRY(unique_impl(q, kv, kv_start, kv_len, o_part, lse_part, softmax_scale, shape, st));
+        MOSKA_TRY(unique_impl(q_unique, kv, kv_start, kv_len, o_part, lse_part, softmax_scale, shape, st));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 1, st));
         if (!dense) {
             MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_ROUTE, 0, side));
@@ -599,7 +651,33 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
         }
     }
     MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_MERGE, 0, st));
-    MOSKA_TRY(moska_merge(o_part, lse_part, out, nullptr, lse_out, shape, st));
+    const long long rows = (long long)shape->B * shape->Hq;
+    const size_t out_bytes = sizeof(uint16_t) * (size_t)rows * shape->D;
+    if (out_host != nullptr && side != nullptr && out_bytes >= kHostPiecesMinBytes) {
+        // result wanted in host memory: merge the rows in pieces on `stream` and copy every piece
+        // on the side stream (idle by now) while the next one is merged
+        REQUIRE_PTR(o_part, 16);
+        REQUIRE_PTR(lse_part, 4);
+        REQUIRE_PTR(out, 8);
+        cudaEvent_t ev_piece = nullptr, ev_done = nullptr;
+        MOSKA_TRY(fork_join_events(&ev_piece, &ev_done));
+        const long long per = ((rows + kHostPieces - 1) / kHostPieces + 7) / 8 * 8;
+        for (long long r0 = 0; r0 < rows; r0 += per) {
+            const long long n = rows - r0 < per ? rows - r0 : per;
+            MOSKA_TRY(launch_merge_rows(o_part, lse_part, out, nullptr, lse_out, shape, r0, n, st));
+            MOSKA_CUDA_TRY(cudaEventRecord(ev_piece, st));
+            MOSKA_CUDA_TRY(cudaStreamWaitEvent(side, ev_piece, 0));
+            MOSKA_CUDA_TRY(cudaMemcpyAsync(out_host + r0 * shape->D, out + r0 * shape->D,
+                                           sizeof(uint16_t) * (size_t)n * shape->D,
+                                           cudaMemcpyDeviceToHost, side));
+        }
+        MOSKA_CUDA_TRY(cudaEventRecord(ev_done, side));
+        MOSKA_CUDA_TRY(cudaStreamWaitEvent(st, ev_done, 0));
+    } else {
+        MOSKA_TRY(moska_merge(o_part, lse_part, out, nullptr, lse_out, shape, st));
+        if (out_host != nullptr)
+            MOSKA_CUDA_TRY(cudaMemcpyAsync(out_host, out, out_bytes, cudaMemcpyDeviceToHost, st));
+    }
     MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_MERGE, 1, st));
     if (prof != nullptr && prof->n_steps < prof->max_steps) ++prof->n_steps;
     return MOSKA_OK;
@@ -739,14 +817,16 @@ int moska_decode_step_host(const uint16_t* q_host, uint16_t* q_dev, const float*
     MOSKA_TRY(check_shape(shape, summaries != nullptr));
     if (q_host == nullptr || q_dev == nullptr || out_dev == nullptr || out_host == nullptr)
         return fail(MOSKA_ERR_INVALID_ARG, "q_host, q_dev, out_dev and out_host must not be NULL");
+    if (!aligned(q_host, 16))
+        return fail(MOSKA_ERR_INVALID_ARG, "q_host is not 16-byte aligned");
     cudaStream_t st = (cudaStream_t)stream;
-    const size_t bytes = sizeof(uint16_t) * (size_t)shape->B * shape->Hq * shape->D;
-    MOSKA_CUDA_TRY(cudaMemcpyAsync(q_dev, q_host, bytes, cudaMemcpyHostToDevice, st));
-    MOSKA_TRY(moska_decode_step(q_dev, summaries, k_shared, v_shared, k_unique, v_unique, kv_start,
-                                kv_len, topk_idx, seg_offsets, seg_entries, o_part, lse_part,
-                                out_dev, nullptr, softmax_scale, shape, ws, ws_bytes, stream,
-                                side_stream, prof));
-    MOSKA_CUDA_TRY(cudaMemcpyAsync(out_host, out_dev, bytes, cudaMemcpyDeviceToHost, st));
+    UniqueKv kv;
+    kv.k = k_unique;
+    kv.v = v_unique;
+    MOSKA_TRY(decode_step_impl(q_dev, summaries, k_shared, v_shared, nullptr, kv, kv_start, kv_len,
+                               topk_idx, seg_offsets, seg_entries, o_part, lse_part, out_dev, nullptr,
+                               softmax_scale, shape, ws, ws_bytes, stream, side_stream, prof, out_host,
+                               q_host));
     MOSKA_CUDA_TRY(cudaStreamSynchronize(st));
     return MOSKA_OK;
 }

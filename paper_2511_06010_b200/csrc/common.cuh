@@ -64,6 +64,16 @@ struct WsHeader {
 };
 static_assert(sizeof(WsHeader) == 256, "header is one 256-byte block");
 
+// A build with -DMOSKA_DEBUG_GUARDS leaves 256 guard bytes behind every region of the workspace,
+// writes a pattern into them (and into the region's alignment padding) before the grouping passes
+// and checks it after them; the work-list writes are also checked against the lists' capacity.
+#ifdef MOSKA_DEBUG_GUARDS
+constexpr size_t kGuardBytes = 256;
+#else
+constexpr size_t kGuardBytes = 0;
+#endif
+constexpr int kWsRegions = 6;  // bit sets, totals, three work lists, router scores
+
 struct WsLayout {
     int32_t words;            // 32-bit words of one key's request bit set
     int32_t n_keys;           // Hkv * C
@@ -76,8 +86,14 @@ struct WsLayout {
     size_t group_total;  // end of what the grouping passes and shared attention use
     size_t off_scores;   // router: fp32 scores [B * Hkv][C] (only when C > kRouteSmallC)
     size_t total;
+    // debug build: guard words fill [guard_begin[r], guard_end[r]) behind region r's payload
+    size_t guard_begin[kWsRegions], guard_end[kWsRegions];
 };
 WsLayout ws_layout(const moska_shape* s);
+// Debug build (MOSKA_DEBUG_GUARDS): writes the guard words behind every workspace region
+// (check = false) or compares them and raises MOSKA_ERR_CORRUPT in the device status word
+// (check = true).  Other builds: does nothing.
+int launch_ws_guards(void* ws, const WsLayout& lay, bool check, cudaStream_t st);
 
 constexpr int kRouteSmallC = 256;   // up to this many chunks the router keeps its scores in shared memory
 constexpr int kSmallTileRows = 16;  // query rows of one small tile (two 8-row MMA column blocks)
@@ -127,5 +143,8 @@ int launch_gemv_baseline(const uint16_t* q, const uint16_t* k_shared, const uint
                          const moska_shape* s, cudaStream_t st);
 int launch_merge(const float* o_part, const float* lse_part, uint16_t* out, float* out_f32,
                  float* lse_out, const moska_shape* s, cudaStream_t st);
+int launch_merge_rows(const float* o_part, const float* lse_part, uint16_t* out, float* out_f32,
+                      float* lse_out, const moska_shape* s, long long row0, long long rows,
+                      cudaStream_t st);
 
 }  // namespace moska

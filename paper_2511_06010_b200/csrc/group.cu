@@ -30,24 +30,55 @@ WsLayout ws_layout(const moska_shape* s)
     w.max_small = P / w.small_entries + segs;
     w.max_big = P / w.big_entries + segs;
     size_t off = sizeof(WsHeader);
-    w.off_hist = off;
-    off += round_up(sizeof(uint32_t) * (size_t)w.words * w.n_keys, 256);
-    w.off_totals = off;
-    off += round_up(sizeof(int32_t) * (size_t)w.n_keys, 256);
-    w.off_small = off;
-    off += round_up(sizeof(TileItem) * (size_t)w.max_small, 256);
-    w.off_big = off;
-    off += round_up(sizeof(TileItem) * (size_t)w.max_big, 256);
-    w.off_tiny = off;
-    off += round_up(sizeof(TileItem) * (size_t)segs, 256);  // at most one 8-row tile per segment
+    int r = 0;
+    // a region of `bytes` at the next 256-byte boundary; returns its offset
+    auto region = [&](size_t bytes) {
+        const size_t begin = off;
+        w.guard_begin[r] = begin + round_up(bytes, 4);
+        off += round_up(bytes, 256) + kGuardBytes;
+        w.guard_end[r] = off;
+        ++r;
+        return begin;
+    };
+    w.off_hist = region(sizeof(uint32_t) * (size_t)w.words * w.n_keys);
+    w.off_totals = region(sizeof(int32_t) * (size_t)w.n_keys);
+    w.off_small = region(sizeof(TileItem) * (size_t)w.max_small);
+    w.off_big = region(sizeof(TileItem) * (size_t)w.max_big);
+    w.off_tiny = region(sizeof(TileItem) * (size_t)segs);  // at most one 8-row tile per segment
     w.group_total = off;
     w.off_scores = off;
-    if (s->C > kRouteSmallC) off += round_up(sizeof(float) * (size_t)s->B * s->Hkv * s->C, 256);
+    if (s->C > kRouteSmallC) {
+        region(sizeof(float) * (size_t)s->B * s->Hkv * s->C);
+    } else {
+        w.guard_begin[r] = w.guard_end[r] = off;
+    }
     w.total = off;
     return w;
 }
 
 namespace {
+
+#ifdef MOSKA_DEBUG_GUARDS
+struct GuardRanges {
+    size_t begin[kWsRegions], end[kWsRegions];
+};
+
+__device__ __forceinline__ uint32_t guard_word(size_t byte_offset)
+{
+    return 0xC0DEFACEu ^ static_cast<uint32_t>(byte_offset);
+}
+
+// One CTA per region: writes (check = 0) or compares (check = 1) the region's guard words.
+__global__ void __launch_bounds__(256)
+ws_guard_kernel(uint32_t* __restrict__ ws_words, GuardRanges g, int check, int* __restrict__ status)
+{
+    const int r = blockIdx.x;
+    for (size_t o = g.begin[r] + 4 * (size_t)threadIdx.x; o < g.end[r]; o += 4 * (size_t)blockDim.x) {
+        if (!check) ws_words[o >> 2] = guard_word(o);
+        else if (ws_words[o >> 2] != guard_word(o)) atomicMin(status, (int)MOSKA_ERR_CORRUPT);
+    }
+}
+#endif
 
 // Pass 1: one thread per routed pair p = (b*Hkv + h)*k + j.  Also checks what the bit-set form
 // relies on: every index inside [0, C) and every (b, h) list strictly ascending (hence distinct).
@@ -93,7 +124,8 @@ group_scan_kernel(const uint32_t* __restrict__ bitmap, int words, const int32_t*
                   int32_t* __restrict__ seg_offsets,
                   WsHeader* __restrict__ hdr, TileItem* __restrict__ small_items,
                   TileItem* __restrict__ tiny_items, TileItem* __restrict__ big_items, int n_keys,
-                  int small_entries, int tiny_entries, int big_entries, int tc)
+                  int small_entries, int tiny_entries, int big_entries, int tc, long long max_small,
+                  long long max_big, long long max_tiny, int* __restrict__ status)
 {
     __shared__ int4 warp_sum[32];
     __shared__ int4 carry;
@@ -155,6 +187,13 @@ group_scan_kernel(const uint32_t* __restrict__ bitmap, int words, const int32_t*
         if (key < n_keys) {
             seg_offsets[key] = ex.x;
             int e = ex.x;
+#ifdef MOSKA_DEBUG_GUARDS
+            // the lists' capacities follow from the shape; a write beyond one is reported, not done
+            if (ex.z + n_big > max_big || ex.y + n_small > max_small || ex.w + n_tiny > max_tiny) {
+                atomicMin(status, (int)MOSKA_ERR_CORRUPT);
+                n_big = n_small = n_tiny = 0;
+            }
+#endif
             for (int t = 0; t < n_big; ++t) {
                 const int cnt = min(big_entries, ex.x + n - e);
                 big_items[ex.z + t] = TileItem{key, e, cnt, 0};
@@ -232,6 +271,24 @@ group_emit_kernel(const int32_t* __restrict__ topk_idx, const uint32_t* __restri
 
 }  // namespace
 
+int launch_ws_guards(void* ws, const WsLayout& lay, bool check, cudaStream_t st)
+{
+#ifdef MOSKA_DEBUG_GUARDS
+    GuardRanges g;
+    for (int r = 0; r < kWsRegions; ++r) {
+        g.begin[r] = lay.guard_begin[r];
+        g.end[r] = lay.guard_end[r];
+    }
+    int* status = nullptr;
+    MOSKA_TRY_STATUS(status_word(&status));
+    ws_guard_kernel<<<kWsRegions, 256, 0, st>>>(static_cast<uint32_t*>(ws), g, check ? 1 : 0, status);
+    MOSKA_LAUNCH_CHECK("ws_guard_kernel");
+#else
+    (void)ws; (void)lay; (void)check; (void)st;
+#endif
+    return MOSKA_OK;
+}
+
 int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
                  const moska_shape* s, void* ws, bool premarked, cudaStream_t st)
 {
@@ -247,7 +304,10 @@ int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_ent
     MOSKA_TRY_STATUS(status_word(&status));
     // header and bit sets must start at zero; the router has done both passes already when the
     // two calls run back to back inside moska_decode_step
-    if (!premarked) MOSKA_CUDA_TRY(cudaMemsetAsync(base, 0, lay.off_totals, st));
+    if (!premarked) {
+        MOSKA_CUDA_TRY(cudaMemsetAsync(base, 0, lay.off_totals, st));
+        MOSKA_TRY_STATUS(launch_ws_guards(ws, lay, false, st));
+    }
     if (!premarked && P > 0) {
         group_mark_kernel<<<(unsigned)((P + 255) / 256), 256, 0, st>>>(topk_idx, bitmap, status, P,
                                                                        s->Hkv, s->C, s->k, lay.words);
@@ -261,12 +321,13 @@ int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_ent
     }
     group_scan_kernel<<<1, 1024, 0, st>>>(bitmap, lay.words, totals, seg_offsets, hdr, small_items, tiny_items, big_items,
                                           lay.n_keys, lay.small_entries, lay.tiny_entries,
-                                          lay.big_entries, lay.tc);
+                                          lay.big_entries, lay.tc, lay.max_small, lay.max_big,
+                                          (long long)(P < lay.n_keys ? P : lay.n_keys), status);
     MOSKA_LAUNCH_CHECK("group_scan_kernel");
     group_emit_kernel<<<(lay.n_keys + 7) / 8, 256, 0, st>>>(topk_idx, bitmap, seg_offsets, seg_entries,
                                                             status, lay.n_keys, s->Hkv, s->C, s->k, lay.words);
     MOSKA_LAUNCH_CHECK("group_emit_kernel");
-    return MOSKA_OK;
+    return launch_ws_guards(ws, lay, true, st);
 }
 
 // ---- grouping without any caller- or library-side allocation -----------------------------------

@@ -232,12 +232,18 @@ int launch_summaries_attn(const uint16_t* k_shared, float* summaries, float prob
     return MOSKA_OK;
 }
 
-int launch_merge(const float* o_part, const float* lse_part, uint16_t* out, float* out_f32,
-                 float* lse_out, const moska_shape* s, cudaStream_t st)
+int launch_merge_rows(const float* o_part, const float* lse_part, uint16_t* out, float* out_f32,
+                      float* lse_out, const moska_shape* s, long long row0, long long rows,
+                      cudaStream_t st)
 {
-    const long long rows = (long long)s->B * s->Hq;
     const int n_slots = s->shared_slots + s->n_unique_splits;
-    if (rows == 0) return MOSKA_OK;
+    if (rows <= 0) return MOSKA_OK;
+    // rows [row0, row0 + rows) of every buffer
+    o_part += row0 * n_slots * s->D;
+    lse_part += row0 * n_slots;
+    out += row0 * s->D;
+    if (out_f32 != nullptr) out_f32 += row0 * s->D;
+    if (lse_out != nullptr) lse_out += row0;
     const unsigned grid = (unsigned)((rows + 7) / 8);
     if (s->D == 128)
         merge_kernel<128><<<grid, 256, 0, st>>>(o_part, lse_part, out, out_f32, lse_out, rows, n_slots);
@@ -245,6 +251,12 @@ int launch_merge(const float* o_part, const float* lse_part, uint16_t* out, floa
         merge_kernel<64><<<grid, 256, 0, st>>>(o_part, lse_part, out, out_f32, lse_out, rows, n_slots);
     MOSKA_LAUNCH_CHECK("merge_kernel");
     return MOSKA_OK;
+}
+
+int launch_merge(const float* o_part, const float* lse_part, uint16_t* out, float* out_f32,
+                 float* lse_out, const moska_shape* s, cudaStream_t st)
+{
+    return launch_merge_rows(o_part, lse_part, out, out_f32, lse_out, s, 0, (long long)s->B * s->Hq, st);
 }
 
 int launch_summaries(const uint16_t* k_shared, float* summaries, const moska_shape* s,

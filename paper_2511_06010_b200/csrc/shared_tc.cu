@@ -44,8 +44,12 @@ constexpr int kStages = MOSKA_TC_STAGES;       // K/V ring slots (5 fill the 227
 // FP8 shared store: the tiles arrive as E4M3 codes (16 KB) in a ring of their own and are widened
 // to f16 operand tiles by the two gather warps; fewer operand slots leave room for the codes.
 constexpr int kCodeBytes = 128 * kD;           // one K or V tile of codes
-constexpr int kCodeStages = 4;
-constexpr int kOpStagesF8 = 3;
+#ifndef MOSKA_F8_CODE_STAGES
+#define MOSKA_F8_CODE_STAGES 4
+#define MOSKA_F8_OP_STAGES 3
+#endif
+constexpr int kCodeStages = MOSKA_F8_CODE_STAGES;
+constexpr int kOpStagesF8 = MOSKA_F8_OP_STAGES;
 constexpr int kThreads = 384;                  // 8 softmax warps, TMA warp, MMA warp, 2 gather warps
 constexpr int kLoadWarp = 8, kMmaWarp = 9, kGatherWarp0 = 10;
 // Per-thread register budgets after set-up.  The CTA is launched with kLaunchRegs per thread (the

@@ -469,6 +469,33 @@ def test_host_buffer_step_equals_device_step():
     assert M.device_status() == 0
 
 
+def test_host_buffer_step_with_the_result_copied_in_pieces():
+    """A result of 4 MiB or more leaves the device in pieces, each copied on the side stream while
+    the next rows are merged: same bits as the device-buffer step, ragged last piece included."""
+    M, MoskaLayer = _mods()
+    w = W.scaled(W.CONFIGS[1], B=517, C=8, k=2, unique_len=64)
+    assert w.B * w.Hq * w.D * 2 >= 4 << 20
+    sh = W.make_shared_store(w, "cuda")
+    un = W.make_unique_store(w, "cuda")
+    q = W.make_queries(w, sh, 0, "cuda")
+    layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, 64)
+    layer.build_summaries(sh.k_shared)
+    ref = layer.step(q, sh.k_shared, sh.v_shared, un.k_unique, un.v_unique, un.kv_start, un.kv_len,
+                     two_streams=True).clone()
+    torch.cuda.synchronize()
+    q_dev = torch.empty_like(q)
+    q_host = q.cpu().pin_memory()
+    for two in (True, False):
+        out_host = torch.zeros(w.B, w.Hq, w.D, dtype=torch.bfloat16).pin_memory()
+        layer.out.zero_()
+        for _ in range(2):
+            layer.step_host(q_host, q_dev, out_host, sh.k_shared, sh.v_shared, un.k_unique, un.v_unique,
+                            un.kv_start, un.kv_len, two_streams=two)
+        assert torch.equal(out_host, ref.cpu()), f"two_streams={two}"
+        assert torch.equal(layer.out.cpu(), ref.cpu())
+    assert M.device_status() == 0
+
+
 def test_shared_and_unique_roles_compose_to_the_single_gpu_step():
     """The two roles of the disaggregated step, run one after the other on one GPU with the exchange
     replaced by direct hand-over: the shared role's result, merged over the routed chunks, placed in
