@@ -262,6 +262,8 @@ int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_
  * for moska_shared_attn, none NULL), D = 128; every segment runs on the tensor-core kernel.
  *   k8_shared, v8_shared  uint8 [Hkv][C][L][D]  OCP FP8 E4M3 codes (128-byte aligned)
  *   k_scale, v_scale      float [Hkv][C]        positive
+ *   ws                    as for moska_shared_attn (the grouping's work lists); the call also keeps
+ *                         an f16 copy of q in it, so it WRITES the workspace
  * Chunk embeddings for the router are built from whichever copy of the keys the caller has in
  * bf16 (moska_build_chunk_summaries*); they are an offline step.
  */

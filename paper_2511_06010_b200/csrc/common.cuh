@@ -72,7 +72,7 @@ constexpr size_t kGuardBytes = 256;
 #else
 constexpr size_t kGuardBytes = 0;
 #endif
-constexpr int kWsRegions = 6;  // bit sets, totals, three work lists, router scores
+constexpr int kWsRegions = 7;  // bit sets, totals, three work lists, router scores, f16 queries
 
 struct WsLayout {
     int32_t words;            // 32-bit words of one key's request bit set
@@ -85,6 +85,7 @@ struct WsLayout {
     size_t off_hist, off_totals, off_small, off_big, off_tiny;
     size_t group_total;  // end of what the grouping passes and shared attention use
     size_t off_scores;   // router: fp32 scores [B * Hkv][C] (only when C > kRouteSmallC)
+    size_t off_q16;      // FP8 shared store: the step's queries as f16 [B][Hq][D] (tensor-core shapes)
     size_t total;
     // debug build: guard words fill [guard_begin[r], guard_end[r]) behind region r's payload
     size_t guard_begin[kWsRegions], guard_end[kWsRegions];

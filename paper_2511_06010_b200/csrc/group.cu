@@ -51,6 +51,13 @@ WsLayout ws_layout(const moska_shape* s)
         region(sizeof(float) * (size_t)s->B * s->Hkv * s->C);
     } else {
         w.guard_begin[r] = w.guard_end[r] = off;
+        ++r;
+    }
+    w.off_q16 = off;
+    if (w.tc) {
+        region(sizeof(uint16_t) * (size_t)s->B * s->Hq * s->D);
+    } else {
+        w.guard_begin[r] = w.guard_end[r] = off;
     }
     w.total = off;
     return w;

@@ -91,7 +91,6 @@ struct __align__(1024) TcSmemT<true> {
     uint64_t full[kOpStagesF8], empty[kOpStagesF8];
     uint64_t code_full[kCodeStages], code_empty[kCodeStages];
     uint64_t q_full[2][2], q_free[2][2];
-    uint64_t q_ready[2][2];       // the gathered rows have been converted to f16
     uint64_t s_full[2], p_full[2], o_full[2];
     uint64_t x_full, x_free;
     float stat_m[kBigTileRows];
@@ -344,11 +343,17 @@ __device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_codes)
     return r;
 }
 
-// Two bf16 values (one 32-bit word) to two f16 values, round to nearest.
-__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t w)
+// Four E4M3 codes (one 32-bit word) widened to two f16 pairs: lo = codes 0, 1; hi = codes 2, 3.
+__device__ __forceinline__ void e4m3x4_to_f16x4(uint32_t four_codes, uint32_t& lo, uint32_t& hi)
 {
-    const __half2 h = __floats2half2_rn(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
-    return *reinterpret_cast<const uint32_t*>(&h);
+    asm("{\n"
+        ".reg .b16 c01, c23;\n"
+        "mov.b32 {c01, c23}, %2;\n"
+        "cvt.rn.f16x2.e4m3x2 %0, c01;\n"
+        "cvt.rn.f16x2.e4m3x2 %1, c23;\n"
+        "}\n"
+        : "=r"(lo), "=r"(hi)
+        : "r"(four_codes));
 }
 
 template <bool F>
@@ -418,9 +423,9 @@ __device__ __forceinline__ void other_roles(TcSmemT<F>& sm, const CUtensorMap& t
         // (lane l owns tile rows 4l .. 4l+3), so the copies do not queue behind the softmax
         // groups' result stores in the load/store pipe.  Rows past the item's last one hold
         // stale or repeated query rows; their results are never written.
-        // FP8 store: the same warp then converts the gathered rows to f16 in place and, together with
-        // the other gather warp (64 token rows each), widens the unit's code tiles into the operand
-        // ring.
+        // FP8 store: the rows come from an f16 copy of the queries; once the unit's gather is on its
+        // way the same warp, together with the other gather warp (64 token rows each), widens the
+        // unit's code tiles into the operand ring.
         const int u = warp - kGatherWarp0;
         uint32_t n_small = 0;
         uint32_t arrivals[2] = {0, 0};  // uses of sub-buffer 0 / 1 so far (a full tile uses both)
@@ -429,7 +434,25 @@ __device__ __forceinline__ void other_roles(TcSmemT<F>& sm, const CUtensorMap& t
         uint32_t fills[2] = {0, 0};     // gathers signalled on q_full[u][0 / 1] so far
         uint32_t cv = 0;                // FP8 store: code tiles widened so far, over all units
         bool ok = true;
-        // FP8 store: widens this warp's half (64 token rows) of every code tile of the unit
+        // FP8 store: widens this warp's half (64 token rows) of every code tile of the unit.  In
+        // step i the warp handles token rows R .. R+3, R = 64u + 4i, every lane 16 codes (dims
+        // 16j .. 16j+15) of one row.  Both tiles carry the 128-byte swizzle (phase = row % 8, which
+        // is one of two values per lane: even and odd steps).  A quarter warp (what one 16-byte
+        // shared-memory access serves at a time) holds dims 0..63 of one row and dims 64..127 of
+        // the next, so that its eight loads and its eight stores each fall on eight different
+        // 16-byte bank groups.  The 16 values are pieces 2 (j % 4) and 2 (j % 4) + 1 of the row's
+        // half j / 4 of the operand tile.
+        uint32_t w_src[2], w_dst[2];
+        {
+            const int qw = lane >> 3, t = (lane >> 2) & 1, m = lane & 3;
+            const int a0 = 2 * (qw >> 1) + t, j = 4 * (t ^ (qw & 1)) + m, r0 = u * 64 + a0;
+#pragma unroll
+            for (int ph = 0; ph < 2; ++ph) {
+                const int a = a0 ^ (4 * ph);
+                w_src[ph] = r0 * 128 + ((j ^ a) << 4);
+                w_dst[ph] = (j >> 2) * kHalfBytes + r0 * 128 + (((2 * (j & 3)) ^ a) << 4);
+            }
+        }
         auto widen_unit = [&](const Unit& it) {
             if constexpr (F) {
                 const int n_loads = (it.mode == kPair ? 4 : 2) * it.n_kv;
@@ -441,25 +464,19 @@ __device__ __forceinline__ void other_roles(TcSmemT<F>& sm, const CUtensorMap& t
                     if (!ok) break;
                     const uint8_t* src = sm.codes[cs];
                     uint8_t* dst = sm.kv[os];
-#pragma unroll 4
+                    // 16 steps of four token rows; every address is a per-lane base (one for each
+                    // of the two swizzle phases a lane's rows alternate between) plus a constant
+#pragma unroll
                     for (int i = 0; i < 16; ++i) {
-                        const int idx = i * 32 + lane;
-                        const int row = u * 64 + (idx >> 3), j = idx & 7;  // 16 codes: dims 16j .. 16j+15
-                        const uint4 c = *reinterpret_cast<const uint4*>(src + row * 128 + ((j ^ (row & 7)) << 4));
+                        const int ph = i & 1;
+                        const uint4 c = *reinterpret_cast<const uint4*>(src + w_src[ph] + i * 512);
                         uint4 lo, hi;
-                        lo.x = e4m3x2_to_f16x2(c.x);
-                        lo.y = e4m3x2_to_f16x2(c.x >> 16);
-                        lo.z = e4m3x2_to_f16x2(c.y);
-                        lo.w = e4m3x2_to_f16x2(c.y >> 16);
-                        hi.x = e4m3x2_to_f16x2(c.z);
-                        hi.y = e4m3x2_to_f16x2(c.z >> 16);
-                        hi.z = e4m3x2_to_f16x2(c.w);
-                        hi.w = e4m3x2_to_f16x2(c.w >> 16);
-                        // the 16 values are pieces 2 (j % 4) and 2 (j % 4) + 1 of the row's half j / 4
-                        uint8_t* drow = dst + (j >> 2) * kHalfBytes + row * 128;
-                        const int c0 = 2 * (j & 3);
-                        *reinterpret_cast<uint4*>(drow + ((c0 ^ (row & 7)) << 4)) = lo;
-                        *reinterpret_cast<uint4*>(drow + (((c0 + 1) ^ (row & 7)) << 4)) = hi;
+                        e4m3x4_to_f16x4(c.x, lo.x, lo.y);
+                        e4m3x4_to_f16x4(c.y, lo.z, lo.w);
+                        e4m3x4_to_f16x4(c.z, hi.x, hi.y);
+                        e4m3x4_to_f16x4(c.w, hi.z, hi.w);
+                        *reinterpret_cast<uint4*>(dst + w_dst[ph] + i * 512) = lo;
+                        *reinterpret_cast<uint4*>(dst + (w_dst[ph] ^ 16) + i * 512) = hi;
                     }
                     fence_proxy_async_smem();
                     __syncwarp();
@@ -517,29 +534,7 @@ __device__ __forceinline__ void other_roles(TcSmemT<F>& sm, const CUtensorMap& t
                 tma_gather4_2d(dst, &tm_q, 0, rr[0], rr[1], rr[2], rr[3], bar);
                 tma_gather4_2d(dst + half, &tm_q, 64, rr[0], rr[1], rr[2], rr[3], bar);
             }
-            if constexpr (F) {
-                // the rows have landed: bf16 -> f16 in place (the copied groups only), then tell
-                // the MMA warp
-                ok = __all_sync(0xffffffffu, mbar_wait(bar, last_phase, ab));
-                if (!ok) break;
-                uint8_t* base = sm.q[u] + (qu.small ? qu.sub * kSubBytes : 0);
-                const int half = qu.small ? kSubBytes / 2 : kHalfBytes;
-                const int n_pieces = n_groups * 4 * 8;  // 16-byte pieces per half
-                for (int i = lane; i < 2 * n_pieces; i += 32) {
-                    uint4* ptr = reinterpret_cast<uint4*>(base + (i >= n_pieces ? half : 0) +
-                                                          (i % n_pieces) * 16);
-                    uint4 v = *ptr;
-                    v.x = bf16x2_to_f16x2(v.x);
-                    v.y = bf16x2_to_f16x2(v.y);
-                    v.z = bf16x2_to_f16x2(v.z);
-                    v.w = bf16x2_to_f16x2(v.w);
-                    *ptr = v;
-                }
-                fence_proxy_async_smem();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.q_ready[u][qu.sub]);
-                widen_unit(it);
-            }
+            widen_unit(it);
         }
         if (*ab && last_full != nullptr) {
             // giving up: let the copies still in flight land before the CTA leaves
@@ -625,7 +620,7 @@ __device__ __forceinline__ void other_roles(TcSmemT<F>& sm, const CUtensorMap& t
                 for (int u = 0; u < 2 && ok; ++u) {
                     if (!qu[u].present) continue;
                     uint64_t* bar;
-                    if constexpr (F) bar = &sm.q_ready[u][qu[u].sub]; else bar = &sm.q_full[u][qu[u].sub];
+                    bar = &sm.q_full[u][qu[u].sub];
                     ok = mbar_wait(bar, fills[u][qu[u].sub]++ & 1, ab);
                 }
                 // first scores of both slots
@@ -667,6 +662,25 @@ __device__ __forceinline__ void other_roles(TcSmemT<F>& sm, const CUtensorMap& t
     }
 }
 
+// FP8 shared store: the step's queries as f16 (the operand type of its MMAs), eight values per
+// thread; round to nearest.
+__global__ void __launch_bounds__(256)
+q_to_f16_kernel(const uint4* __restrict__ q, uint4* __restrict__ q16, long long n_vec)
+{
+    const long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= n_vec) return;
+    uint4 v = q[i];
+    auto cv = [](uint32_t w) {
+        const __half2 h = __floats2half2_rn(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+        return *reinterpret_cast<const uint32_t*>(&h);
+    };
+    v.x = cv(v.x);
+    v.y = cv(v.y);
+    v.z = cv(v.z);
+    v.w = cv(v.w);
+    q16[i] = v;
+}
+
 template <bool F>
 __global__ void __launch_bounds__(kThreads, 1)
 shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant__ CUtensorMap tm_v,
@@ -693,8 +707,6 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 mbar_init(&sm.code_full[s], 1);
                 mbar_init(&sm.code_empty[s], 2);
             }
-            for (int u = 0; u < 2; ++u)
-                for (int sb = 0; sb < 2; ++sb) mbar_init(&sm.q_ready[u][sb], 1);
         }
         for (int u = 0; u < 2; ++u) {
             for (int sb = 0; sb < 2; ++sb) {
@@ -1070,7 +1082,17 @@ int launch_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_sha
         MOSKA_TRY_STATUS(make_kv_map(&tm_k, k_shared, kv_rows));
         MOSKA_TRY_STATUS(make_kv_map(&tm_v, v_shared, kv_rows));
     }
-    MOSKA_TRY_STATUS(make_q_map(&tm_q, q, (long long)s->B * s->Hq));
+    const uint16_t* q_rows = q;
+    if (fp8) {
+        // the gathers read an f16 copy of the queries kept in the workspace
+        const long long n_vec = (long long)s->B * s->Hq * kD / 8;
+        uint16_t* q16 = reinterpret_cast<uint16_t*>(static_cast<char*>(ws) + ws_layout(s).off_q16);
+        q_to_f16_kernel<<<(unsigned)((n_vec + 255) / 256), 256, 0, st>>>(
+            reinterpret_cast<const uint4*>(q), reinterpret_cast<uint4*>(q16), n_vec);
+        MOSKA_LAUNCH_CHECK("q_to_f16_kernel");
+        q_rows = q16;
+    }
+    MOSKA_TRY_STATUS(make_q_map(&tm_q, q_rows, (long long)s->B * s->Hq));
     int* status = nullptr;
     MOSKA_TRY_STATUS(status_word(&status));
     p.q = q;

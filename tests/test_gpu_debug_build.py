@@ -28,7 +28,7 @@ def test_debug_library_exports_the_same_symbols_and_a_larger_workspace(libs):
     for lib in (regular, debug):
         lib.moska_workspace_bytes.restype = ctypes.c_size_t
     extra = debug.moska_workspace_bytes(ctypes.byref(s)) - regular.moska_workspace_bytes(ctypes.byref(s))
-    assert extra == 6 * 256  # bit sets, totals, three work lists, router scores (C > 256)
+    assert extra == 7 * 256  # bit sets, totals, three work lists, router scores (C > 256), f16 queries
     # the regular build has no guard words to compare
     regular.moska_debug_check_workspace.restype = ctypes.c_int
     rc = regular.moska_debug_check_workspace(None, ctypes.c_size_t(0), ctypes.byref(s), None)
