@@ -352,8 +352,8 @@ def measure(args, w_full, rank, world, dev, headline: bool):
         f8 = W.quantize_unique_store_fp8(un, release=True)
         torch.cuda.empty_cache()
     sfp8 = args.shared_kv == "fp8"
-    if sfp8 and (w.D != 128 or w.dense or fp8 or T > 1):
-        raise SystemExit("--shared-kv fp8 needs head dimension 128, routed mode, the bf16 private store and q_len 1")
+    if sfp8 and (w.D != 128 or w.dense or T > 1):
+        raise SystemExit("--shared-kv fp8 needs head dimension 128, routed mode and q_len 1")
     n_q = max(1, w.steps)
     qs = [W.make_queries(w, sh, s, dev) for s in range(n_q)]
     kv_lens = [(un.kv_len + s).to(torch.int32) for s in range(n_q)]
@@ -382,7 +382,10 @@ def measure(args, w_full, rank, world, dev, headline: bool):
 
     def step(i, prof=None):
         s = i % n_q
-        if sfp8:
+        if sfp8 and fp8:
+            layer.step_fp8(qs[s], sf8, f8, un.kv_start, kv_lens[s], two_streams=two_streams, prof=prof,
+                           unique_tokens=tokens[s])
+        elif sfp8:
             layer.step_fp8shared(qs[s], sf8, un.k_unique, un.v_unique, un.kv_start, kv_lens[s],
                                  two_streams=two_streams, prof=prof, unique_tokens=tokens[s])
         elif fp8:
@@ -399,7 +402,10 @@ def measure(args, w_full, rank, world, dev, headline: bool):
         if fp8 or sfp8:
             # no host-buffer entry point for the FP8 stores: the same copies around the device call
             q_dev.copy_(q_host[s], non_blocking=True)
-            if sfp8:
+            if sfp8 and fp8:
+                out = layer.step_fp8(q_dev, sf8, f8, un.kv_start, kv_lens[s], two_streams=two_streams,
+                                     unique_tokens=tokens[s])
+            elif sfp8:
                 out = layer.step_fp8shared(q_dev, sf8, un.k_unique, un.v_unique, un.kv_start, kv_lens[s],
                                            two_streams=two_streams, unique_tokens=tokens[s])
             else:
@@ -622,9 +628,9 @@ def measure(args, w_full, rank, world, dev, headline: bool):
     rows_merge_bytes = w.B * w.Hq * ((S.shared_slots + S.n_unique_splits) * (w.D + 1) * 4 + w.D * 2)
     # kernels of one step: route (scoring + selection beyond 256 chunks), 2-3 grouping passes, unique,
     # shared, merge
-    # the tensor-core kernel and the 8-row streaming tiles (FP8 store: the tensor-core kernel alone), or
-    # 16-row and 8-row tiles
-    n_shared_launches = 1 if sfp8 else 2
+    # the tensor-core kernel and the 8-row streaming tiles (FP8 shared store: plus the query
+    # conversion), or 16-row and 8-row tiles
+    n_shared_launches = 3 if sfp8 else 2
     n_launch = 3 if w.dense else (1 + (w.C > 256)) + (3 if w.B > 64 else 2) + 1 + n_shared_launches + 1
     hbm_bytes = work["unique_bytes"] + work["shared_bytes"] + rows_merge_bytes
     amort = P / max(1, touched)

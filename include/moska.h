@@ -259,7 +259,8 @@ int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_
  * scale and the value scale the final normalisation.  The code tiles arrive by TMA (half the bytes
  * of the bf16 store), are widened exactly to f16 in shared memory and multiplied on the tensor cores
  * with f16 Q and P and fp32 accumulation.  Routed mode only (topk_idx, seg_offsets, seg_entries as
- * for moska_shared_attn, none NULL), D = 128; every segment runs on the tensor-core kernel.
+ * for moska_shared_attn, none NULL), D = 128.  Segments of at most 8 query rows are streamed by a
+ * kernel of their own (codes widened in registers, f16 warp MMAs), as with the bf16 store.
  *   k8_shared, v8_shared  uint8 [Hkv][C][L][D]  OCP FP8 E4M3 codes (128-byte aligned)
  *   k_scale, v_scale      float [Hkv][C]        positive
  *   ws                    as for moska_shared_attn (the grouping's work lists); the call also keeps
@@ -387,6 +388,22 @@ int moska_decode_step_fp8shared(const uint16_t* q, const float* summaries, const
                                 float* o_part, float* lse_part, uint16_t* out, float* lse_out,
                                 float softmax_scale, const moska_shape* shape, void* ws, size_t ws_bytes,
                                 moska_stream stream, moska_stream side_stream, moska_profiler* prof);
+
+/*
+ * moska_decode_step with BOTH stores in FP8, the KV precision of the paper's evaluation (Section
+ * IV) on the whole path: the shared store as for moska_shared_attn_fp8 (one scale per (KV head,
+ * chunk)), the private store as for moska_unique_attn_fp8 (one scale per (token, KV head)).  Same
+ * schedule, buffers, outputs and error behaviour as moska_decode_step; routed mode only (summaries
+ * must not be NULL), D = 128.
+ */
+int moska_decode_step_fp8(const uint16_t* q, const float* summaries, const uint8_t* k8_shared,
+                          const uint8_t* v8_shared, const float* k_scale_shared, const float* v_scale_shared,
+                          const uint8_t* k8_unique, const uint8_t* v8_unique, const float* k_scale_unique,
+                          const float* v_scale_unique, const int64_t* kv_start, const int32_t* kv_len,
+                          int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries, float* o_part,
+                          float* lse_part, uint16_t* out, float* lse_out, float softmax_scale,
+                          const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream,
+                          moska_stream side_stream, moska_profiler* prof);
 
 /*
  * moska_decode_step for a caller whose step inputs live in HOST memory: copies q_host (bf16

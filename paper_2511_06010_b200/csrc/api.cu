@@ -379,8 +379,11 @@ int moska_shared_attn_fp8(const uint16_t* q, const uint8_t* k8_shared, const uin
         return fail(MOSKA_ERR_WORKSPACE, "workspace missing, misaligned or smaller than %zu bytes",
                     ws_layout(shape).total);
     MOSKA_TRY(check_device());
-    return launch_shared_tc_fp8(q, k8_shared, v8_shared, k_scale, v_scale, seg_entries, o_part, lse_part,
-                                softmax_scale, shape, ws, 0, (cudaStream_t)stream);
+    // segments of more than 8 rows on the tensor-core kernel, the 8-row tiles streamed
+    MOSKA_TRY(launch_shared_tc_fp8(q, k8_shared, v8_shared, k_scale, v_scale, seg_entries, o_part, lse_part,
+                                   softmax_scale, shape, ws, 0, (cudaStream_t)stream));
+    return launch_shared_small_fp8(q, k8_shared, v8_shared, k_scale, v_scale, seg_entries, o_part,
+                                   lse_part, softmax_scale, shape, ws, (cudaStream_t)stream);
 }
 
 int moska_device_status(int32_t* status_host)
@@ -637,9 +640,11 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
         const bool beside = tc && (dense || unique_ms >= MOSKA_BESIDE_MS);
         if (tc && beside) MOSKA_TRY(shared_tc(dense, tc_sm_share(shape, dense, unique_ms), side));
         // the streaming tiles (every tile of a shape the tensor-core kernel does not serve, else the
-        // 8-row tiles of routed mode) always run beside unique attention; with the FP8 store the
-        // tensor-core kernel takes those items as well
-        if ((!tc || !dense) && f8 == nullptr)
+        // 8-row tiles of routed mode) always run beside unique attention
+        if (f8 != nullptr)
+            MOSKA_TRY(launch_shared_small_fp8(q, f8->k8, f8->v8, f8->k_scale, f8->v_scale, seg_entries,
+                                              o_part, lse_part, softmax_scale, shape, ws, side));
+        else if (!tc || !dense)
             MOSKA_TRY(launch_shared_small(q, k_shared, v_shared, dense ? nullptr : seg_entries, o_part,
                                           lse_part, softmax_scale, shape, ws, dense, tc, side));
         if (beside || !tc) MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, side));
@@ -716,6 +721,34 @@ int moska_decode_step_fp8shared(const uint16_t* q, const float* summaries, const
     UniqueKv kv;
     kv.k = k_unique;
     kv.v = v_unique;
+    SharedF8 f8;
+    f8.k8 = k8_shared;
+    f8.v8 = v8_shared;
+    f8.k_scale = k_scale_shared;
+    f8.v_scale = v_scale_shared;
+    return decode_step_impl(q, summaries, nullptr, nullptr, &f8, kv, kv_start, kv_len, topk_idx, seg_offsets,
+                            seg_entries, o_part, lse_part, out, lse_out, softmax_scale, shape, ws, ws_bytes,
+                            stream, side_stream, prof);
+}
+
+int moska_decode_step_fp8(const uint16_t* q, const float* summaries, const uint8_t* k8_shared,
+                          const uint8_t* v8_shared, const float* k_scale_shared, const float* v_scale_shared,
+                          const uint8_t* k8_unique, const uint8_t* v8_unique, const float* k_scale_unique,
+                          const float* v_scale_unique, const int64_t* kv_start, const int32_t* kv_len,
+                          int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries, float* o_part,
+                          float* lse_part, uint16_t* out, float* lse_out, float softmax_scale,
+                          const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream,
+                          moska_stream side_stream, moska_profiler* prof)
+{
+    MOSKA_API_RANGE();
+    if (summaries == nullptr)
+        return fail(MOSKA_ERR_UNSUPPORTED, "the FP8 shared store is built for routed mode (no dense mode)");
+    UniqueKv kv;
+    kv.k8 = k8_unique;
+    kv.v8 = v8_unique;
+    kv.k_scale = k_scale_unique;
+    kv.v_scale = v_scale_unique;
+    kv.fp8 = true;
     SharedF8 f8;
     f8.k8 = k8_shared;
     f8.v8 = v8_shared;

@@ -135,6 +135,10 @@ int read_status(int* out);
 int launch_unique(const uint16_t* q, const uint16_t* k_unique, const uint16_t* v_unique,
                   const int64_t* kv_start, const int32_t* kv_len, float* o_part, float* lse_part,
                   float scale, const moska_shape* s, cudaStream_t st);
+// FP8 shared store: the grouping pass's 8-row tiles on the streaming block (routed mode)
+int launch_shared_small_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v8, const float* k_scale,
+                            const float* v_scale, const int32_t* seg_entries, float* o_part,
+                            float* lse_part, float scale, const moska_shape* s, void* ws, cudaStream_t st);
 int launch_unique_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v8, const float* k_scale,
                       const float* v_scale, const int64_t* kv_start, const int32_t* kv_len,
                       float* o_part, float* lse_part, float scale, const moska_shape* s,

@@ -108,7 +108,6 @@ struct TcParams {
     const WsHeader* hdr;
     const TileItem* items;    // items of two query tiles (more than 128 rows)
     const TileItem* singles;  // items of one query tile
-    const TileItem* tiny;     // FP8 store: the 8-row items as well (further single-tile items)
     const float* k_scale;     // FP8 store: scale per (KV head, chunk) of the keys / values
     const float* v_scale;
     float* o_part;
@@ -214,19 +213,17 @@ __device__ __forceinline__ Schedule make_schedule(const TcParams& p)
         s.n_units = p.n_items_dense;
     } else {
         s.n_two = p.hdr->n_big_tiles;
-        const int n1 = p.hdr->n_small_tiles + (p.tiny != nullptr ? p.hdr->n_tiny_tiles : 0);
+        const int n1 = p.hdr->n_small_tiles;
         s.n_pairs = (n1 / (2 * (int)gridDim.x)) * (int)gridDim.x;
         s.n_units = s.n_two + s.n_pairs + (n1 - 2 * s.n_pairs);
     }
     return s;
 }
 
-// i-th single-tile item: the second work list, then (FP8 store) the third
+// i-th single-tile item (the second work list)
 __device__ __forceinline__ int4 single_item(const TcParams& p, int i)
 {
-    const int n_small = p.hdr->n_small_tiles;
-    const TileItem* src = i < n_small ? p.singles + i : p.tiny + (i - n_small);
-    return __ldg(reinterpret_cast<const int4*>(src));
+    return __ldg(reinterpret_cast<const int4*>(p.singles + i));
 }
 
 __device__ __forceinline__ Unit decode_unit(const TcParams& p, const Schedule& sch, int unit, int G,
@@ -1042,7 +1039,7 @@ int make_code_map(CUtensorMap* tm, const uint8_t* base, long long rows)
 }
 
 // Common part of the two launchers.  k8 / v8 != nullptr selects the FP8 shared store (routed mode
-// only; every single-tile item, the 8-row ones included, runs on this kernel then).
+// only).
 int launch_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared, const uint8_t* k8,
               const uint8_t* v8, const float* k_scale, const float* v_scale, const int32_t* seg_entries,
               float* o_part, float* lse_part, float scale, const moska_shape* s, void* ws, bool dense,
@@ -1062,7 +1059,6 @@ int launch_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_sha
         p.hdr = reinterpret_cast<const WsHeader*>(ws);
         p.items = reinterpret_cast<const TileItem*>(static_cast<const char*>(ws) + lay.off_big);
         p.singles = reinterpret_cast<const TileItem*>(static_cast<const char*>(ws) + lay.off_small);
-        if (fp8) p.tiny = reinterpret_cast<const TileItem*>(static_cast<const char*>(ws) + lay.off_tiny);
     }
     if (grid == 0) return MOSKA_OK;
     if (grid > 0x7fffffffLL) return fail(MOSKA_ERR_UNSUPPORTED, "shared attention grid too large");

@@ -132,6 +132,19 @@ class MoskaLayer:
                                 self.ws, None, self.side_stream if two_streams else None, prof)
         return self.out
 
+    def step_fp8(self, q, sf8, f8, kv_start, kv_len, two_streams=False, prof=None, unique_tokens=0):
+        """One decode step with both stores in FP8 (`sf8`: shared codes and per-chunk scales, `f8`:
+        private codes and per-token scales)."""
+        self.shape.unique_tokens = int(unique_tokens)
+        two_streams = two_streams and self.overlap_routing
+        if two_streams and self.side_stream is None:
+            self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
+        M.decode_step_fp8(q, self.summaries, sf8.k8, sf8.v8, sf8.k_scale, sf8.v_scale, f8.k8, f8.v8,
+                          f8.k_scale, f8.v_scale, kv_start, kv_len, self.topk_idx, self.seg_offsets,
+                          self.seg_entries, self.o_part, self.lse_part, self.out, self.lse_out, self.scale,
+                          self.shape, self.ws, None, self.side_stream if two_streams else None, prof)
+        return self.out
+
     def bind_step_host(self, q_host, q_dev, out_host, k_shared, v_shared, k_unique, v_unique,
                        kv_start, kv_len, two_streams=False, unique_tokens=0):
         """step_host for a loop over fixed buffers: marshals the arguments once and returns a

@@ -78,6 +78,41 @@ def test_fp8_shared_full_cfg1_sampled_two_streams():
           unique_tokens=w.B * w.unique_len)
 
 
+def test_decode_step_with_both_stores_in_fp8():
+    """moska_decode_step_fp8: shared codes with per-chunk scales, private codes with per-token scales;
+    the oracle merges its FP8 shared partials with its FP8 private-store attention.  One and two
+    streams; segments on every work list; empty and ragged private contexts."""
+    M, MoskaLayer = _mods()
+    lens = np.array([300, 1, 0, 1000, 64, 17, 129, 511, 2048, 77, 5, 900, 33, 640, 256, 4], dtype=np.int64)
+    for B, C, k in ((16, 16, 4), (80, 4, 2)):
+        w = W.scaled(W.CONFIGS[1], B=B, C=C, k=k, unique_len=0)
+        sh = W.make_shared_store(w, "cuda")
+        un = W.make_unique_store(w, "cuda", np.resize(lens, B))
+        q = W.make_queries(w, sh, 0, "cuda")
+        sf8 = W.quantize_shared_store_fp8(sh)
+        kv_start, kv_len = un.kv_start, un.kv_len
+        f8 = W.quantize_unique_store_fp8(un)
+        layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, int(lens.max()), n_unique_splits=3,
+                           fp8_unique=True)
+        layer.build_summaries(sh.k_shared)
+        for two in (False, True):
+            layer.out.zero_()
+            out = layer.step_fp8(q, sf8, f8, kv_start, kv_len, two_streams=two,
+                                 unique_tokens=int(kv_len.sum().item())).clone()
+            torch.cuda.synchronize()
+            topk = layer.topk_idx.cpu().numpy()
+            o_sh, l_sh = O.shared_partials_fp8(q.cpu(), sf8.k8.cpu(), sf8.v8.cpu(), sf8.k_scale.cpu(),
+                                               sf8.v_scale.cpu(), topk, layer.scale)
+            o_u, l_u = O.attend_unique_fp8(q.cpu(), f8.k8.cpu(), f8.v8.cpu(), f8.k_scale.cpu(),
+                                           f8.v_scale.cpu(), kv_start.cpu().numpy(), kv_len.cpu().numpy(),
+                                           layer.scale)
+            want, want_lse = O.merge(np.concatenate([o_sh, o_u[:, :, None, :]], axis=2),
+                                     np.concatenate([l_sh, l_u[:, :, None]], axis=2))
+            PU.check_attention(out.float().cpu().numpy(), want, f"all-fp8 decode step out (two_streams={two})")
+            PU.check_lse(layer.lse_out.cpu().numpy(), want_lse, "all-fp8 decode step lse")
+            assert M.device_status() == 0
+
+
 def test_fp8_shared_rejects_what_it_does_not_serve():
     M, MoskaLayer = _mods()
     layer = MoskaLayer(4, 4, 1, 64, 8, 128, 2, 16)          # D = 64
