@@ -117,8 +117,10 @@ int moska_device_status(int32_t* status_host);
 /* n_slots = shared_slots + n_unique_splits; negative status if the shape is invalid. Host only. */
 int moska_partial_slots(const moska_shape* shape);
 
-/* Bytes of workspace that moska_route / moska_group_by_chunk / moska_shared_attn need for this
- * shape (one workspace serves all three; 256-byte aligned base required).  Host only, pure.   */
+/* Bytes of workspace that moska_route / moska_group_by_chunk / moska_shared_attn[_fp8] need for
+ * this shape (one workspace serves all of them; 256-byte aligned base required): the grouping's bit
+ * sets and work lists, the router's scores beyond 256 chunks, and, for D = 128, room for an f16
+ * copy of the queries (B*Hq*D*2 bytes, used by the FP8 shared store only).  Host only, pure.  */
 size_t moska_workspace_bytes(const moska_shape* shape);
 
 /* A reasonable n_unique_splits for a batch whose longest unique context has `max_len` tokens.
