@@ -400,12 +400,18 @@ def measure(args, w_full, rank, world, dev, headline: bool):
     def step_host(i):
         s = i % n_q
         if fp8 or sfp8:
-            # no host-buffer entry point for the FP8 stores: the same copies around the device call
-            q_dev.copy_(q_host[s], non_blocking=True)
+            # one store in FP8: no host-buffer entry point, the same copies around the device call
             if sfp8 and fp8:
-                out = layer.step_fp8(q_dev, sf8, f8, un.kv_start, kv_lens[s], two_streams=two_streams,
-                                     unique_tokens=tokens[s])
-            elif sfp8:
+                # both stores in FP8: the host-buffer entry point of that step
+                if s not in bound_host:
+                    bound_host[s] = layer.bind_step_fp8_host(q_host[s], q_dev, out_host, sf8, f8, un.kv_start,
+                                                             kv_lens[s], two_streams=two_streams,
+                                                             unique_tokens=tokens[s])
+                layer.shape.unique_tokens = tokens[s]
+                bound_host[s]()
+                return
+            q_dev.copy_(q_host[s], non_blocking=True)
+            if sfp8:
                 out = layer.step_fp8shared(q_dev, sf8, un.k_unique, un.v_unique, un.kv_start, kv_lens[s],
                                            two_streams=two_streams, unique_tokens=tokens[s])
             else:

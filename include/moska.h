@@ -428,6 +428,23 @@ int moska_decode_step_host(const uint16_t* q_host, uint16_t* q_dev, const float*
                            size_t ws_bytes, moska_stream stream, moska_stream side_stream,
                            moska_profiler* prof);
 
+/*
+ * moska_decode_step_fp8 (both stores in FP8, Section IV's precision) for a caller whose step inputs
+ * live in HOST memory: q_host in, out_host out, the call returns when the result is there.  Copies,
+ * their overlap with the step and the conditions on the host buffers are those of
+ * moska_decode_step_host.
+ */
+int moska_decode_step_fp8_host(const uint16_t* q_host, uint16_t* q_dev, const float* summaries,
+                               const uint8_t* k8_shared, const uint8_t* v8_shared,
+                               const float* k_scale_shared, const float* v_scale_shared,
+                               const uint8_t* k8_unique, const uint8_t* v8_unique,
+                               const float* k_scale_unique, const float* v_scale_unique,
+                               const int64_t* kv_start, const int32_t* kv_len, int32_t* topk_idx,
+                               int32_t* seg_offsets, int32_t* seg_entries, float* o_part, float* lse_part,
+                               uint16_t* out_dev, uint16_t* out_host, float softmax_scale,
+                               const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream,
+                               moska_stream side_stream, moska_profiler* prof);
+
 #ifdef __cplusplus
 }
 #endif

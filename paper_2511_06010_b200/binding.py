@@ -67,6 +67,7 @@ EXPORTS = {
     "moska_decode_step_fp8shared": (_i, [_vp] * 17 + [_f, _sp, _vp, _sz, _vp, _vp, _vp]),
     "moska_decode_step_fp8": (_i, [_vp] * 19 + [_f, _sp, _vp, _sz, _vp, _vp, _vp]),
     "moska_decode_step_host": (_i, [_vp] * 16 + [_f, _sp, _vp, _sz, _vp, _vp, _vp]),
+    "moska_decode_step_fp8_host": (_i, [_vp] * 20 + [_f, _sp, _vp, _sz, _vp, _vp, _vp]),
     "moska_profiler_create": (_i, [ctypes.POINTER(_vp), ctypes.c_int32]),
     "moska_profiler_destroy": (None, [_vp]),
     "moska_profiler_select": (_i, [_vp, ctypes.c_uint32]),
@@ -305,6 +306,42 @@ def bind_decode_step_host(q_host, q_dev, summaries, k_shared, v_shared, k_unique
         status = fn(*args)
         if status != OK:
             raise MoskaError(status, "moska_decode_step_host")
+
+    return call
+
+
+def decode_step_fp8_host(q_host, q_dev, summaries, k8_shared, v8_shared, k_scale_shared, v_scale_shared,
+                         k8_unique, v8_unique, k_scale_unique, v_scale_unique, kv_start, kv_len, topk_idx,
+                         seg_offsets, seg_entries, o_part, lse_part, out_dev, out_host, softmax_scale, s, ws,
+                         stream=None, side_stream=None, prof=None) -> None:
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    _check(_lib.moska_decode_step_fp8_host(
+        _ptr(q_host), _ptr(q_dev), _ptr(summaries), _ptr(k8_shared), _ptr(v8_shared), _ptr(k_scale_shared),
+        _ptr(v_scale_shared), _ptr(k8_unique), _ptr(v8_unique), _ptr(k_scale_unique), _ptr(v_scale_unique),
+        _ptr(kv_start), _ptr(kv_len), _ptr(topk_idx), _ptr(seg_offsets), _ptr(seg_entries), _ptr(o_part),
+        _ptr(lse_part), _ptr(out_dev), _ptr(out_host), softmax_scale, ctypes.byref(s), _ptr(ws), ws_bytes,
+        _stream(stream), None if side_stream is None else _stream(side_stream), prof),
+        "moska_decode_step_fp8_host")
+
+
+def bind_decode_step_fp8_host(q_host, q_dev, summaries, k8_shared, v8_shared, k_scale_shared, v_scale_shared,
+                              k8_unique, v8_unique, k_scale_unique, v_scale_unique, kv_start, kv_len,
+                              topk_idx, seg_offsets, seg_entries, o_part, lse_part, out_dev, out_host,
+                              softmax_scale, s, ws, stream=None, side_stream=None, prof=None):
+    """decode_step_fp8_host with its arguments marshalled once (see bind_decode_step_host)."""
+    ws_bytes = 0 if ws is None else ws.numel() * ws.element_size()
+    args = (_ptr(q_host), _ptr(q_dev), _ptr(summaries), _ptr(k8_shared), _ptr(v8_shared),
+            _ptr(k_scale_shared), _ptr(v_scale_shared), _ptr(k8_unique), _ptr(v8_unique),
+            _ptr(k_scale_unique), _ptr(v_scale_unique), _ptr(kv_start), _ptr(kv_len), _ptr(topk_idx),
+            _ptr(seg_offsets), _ptr(seg_entries), _ptr(o_part), _ptr(lse_part), _ptr(out_dev),
+            _ptr(out_host), softmax_scale, ctypes.byref(s), _ptr(ws), ws_bytes, _stream(stream),
+            None if side_stream is None else _stream(side_stream), prof)
+    fn = _lib.moska_decode_step_fp8_host
+
+    def call() -> None:
+        status = fn(*args)
+        if status != OK:
+            raise MoskaError(status, "moska_decode_step_fp8_host")
 
     return call
 

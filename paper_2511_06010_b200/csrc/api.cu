@@ -864,4 +864,41 @@ int moska_decode_step_host(const uint16_t* q_host, uint16_t* q_dev, const float*
     return MOSKA_OK;
 }
 
+int moska_decode_step_fp8_host(const uint16_t* q_host, uint16_t* q_dev, const float* summaries,
+                               const uint8_t* k8_shared, const uint8_t* v8_shared,
+                               const float* k_scale_shared, const float* v_scale_shared,
+                               const uint8_t* k8_unique, const uint8_t* v8_unique,
+                               const float* k_scale_unique, const float* v_scale_unique,
+                               const int64_t* kv_start, const int32_t* kv_len, int32_t* topk_idx,
+                               int32_t* seg_offsets, int32_t* seg_entries, float* o_part, float* lse_part,
+                               uint16_t* out_dev, uint16_t* out_host, float softmax_scale,
+                               const moska_shape* shape, void* ws, size_t ws_bytes, moska_stream stream,
+                               moska_stream side_stream, moska_profiler* prof)
+{
+    MOSKA_API_RANGE();
+    if (summaries == nullptr)
+        return fail(MOSKA_ERR_UNSUPPORTED, "the FP8 shared store is built for routed mode (no dense mode)");
+    MOSKA_TRY(check_shape(shape, true));
+    if (q_host == nullptr || q_dev == nullptr || out_dev == nullptr || out_host == nullptr)
+        return fail(MOSKA_ERR_INVALID_ARG, "q_host, q_dev, out_dev and out_host must not be NULL");
+    if (!aligned(q_host, 16))
+        return fail(MOSKA_ERR_INVALID_ARG, "q_host is not 16-byte aligned");
+    UniqueKv kv;
+    kv.k8 = k8_unique;
+    kv.v8 = v8_unique;
+    kv.k_scale = k_scale_unique;
+    kv.v_scale = v_scale_unique;
+    kv.fp8 = true;
+    SharedF8 f8;
+    f8.k8 = k8_shared;
+    f8.v8 = v8_shared;
+    f8.k_scale = k_scale_shared;
+    f8.v_scale = v_scale_shared;
+    MOSKA_TRY(decode_step_impl(q_dev, summaries, nullptr, nullptr, &f8, kv, kv_start, kv_len, topk_idx,
+                               seg_offsets, seg_entries, o_part, lse_part, out_dev, nullptr, softmax_scale,
+                               shape, ws, ws_bytes, stream, side_stream, prof, out_host, q_host));
+    MOSKA_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    return MOSKA_OK;
+}
+
 }  // extern "C"

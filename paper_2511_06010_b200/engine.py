@@ -145,6 +145,34 @@ class MoskaLayer:
                           self.shape, self.ws, None, self.side_stream if two_streams else None, prof)
         return self.out
 
+    def step_fp8_host(self, q_host, q_dev, out_host, sf8, f8, kv_start, kv_len, two_streams=False,
+                      prof=None, unique_tokens=0):
+        """step_fp8 with the queries taken from and the result delivered to host memory."""
+        self.shape.unique_tokens = int(unique_tokens)
+        two_streams = two_streams and self.overlap_routing
+        if two_streams and self.side_stream is None:
+            self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
+        M.decode_step_fp8_host(q_host, q_dev, self.summaries, sf8.k8, sf8.v8, sf8.k_scale, sf8.v_scale,
+                               f8.k8, f8.v8, f8.k_scale, f8.v_scale, kv_start, kv_len, self.topk_idx,
+                               self.seg_offsets, self.seg_entries, self.o_part, self.lse_part, self.out,
+                               out_host, self.scale, self.shape, self.ws, None,
+                               self.side_stream if two_streams else None, prof)
+        return out_host
+
+    def bind_step_fp8_host(self, q_host, q_dev, out_host, sf8, f8, kv_start, kv_len, two_streams=False,
+                           unique_tokens=0):
+        """step_fp8_host for a loop over fixed buffers: arguments marshalled once (see bind_step_host)."""
+        self.shape.unique_tokens = int(unique_tokens)
+        two_streams = two_streams and self.overlap_routing
+        if two_streams and self.side_stream is None:
+            self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
+        return M.bind_decode_step_fp8_host(q_host, q_dev, self.summaries, sf8.k8, sf8.v8, sf8.k_scale,
+                                           sf8.v_scale, f8.k8, f8.v8, f8.k_scale, f8.v_scale, kv_start,
+                                           kv_len, self.topk_idx, self.seg_offsets, self.seg_entries,
+                                           self.o_part, self.lse_part, self.out, out_host, self.scale,
+                                           self.shape, self.ws, None,
+                                           self.side_stream if two_streams else None)
+
     def bind_step_host(self, q_host, q_dev, out_host, k_shared, v_shared, k_unique, v_unique,
                        kv_start, kv_len, two_streams=False, unique_tokens=0):
         """step_host for a loop over fixed buffers: marshals the arguments once and returns a

@@ -111,6 +111,12 @@ def test_decode_step_with_both_stores_in_fp8():
             PU.check_attention(out.float().cpu().numpy(), want, f"all-fp8 decode step out (two_streams={two})")
             PU.check_lse(layer.lse_out.cpu().numpy(), want_lse, "all-fp8 decode step lse")
             assert M.device_status() == 0
+            # the host-buffer form of the same step: same bits
+            q_host = q.cpu().pin_memory()
+            out_host = torch.zeros(w.B, w.Hq, w.D, dtype=torch.bfloat16).pin_memory()
+            layer.step_fp8_host(q_host, torch.empty_like(q), out_host, sf8, f8, kv_start, kv_len,
+                                two_streams=two, unique_tokens=int(kv_len.sum().item()))
+            assert torch.equal(out_host, out.cpu())
 
 
 def test_fp8_shared_rejects_what_it_does_not_serve():
