@@ -36,6 +36,37 @@ def test_every_declared_symbol_is_exported_and_bound(M):
     assert M.version() >= 100
 
 
+def test_header_is_plain_c_and_a_c_program_links_against_the_library(M, tmp_path):
+    """include/moska.h compiles as C99 with warnings as errors, and a C program that includes it
+    links against the shared library and runs its host-only calls (no GPU needed)."""
+    import shutil
+    import subprocess
+
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    src = tmp_path / "use_moska.c"
+    src.write_text(
+        '#include <stdio.h>\n#include "moska.h"\n'
+        "int main(void) {\n"
+        "    moska_shape s = {64, 32, 8, 128, 128, 512, 8, 8, 4, 0, 0};\n"
+        "    if (moska_version() < 100) return 1;\n"
+        "    if (moska_partial_slots(&s) != 12) return 2;\n"
+        "    if (moska_workspace_bytes(&s) == 0) return 3;\n"
+        "    s.k = 1000; /* k > C */\n"
+        "    if (moska_workspace_bytes(&s) != 0) return 4;\n"
+        '    printf("%s\\n", moska_last_error());\n'
+        "    return 0;\n}\n")
+    exe = tmp_path / "use_moska"
+    lib_dir = os.path.dirname(M.LIB_PATH)
+    subprocess.run([gcc, "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-I", os.path.join(ROOT, "include"),
+                    str(src), "-o", str(exe), "-L", lib_dir, "-l:" + os.path.basename(M.LIB_PATH),
+                    "-Wl,-rpath," + lib_dir], check=True, capture_output=True, text=True)
+    r = subprocess.run([str(exe)], capture_output=True, text=True, timeout=60)
+    assert r.returncode == 0, (r.returncode, r.stdout, r.stderr)
+    assert r.stdout.strip() != ""   # the text of the rejected shape
+
+
 def test_pure_host_helpers(M):
     s = M.shape(64, 32, 8, 128, 128, 512, 8, n_unique_splits=4)
     assert M.partial_slots(s) == 12
