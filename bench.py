@@ -352,8 +352,8 @@ def measure(args, w_full, rank, world, dev, headline: bool):
         f8 = W.quantize_unique_store_fp8(un, release=True)
         torch.cuda.empty_cache()
     sfp8 = args.shared_kv == "fp8"
-    if sfp8 and (w.D != 128 or w.dense or T > 1):
-        raise SystemExit("--shared-kv fp8 needs head dimension 128, routed mode and q_len 1")
+    if sfp8 and (w.D != 128 or T > 1):
+        raise SystemExit("--shared-kv fp8 needs head dimension 128 and q_len 1")
     n_q = max(1, w.steps)
     qs = [W.make_queries(w, sh, s, dev) for s in range(n_q)]
     kv_lens = [(un.kv_len + s).to(torch.int32) for s in range(n_q)]
@@ -637,7 +637,8 @@ def measure(args, w_full, rank, world, dev, headline: bool):
     # the tensor-core kernel and the 8-row streaming tiles (FP8 shared store: plus the query
     # conversion), or 16-row and 8-row tiles
     n_shared_launches = 3 if sfp8 else 2
-    n_launch = 3 if w.dense else (1 + (w.C > 256)) + (3 if w.B > 64 else 2) + 1 + n_shared_launches + 1
+    n_launch = (3 + (1 if sfp8 else 0)) if w.dense else \
+        (1 + (w.C > 256)) + (3 if w.B > 64 else 2) + 1 + n_shared_launches + 1
     hbm_bytes = work["unique_bytes"] + work["shared_bytes"] + rows_merge_bytes
     amort = P / max(1, touched)
     rec = {

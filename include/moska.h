@@ -260,13 +260,15 @@ int moska_shared_attn(const uint16_t* q, const uint16_t* k_shared, const uint16_
  * e4m3(v8[h][c][t][:]): ONE scale per (KV head, chunk) and tensor, so the key scale joins the softmax
  * scale and the value scale the final normalisation.  The code tiles arrive by TMA (half the bytes
  * of the bf16 store), are widened exactly to f16 in shared memory and multiplied on the tensor cores
- * with f16 Q and P and fp32 accumulation.  Routed mode only (topk_idx, seg_offsets, seg_entries as
- * for moska_shared_attn, none NULL), D = 128.  Segments of at most 8 query rows are streamed by a
+ * with f16 Q and P and fp32 accumulation.  Routed or dense mode as for moska_shared_attn (in dense
+ * mode a partial slot covers a run of chunks with different scales: the running maximum is kept in
+ * scaled units and a chunk's value scale, relative to the run's first, joins its P tiles), D = 128.  Segments of at most 8 query rows are streamed by a
  * kernel of their own (codes widened in registers, f16 warp MMAs), as with the bf16 store.
  *   k8_shared, v8_shared  uint8 [Hkv][C][L][D]  OCP FP8 E4M3 codes (128-byte aligned)
  *   k_scale, v_scale      float [Hkv][C]        positive
  *   ws                    as for moska_shared_attn (the grouping's work lists); the call also keeps
- *                         an f16 copy of q in it, so it WRITES the workspace
+ *                         an f16 copy of q in it, so it WRITES the workspace and needs it in dense
+ *                         mode too
  * Chunk embeddings for the router are built from whichever copy of the keys the caller has in
  * bf16 (moska_build_chunk_summaries*); they are an offline step.
  */
@@ -379,8 +381,8 @@ int moska_decode_step_fp8kv(const uint16_t* q, const float* summaries, const uin
 
 /*
  * moska_decode_step with the SHARED store in FP8 (laid out as for moska_shared_attn_fp8); the
- * private store stays bf16.  Same schedule, buffers, outputs and error behaviour; routed mode only
- * (summaries must not be NULL), D = 128.
+ * private store stays bf16.  Same schedule, buffers, outputs and error behaviour (summaries NULL
+ * selects dense mode); D = 128; the workspace is needed in dense mode too.
  */
 int moska_decode_step_fp8shared(const uint16_t* q, const float* summaries, const uint8_t* k8_shared,
                                 const uint8_t* v8_shared, const float* k_scale_shared,
@@ -395,8 +397,8 @@ int moska_decode_step_fp8shared(const uint16_t* q, const float* summaries, const
  * moska_decode_step with BOTH stores in FP8, the KV precision of the paper's evaluation (Section
  * IV) on the whole path: the shared store as for moska_shared_attn_fp8 (one scale per (KV head,
  * chunk)), the private store as for moska_unique_attn_fp8 (one scale per (token, KV head)).  Same
- * schedule, buffers, outputs and error behaviour as moska_decode_step; routed mode only (summaries
- * must not be NULL), D = 128.
+ * schedule, buffers, outputs and error behaviour as moska_decode_step (summaries NULL selects dense
+ * mode); D = 128; the workspace is needed in dense mode too.
  */
 int moska_decode_step_fp8(const uint16_t* q, const float* summaries, const uint8_t* k8_shared,
                           const uint8_t* v8_shared, const float* k_scale_shared, const float* v_scale_shared,

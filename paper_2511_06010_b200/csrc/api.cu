@@ -371,17 +371,26 @@ int moska_shared_attn_fp8(const uint16_t* q, const uint8_t* k8_shared, const uin
     REQUIRE_PTR(v_scale, 4);
     REQUIRE_PTR(o_part, 32);
     REQUIRE_PTR(lse_part, 4);
-    if (topk_idx == nullptr || seg_offsets == nullptr || seg_entries == nullptr)
-        return fail(MOSKA_ERR_UNSUPPORTED, "the FP8 shared store is built for routed mode (no dense mode)");
-    if (shape->shared_slots != shape->k)
-        return fail(MOSKA_ERR_INVALID_ARG, "routed mode needs shared_slots == k");
+    const bool dense = (topk_idx == nullptr && seg_offsets == nullptr && seg_entries == nullptr);
+    if (!dense) {
+        REQUIRE_PTR(topk_idx, 4);
+        REQUIRE_PTR(seg_offsets, 4);
+        REQUIRE_PTR(seg_entries, 4);
+        if (shape->shared_slots != shape->k)
+            return fail(MOSKA_ERR_INVALID_ARG, "routed mode needs shared_slots == k");
+    } else if (shape->shared_slots > shape->C) {
+        return fail(MOSKA_ERR_INVALID_ARG, "dense mode needs shared_slots <= C");
+    }
+    // (dense mode too: the workspace holds the f16 copy of the queries)
     if (ws == nullptr || !aligned(ws, 256) || ws_bytes < ws_layout(shape).total)
         return fail(MOSKA_ERR_WORKSPACE, "workspace missing, misaligned or smaller than %zu bytes",
                     ws_layout(shape).total);
     MOSKA_TRY(check_device());
-    // segments of more than 8 rows on the tensor-core kernel, the 8-row tiles streamed
-    MOSKA_TRY(launch_shared_tc_fp8(q, k8_shared, v8_shared, k_scale, v_scale, seg_entries, o_part, lse_part,
-                                   softmax_scale, shape, ws, 0, (cudaStream_t)stream));
+    // dense mode: every item on the tensor-core kernel; routed mode: segments of more than 8 rows
+    // there, the 8-row tiles streamed
+    MOSKA_TRY(launch_shared_tc_fp8(q, k8_shared, v8_shared, k_scale, v_scale, dense ? nullptr : seg_entries,
+                                   o_part, lse_part, softmax_scale, shape, ws, dense, 0, (cudaStream_t)stream));
+    if (dense) return MOSKA_OK;
     return launch_shared_small_fp8(q, k8_shared, v8_shared, k_scale, v_scale, seg_entries, o_part,
                                    lse_part, softmax_scale, shape, ws, (cudaStream_t)stream);
 }
@@ -552,13 +561,12 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
         if (!copy_on_side)
             MOSKA_CUDA_TRY(cudaMemcpyAsync(const_cast<uint16_t*>(q), q_host, q_bytes, cudaMemcpyHostToDevice, st));
     }
-    if (f8 != nullptr && dense)
-        return fail(MOSKA_ERR_UNSUPPORTED, "the FP8 shared store is built for routed mode (no dense mode)");
     // the tensor-core kernel over whichever shared store the step has
     auto shared_tc = [&](bool dense_mode, int max_ctas, cudaStream_t s_) {
         if (f8 != nullptr)
-            return launch_shared_tc_fp8(q, f8->k8, f8->v8, f8->k_scale, f8->v_scale, seg_entries, o_part,
-                                        lse_part, softmax_scale, shape, ws, max_ctas, s_);
+            return launch_shared_tc_fp8(q, f8->k8, f8->v8, f8->k_scale, f8->v_scale,
+                                        dense_mode ? nullptr : seg_entries, o_part, lse_part, softmax_scale,
+                                        shape, ws, dense_mode, max_ctas, s_);
         return launch_shared_tc(q, k_shared, v_shared, dense_mode ? nullptr : seg_entries, o_part, lse_part,
                                 softmax_scale, shape, ws, dense_mode, max_ctas, s_);
     };
@@ -578,8 +586,10 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_UNIQUE, 1, st));
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 0, st));
         if (f8 != nullptr)
-            MOSKA_TRY(moska_shared_attn_fp8(q, f8->k8, f8->v8, f8->k_scale, f8->v_scale, topk_idx, seg_offsets,
-                                            seg_entries, o_part, lse_part, softmax_scale, shape, ws, ws_bytes, st));
+            MOSKA_TRY(moska_shared_attn_fp8(q, f8->k8, f8->v8, f8->k_scale, f8->v_scale,
+                                            dense ? nullptr : topk_idx, dense ? nullptr : seg_offsets,
+                                            dense ? nullptr : seg_entries, o_part, lse_part, softmax_scale,
+                                            shape, ws, ws_bytes, st));
         else
             MOSKA_TRY(moska_shared_attn(q, k_shared, v_shared, dense ? nullptr : topk_idx,
                                         dense ? nullptr : seg_offsets, dense ? nullptr : seg_entries,
@@ -603,6 +613,10 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
             REQUIRE_PTR(f8->v8, 128);
             REQUIRE_PTR(f8->k_scale, 4);
             REQUIRE_PTR(f8->v_scale, 4);
+            // (dense mode too: the workspace holds the f16 copy of the queries)
+            if (ws == nullptr || !aligned(ws, 256) || ws_bytes < ws_layout(shape).total)
+                return fail(MOSKA_ERR_WORKSPACE, "workspace missing, misaligned or smaller than %zu bytes",
+                            ws_layout(shape).total);
         } else {
             REQUIRE_PTR(k_shared, 128);
             REQUIRE_PTR(v_shared, 128);
@@ -629,8 +643,10 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
             MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_GROUP, 1, side));
         }
         MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 0, side));
+        // (with the FP8 store the tensor-core kernel takes dense batches of any size)
         const bool tc = shared_tc_supported(shape) &&
-                        (!dense || (long long)shape->B * (shape->Hq / shape->Hkv) >= kDenseTcMinRows);
+                        (!dense || f8 != nullptr ||
+                         (long long)shape->B * (shape->Hq / shape->Hkv) >= kDenseTcMinRows);
         // Sharing the SMs pays when unique attention runs long enough for the tensor-core kernel
         // to start beside it (the routing chain in front of it takes a few hundred microseconds
         // under contention); for a short unique attention the tensor-core items run after it, on
@@ -641,10 +657,11 @@ int decode_step_impl(const uint16_t* q, const float* summaries, const uint16_t* 
         if (tc && beside) MOSKA_TRY(shared_tc(dense, tc_sm_share(shape, dense, unique_ms), side));
         // the streaming tiles (every tile of a shape the tensor-core kernel does not serve, else the
         // 8-row tiles of routed mode) always run beside unique attention
-        if (f8 != nullptr)
-            MOSKA_TRY(launch_shared_small_fp8(q, f8->k8, f8->v8, f8->k_scale, f8->v_scale, seg_entries,
-                                              o_part, lse_part, softmax_scale, shape, ws, side));
-        else if (!tc || !dense)
+        if (f8 != nullptr) {
+            if (!dense)
+                MOSKA_TRY(launch_shared_small_fp8(q, f8->k8, f8->v8, f8->k_scale, f8->v_scale, seg_entries,
+                                                  o_part, lse_part, softmax_scale, shape, ws, side));
+        } else if (!tc || !dense)
             MOSKA_TRY(launch_shared_small(q, k_shared, v_shared, dense ? nullptr : seg_entries, o_part,
                                           lse_part, softmax_scale, shape, ws, dense, tc, side));
         if (beside || !tc) MOSKA_CUDA_TRY(prof_mark(prof, MOSKA_STAGE_SHARED, 1, side));
@@ -716,8 +733,6 @@ int moska_decode_step_fp8shared(const uint16_t* q, const float* summaries, const
                                 moska_stream stream, moska_stream side_stream, moska_profiler* prof)
 {
     MOSKA_API_RANGE();
-    if (summaries == nullptr)
-        return fail(MOSKA_ERR_UNSUPPORTED, "the FP8 shared store is built for routed mode (no dense mode)");
     UniqueKv kv;
     kv.k = k_unique;
     kv.v = v_unique;
@@ -741,8 +756,6 @@ int moska_decode_step_fp8(const uint16_t* q, const float* summaries, const uint8
                           moska_stream side_stream, moska_profiler* prof)
 {
     MOSKA_API_RANGE();
-    if (summaries == nullptr)
-        return fail(MOSKA_ERR_UNSUPPORTED, "the FP8 shared store is built for routed mode (no dense mode)");
     UniqueKv kv;
     kv.k8 = k8_unique;
     kv.v8 = v8_unique;
@@ -876,8 +889,6 @@ int moska_decode_step_fp8_host(const uint16_t* q_host, uint16_t* q_dev, const fl
                                moska_stream side_stream, moska_profiler* prof)
 {
     MOSKA_API_RANGE();
-    if (summaries == nullptr)
-        return fail(MOSKA_ERR_UNSUPPORTED, "the FP8 shared store is built for routed mode (no dense mode)");
     MOSKA_TRY(check_shape(shape, true));
     if (q_host == nullptr || q_dev == nullptr || out_dev == nullptr || out_host == nullptr)
         return fail(MOSKA_ERR_INVALID_ARG, "q_host, q_dev, out_dev and out_host must not be NULL");

@@ -124,7 +124,7 @@ int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t
 // The same over a shared store of FP8 (E4M3) codes with one scale per (KV head, chunk); routed mode.
 int launch_shared_tc_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v8, const float* k_scale,
                          const float* v_scale, const int32_t* seg_entries, float* o_part, float* lse_part,
-                         float scale, const moska_shape* s, void* ws, int max_ctas, cudaStream_t st);
+                         float scale, const moska_shape* s, void* ws, bool dense, int max_ctas, cudaStream_t st);
 // Estimated SM-milliseconds of the tensor-core kernel for this shape (host, pure).
 double shared_tc_cost_sm_ms(const moska_shape* s, bool dense);
 // Device address (on the current device) of the library's sticky status word: kernels lower it

@@ -194,7 +194,7 @@ struct Unit {
     int slot_dense;      // dense: partial slot (= run of chunks)
     int n_it[2];         // K/V tiles handled by slot 0 / 1
     long long kv_row0[2];  // first token row of the slot's K/V range in the [Hkv*C*L][D] store
-    int key[2];            // routed: h * C + chunk of the slot's item (index of its scales)
+    int key[2];            // h * C + chunk of the slot's item (dense: the run's first chunk): index of its scales
 };
 
 // Where the routed work lists end and how the single-tile items are scheduled on this grid: whole
@@ -277,6 +277,7 @@ __device__ __forceinline__ Unit decode_unit(const TcParams& p, const Schedule& s
         it.n_e[0] = min(per_tile, p.B - it.b0[0]);
         it.n_e[1] = max(0, min(per_tile, p.B - it.b0[1]));
         it.kv_row0[0] = it.kv_row0[1] = ((long long)it.h[0] * p.C + c0) * p.L;
+        it.key[0] = it.key[1] = it.h[0] * p.C + c0;  // the run's first chunk (index of its scales)
         it.n_kv = (c1 - c0) * (p.L / kKvTile);
         it.entry_begin[0] = it.entry_begin[1] = 0;
         it.mode = kTwoTiles;
@@ -755,11 +756,18 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             oc[0] += it.n_it[0] > 0;
             oc[1] += it.n_it[1] > 0;
             xc += split;
-            // FP8 store: the chunk's key scale joins the softmax scale, its value scale the final
-            // normalisation (routed mode: one chunk per item)
-            const float ksc = F ? __ldg(p.k_scale + pick(it.key, t)) : 1.f;
-            const float vsc = F ? __ldg(p.v_scale + pick(it.key, t)) : 1.f;
-            const float sl2 = p.scale * kLog2e * ksc;
+            // FP8 store: a chunk's key scale joins the softmax scale of its tiles; its value scale
+            // joins the final normalisation (routed mode: one chunk per item) or, relative to the
+            // scale of the run's first chunk, the P tile (dense mode: a run of chunks per item).
+            // The running maximum is then kept in scaled log2 units, so that it carries across
+            // chunks; with the bf16 store it stays in raw score units (`conv` converts).
+            const int key0 = pick(it.key, t);
+            const float v_ref = F ? __ldg(p.v_scale + key0) : 1.f;
+            float ksc = F ? __ldg(p.k_scale + key0) : 1.f;
+            float p_mul = 1.f;  // dense FP8: value scale of the tile's chunk / v_ref
+            float sl2 = p.scale * kLog2e * ksc;
+            const float conv = F ? 1.f : sl2;
+            const int tiles_per_chunk = p.L / kKvTile;
             const int n_rows = pick(it.n_e, t) * G;
             // a warp none of whose rows exists skips the arithmetic (every row of the products
             // depends on its own query row only), but keeps every barrier in step
@@ -793,6 +801,15 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
             }
             float m_ref = -INFINITY, l_sum = 0.f;
             for (int j = 0; j < n_it; ++j) {
+                if constexpr (F) {
+                    if (p.dense) {  // scales of the chunk this tile lies in (asked for before the wait)
+                        const int tile = split ? 2 * j + t : j;
+                        const int c = key0 + tile / tiles_per_chunk;
+                        ksc = __ldg(p.k_scale + c);
+                        p_mul = __ldg(p.v_scale + c) / v_ref;
+                        sl2 = p.scale * kLog2e * ksc;
+                    }
+                }
                 alive = __all_sync(0xffffffffu, mbar_wait(&sm.s_full[t], sc & 1, ab));
                 if (!alive) break;
                 ++sc;
@@ -816,16 +833,17 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
 #pragma unroll
                         for (int x = 0; x < 16; ++x)
                             mxs[x & 7] = fmax3(mxs[x & 7], __uint_as_float(r[c][2 * x]), __uint_as_float(r[c][2 * x + 1]));
-                    const float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
-                                           fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
+                    float mx = fmaxf(fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3])),
+                                     fmaxf(fmaxf(mxs[4], mxs[5]), fmaxf(mxs[6], mxs[7])));
+                    if constexpr (F) mx *= sl2;  // scaled log2 units
                     if (j == 0) {
                         m_ref = mx;
                     } else {
                         // rows that do not exist hold arbitrary bits: they never ask for a rescale
-                        const bool need = i < n_rows && (mx - m_ref) * sl2 > kRescaleThreshold;
+                        const bool need = i < n_rows && (mx - m_ref) * conv > kRescaleThreshold;
                         if (__any_sync(0xffffffffu, need)) {
                             // every MMA issued before S_t(j), PV_t(j-1) included, has completed
-                            const float alpha = need ? fast_exp2((m_ref - mx) * sl2) : 1.f;
+                            const float alpha = need ? fast_exp2((m_ref - mx) * conv) : 1.f;
                             if (need) m_ref = mx;
                             l_sum *= alpha;
 #pragma unroll 1
@@ -842,7 +860,7 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     }
                     // P = exp2((S - m_ref) * scale * log2 e) as bf16, written over the columns of S
                     const float2 sl2_2 = make_float2(sl2, sl2);
-                    const float2 nmb_2 = make_float2(-m_ref * sl2, -m_ref * sl2);
+                    const float2 nmb_2 = make_float2(-m_ref * conv, -m_ref * conv);
                     float2 ls[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};  // partial row sums
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
@@ -857,7 +875,7 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                             pr.y = fast_exp2(e.y);
                             ls[x & 1] = fadd2(ls[x & 1], pr);
                             if constexpr (F) {
-                                const __half2 h2 = __floats2half2_rn(pr.x, pr.y);
+                                const __half2 h2 = __floats2half2_rn(pr.x * p_mul, pr.y * p_mul);
                                 pk[x] = *reinterpret_cast<const uint32_t*>(&h2);
                             } else {
                                 const __nv_bfloat162 b2 = __floats2bfloat162_rn(pr.x, pr.y);
@@ -893,13 +911,13 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                 if (!alive) break;
                 const float m1 = sm.stat_m[i], l1 = sm.stat_l[i];
                 m_all = fmaxf(m_ref, m1);
-                a_mine = fast_exp2((m_ref - m_all) * sl2);
-                a_other = fast_exp2((m1 - m_all) * sl2);
+                a_mine = fast_exp2((m_ref - m_all) * conv);
+                a_other = fast_exp2((m1 - m_all) * conv);
                 den = a_mine * l_sum + a_other * l1;
             }
             if (warp_live) {
                 tc_fence_after_sync();
-                const float inv = vsc / den;
+                const float inv = v_ref / den;
                 a_mine *= inv;
                 a_other *= inv;
                 float4* o = my_r >= 0
@@ -938,7 +956,7 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                         for (int x = 0; x < 4; ++x)
                             st_global_v8(reinterpret_cast<float*>(o) + c * 32 + x * 8,
                                          reinterpret_cast<const float*>(&r[c][8 * x]));
-                    p.lse_part[my_r * p.n_slots + my_slot] = m_all * (p.scale * ksc) + logf(den);
+                    p.lse_part[my_r * p.n_slots + my_slot] = (F ? m_all * kLn2 : m_all * p.scale) + logf(den);
                 }
             }
             if (split) {
@@ -1038,8 +1056,7 @@ int make_code_map(CUtensorMap* tm, const uint8_t* base, long long rows)
     return MOSKA_OK;
 }
 
-// Common part of the two launchers.  k8 / v8 != nullptr selects the FP8 shared store (routed mode
-// only).
+// Common part of the two launchers.  k8 / v8 != nullptr selects the FP8 shared store.
 int launch_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared, const uint8_t* k8,
               const uint8_t* v8, const float* k_scale, const float* v_scale, const int32_t* seg_entries,
               float* o_part, float* lse_part, float scale, const moska_shape* s, void* ws, bool dense,
@@ -1133,10 +1150,11 @@ int launch_shared_tc(const uint16_t* q, const uint16_t* k_shared, const uint16_t
 
 int launch_shared_tc_fp8(const uint16_t* q, const uint8_t* k8, const uint8_t* v8, const float* k_scale,
                          const float* v_scale, const int32_t* seg_entries, float* o_part, float* lse_part,
-                         float scale, const moska_shape* s, void* ws, int max_ctas, cudaStream_t st)
+                         float scale, const moska_shape* s, void* ws, bool dense, int max_ctas,
+                         cudaStream_t st)
 {
     return launch_tc(q, nullptr, nullptr, k8, v8, k_scale, v_scale, seg_entries, o_part, lse_part, scale, s,
-                     ws, false, max_ctas, st);
+                     ws, dense, max_ctas, st);
 }
 
 // Measured on B200: an item costs about 6 us of fill, drain and epilogue plus 2.2 us per K/V

@@ -126,7 +126,7 @@ class MoskaLayer:
         two_streams = two_streams and self.overlap_routing
         if two_streams and self.side_stream is None:
             self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
-        M.decode_step_fp8shared(q, self.summaries, sf8.k8, sf8.v8, sf8.k_scale, sf8.v_scale, k_unique,
+        M.decode_step_fp8shared(q, None if self.dense else self.summaries, sf8.k8, sf8.v8, sf8.k_scale, sf8.v_scale, k_unique,
                                 v_unique, kv_start, kv_len, self.topk_idx, self.seg_offsets, self.seg_entries,
                                 self.o_part, self.lse_part, self.out, self.lse_out, self.scale, self.shape,
                                 self.ws, None, self.side_stream if two_streams else None, prof)
@@ -139,7 +139,7 @@ class MoskaLayer:
         two_streams = two_streams and self.overlap_routing
         if two_streams and self.side_stream is None:
             self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
-        M.decode_step_fp8(q, self.summaries, sf8.k8, sf8.v8, sf8.k_scale, sf8.v_scale, f8.k8, f8.v8,
+        M.decode_step_fp8(q, None if self.dense else self.summaries, sf8.k8, sf8.v8, sf8.k_scale, sf8.v_scale, f8.k8, f8.v8,
                           f8.k_scale, f8.v_scale, kv_start, kv_len, self.topk_idx, self.seg_offsets,
                           self.seg_entries, self.o_part, self.lse_part, self.out, self.lse_out, self.scale,
                           self.shape, self.ws, None, self.side_stream if two_streams else None, prof)
@@ -152,7 +152,7 @@ class MoskaLayer:
         two_streams = two_streams and self.overlap_routing
         if two_streams and self.side_stream is None:
             self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
-        M.decode_step_fp8_host(q_host, q_dev, self.summaries, sf8.k8, sf8.v8, sf8.k_scale, sf8.v_scale,
+        M.decode_step_fp8_host(q_host, q_dev, None if self.dense else self.summaries, sf8.k8, sf8.v8, sf8.k_scale, sf8.v_scale,
                                f8.k8, f8.v8, f8.k_scale, f8.v_scale, kv_start, kv_len, self.topk_idx,
                                self.seg_offsets, self.seg_entries, self.o_part, self.lse_part, self.out,
                                out_host, self.scale, self.shape, self.ws, None,
@@ -166,7 +166,7 @@ class MoskaLayer:
         two_streams = two_streams and self.overlap_routing
         if two_streams and self.side_stream is None:
             self.side_stream = torch.cuda.Stream(device=self.device, priority=-1)
-        return M.bind_decode_step_fp8_host(q_host, q_dev, self.summaries, sf8.k8, sf8.v8, sf8.k_scale,
+        return M.bind_decode_step_fp8_host(q_host, q_dev, None if self.dense else self.summaries, sf8.k8, sf8.v8, sf8.k_scale,
                                            sf8.v_scale, f8.k8, f8.v8, f8.k_scale, f8.v_scale, kv_start,
                                            kv_len, self.topk_idx, self.seg_offsets, self.seg_entries,
                                            self.o_part, self.lse_part, self.out, out_host, self.scale,

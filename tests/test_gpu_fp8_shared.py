@@ -126,3 +126,59 @@ def test_fp8_shared_rejects_what_it_does_not_serve():
     with pytest.raises(M.MoskaError) as e:
         layer.shared_fp8(torch.zeros(4, 4, 64, dtype=torch.bfloat16, device="cuda"), f8)
     assert e.value.status == M.ERR_UNSUPPORTED
+
+
+def _dense_reference(q, sf8, C, slots, scale):
+    """Oracle for dense mode over the FP8 shared store: the per-chunk partials of every row (all C
+    chunks), merged over each run of ceil(C / slots) consecutive chunks."""
+    B, Hq, _ = q.shape
+    Hkv = sf8.k8.shape[0]
+    all_chunks = np.tile(np.arange(C, dtype=np.int32), (B, Hkv, 1))
+    o_c, l_c = O.shared_partials_fp8(q.cpu(), sf8.k8.cpu(), sf8.v8.cpu(), sf8.k_scale.cpu(), sf8.v_scale.cpu(),
+                                     all_chunks, scale)
+    run = (C + slots - 1) // slots
+    o_r = np.zeros((B, Hq, slots, q.shape[2]))
+    l_r = np.full((B, Hq, slots), -np.inf)
+    for s in range(slots):
+        c0, c1 = min(C, s * run), min(C, (s + 1) * run)
+        if c1 > c0:
+            o_r[:, :, s], l_r[:, :, s] = O.merge(o_c[:, :, c0:c1], l_c[:, :, c0:c1])
+    return o_r, l_r
+
+
+def test_fp8_shared_dense_mode_runs_of_chunks_with_different_scales():
+    """Dense mode (no routing): a partial slot covers a run of chunks whose key and value scales
+    differ, so the running maximum and the value scale have to carry across chunks.  Batches of one
+    row tile (split over the two slots), two tiles, several items, a partial last run, G = 4 and 8."""
+    M, MoskaLayer = _mods()
+    for Hq, Hkv, B, C, L, slots in ((8, 2, 20, 6, 256, 3), (8, 2, 70, 5, 128, 2), (16, 2, 40, 4, 384, 4),
+                                    (8, 2, 3, 7, 128, 3), (8, 2, 200, 3, 256, 1)):
+        w = W.Workload("f8dense", B=B, Hq=Hq, Hkv=Hkv, D=128, C=C, L=L, k=C, unique_len=64, seed=300 + B)
+        sh = W.make_shared_store(w, "cuda")
+        # chunk-dependent magnitudes, so that the scales really differ from chunk to chunk
+        mag = torch.linspace(0.5, 3.0, C, device="cuda").view(1, C, 1, 1)
+        sh = W.SharedStore((sh.k_shared.float() * mag).to(torch.bfloat16), (sh.v_shared.float() * mag.flip(1)).to(torch.bfloat16), sh.mu)
+        un = W.make_unique_store(w, "cuda")
+        q = W.make_queries(w, sh, 0, "cuda")
+        sf8 = W.quantize_shared_store_fp8(sh)
+        layer = MoskaLayer(B, Hq, Hkv, 128, C, L, C, 64, dense=True, dense_slots=slots, n_unique_splits=2)
+        layer.o_part.fill_(float("nan"))
+        layer.lse_part.fill_(float("nan"))
+        layer.shared_fp8(q, sf8)
+        torch.cuda.synchronize()
+        o_ref, l_ref = _dense_reference(q, sf8, C, slots, layer.scale)
+        PU.check_lse(layer.lse_part[:, :, :slots].cpu().numpy(), l_ref, "fp8 dense lse")
+        PU.check_attention(layer.o_part[:, :, :slots].cpu().numpy(), o_ref, "fp8 dense partial o")
+        # the whole step, one and two streams
+        dummy = torch.zeros(Hkv, 1, 128, 128, dtype=torch.bfloat16)
+        o_un, l_un = O.attend_direct(q.cpu(), dummy, dummy, un.k_unique.cpu(), un.v_unique.cpu(),
+                                     un.kv_start.cpu().numpy(), un.kv_len.cpu().numpy(),
+                                     np.zeros((B, Hkv, 1), dtype=np.int32), layer.scale, use_shared=False)
+        want, _ = O.merge(np.concatenate([o_ref, o_un[:, :, None, :]], axis=2),
+                          np.concatenate([l_ref, l_un[:, :, None]], axis=2))
+        for two in (False, True):
+            out = layer.step_fp8shared(q, sf8, un.k_unique, un.v_unique, un.kv_start, un.kv_len, two_streams=two,
+                                       unique_tokens=int(un.kv_len.sum().item()))
+            torch.cuda.synchronize()
+            PU.check_attention(out.float().cpu().numpy(), want, f"fp8 dense step out (two_streams={two})")
+        assert M.device_status() == 0
