@@ -861,6 +861,7 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                     // P = exp2((S - m_ref) * scale * log2 e) as bf16, written over the columns of S
                     const float2 sl2_2 = make_float2(sl2, sl2);
                     const float2 nmb_2 = make_float2(-m_ref * conv, -m_ref * conv);
+                    const float2 pmul_2 = make_float2(p_mul, p_mul);
                     float2 ls[2] = {make_float2(0.f, 0.f), make_float2(0.f, 0.f)};  // partial row sums
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
@@ -875,7 +876,8 @@ shared_tc_kernel(const __grid_constant__ CUtensorMap tm_k, const __grid_constant
                             pr.y = fast_exp2(e.y);
                             ls[x & 1] = fadd2(ls[x & 1], pr);
                             if constexpr (F) {
-                                const __half2 h2 = __floats2half2_rn(pr.x * p_mul, pr.y * p_mul);
+                                const float2 ps = ffma2(pr, pmul_2, make_float2(0.f, 0.f));
+                                const __half2 h2 = __floats2half2_rn(ps.x, ps.y);
                                 pk[x] = *reinterpret_cast<const uint32_t*>(&h2);
                             } else {
                                 const __nv_bfloat162 b2 = __floats2bfloat162_rn(pr.x, pr.y);
