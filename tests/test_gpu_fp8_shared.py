@@ -182,3 +182,37 @@ def test_fp8_shared_dense_mode_runs_of_chunks_with_different_scales():
             torch.cuda.synchronize()
             PU.check_attention(out.float().cpu().numpy(), want, f"fp8 dense step out (two_streams={two})")
         assert M.device_status() == 0
+
+
+def test_several_query_tokens_per_request_with_both_stores_in_fp8():
+    """shape.q_len > 1 with the all-FP8 step: the batch rows are requests x q_len; shared attention
+    treats every row as a request of its own, unique attention reads a request's codes once for all
+    its tokens.  The oracle gets the batch-expanded problem (aliased kv_start, per-token context end)."""
+    M, MoskaLayer = _mods()
+    for Hq, Hkv, t, splits in ((8, 2, 2, 1), (4, 2, 4, 2), (8, 4, 3, 1)):
+        lens_last = np.array([40, 1, 130, 77, 300, 16, 2, 0, 600, 65], dtype=np.int64)
+        base = len(lens_last)
+        w = W.Workload("f8multi", B=base * t, Hq=Hq, Hkv=Hkv, D=128, C=8, L=256, k=2, unique_len=0, seed=47)
+        sh = W.make_shared_store(w, "cuda")
+        un = W.make_unique_store(W.scaled(w, B=base, steps=0), "cuda", lens_last)
+        q = W.make_queries(w, sh, 0, "cuda")
+        sf8 = W.quantize_shared_store_fp8(sh)
+        kv_start_dev, kv_len_dev = un.kv_start, un.kv_len
+        f8 = W.quantize_unique_store_fp8(un)
+        layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, int(lens_last.max()), n_unique_splits=splits,
+                           fp8_unique=True, q_len=t)
+        layer.build_summaries(sh.k_shared)
+        out = layer.step_fp8(q, sf8, f8, kv_start_dev, kv_len_dev, two_streams=bool(t % 2))
+        torch.cuda.synchronize()
+        kv_start = kv_start_dev.repeat_interleave(t).cpu().numpy()
+        back = np.tile(np.arange(t - 1, -1, -1), base)
+        kv_len = np.maximum(0, np.repeat(lens_last, t) - back).astype(np.int32)
+        o_sh, l_sh = O.shared_partials_fp8(q.cpu(), sf8.k8.cpu(), sf8.v8.cpu(), sf8.k_scale.cpu(),
+                                           sf8.v_scale.cpu(), layer.topk_idx.cpu().numpy(), layer.scale)
+        o_u, l_u = O.attend_unique_fp8(q.cpu(), f8.k8.cpu(), f8.v8.cpu(), f8.k_scale.cpu(), f8.v_scale.cpu(),
+                                       kv_start, kv_len, layer.scale)
+        want, want_lse = O.merge(np.concatenate([o_sh, o_u[:, :, None, :]], axis=2),
+                                 np.concatenate([l_sh, l_u[:, :, None]], axis=2))
+        PU.check_attention(out.float().cpu().numpy(), want, f"all-fp8 q_len={t} out")
+        PU.check_lse(layer.lse_out.cpu().numpy(), want_lse, f"all-fp8 q_len={t} lse")
+        assert M.device_status() == 0
