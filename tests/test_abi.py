@@ -160,3 +160,35 @@ def test_misaligned_pointers_are_rejected_on_the_host(M):
     need = M.workspace_bytes(s)
     assert lib.moska_group_by_chunk(A, A, A, ctypes.byref(s), A + 128, need, 0) == M.ERR_WORKSPACE
     assert lib.moska_group_by_chunk(A, A, A, ctypes.byref(s), A, need - 1, 0) == M.ERR_WORKSPACE
+
+
+def test_fp8_shared_store_entry_points_reject_bad_arguments_on_the_host(M):
+    """The FP8 shared-store calls: D = 64 is refused, misaligned code pointers and a missing
+    workspace (needed in dense mode too, for the f16 copy of the queries) are reported before any
+    launch, and the host-buffer step insists on its four buffers."""
+    A = 0x10000
+    s = M.shape(4, 32, 8, 128, 128, 512, 8)
+    ws_fake = type("Ws", (), {"numel": lambda self: 1 << 30, "element_size": lambda self: 1,
+                              "is_contiguous": lambda self: True, "data_ptr": lambda self: A})()
+    with pytest.raises(M.MoskaError) as e:
+        M.shared_attn_fp8(A, A, A, A, A, A, A, A, A, A, 1.0, M.shape(4, 32, 8, 64, 128, 512, 8), ws_fake, stream=0)
+    assert e.value.status == M.ERR_UNSUPPORTED
+    with pytest.raises(M.MoskaError) as e:
+        M.shared_attn_fp8(A, A + 64, A, A, A, A, A, A, A, A, 1.0, s, ws_fake, stream=0)
+    assert e.value.status == M.ERR_INVALID_ARG and "aligned" in M.last_error()
+    # dense mode (no routing arrays) still needs the workspace
+    sd = M.shape(4, 32, 8, 128, 128, 512, 128, shared_slots=16)
+    with pytest.raises(M.MoskaError) as e:
+        M.shared_attn_fp8(A, A, A, A, A, None, None, None, A, A, 1.0, sd, None, stream=0)
+    assert e.value.status == M.ERR_WORKSPACE
+    # dense mode with more partial slots than chunks
+    with pytest.raises(M.MoskaError) as e:
+        M.shared_attn_fp8(A, A, A, A, A, None, None, None, A, A, 1.0,
+                          M.shape(4, 32, 8, 128, 8, 512, 8, shared_slots=16), ws_fake, stream=0)
+    assert e.value.status == M.ERR_INVALID_ARG
+    with pytest.raises(M.MoskaError) as e:
+        M.decode_step_fp8_host(None, A, A, A, A, A, A, A, A, A, A, A, A, A, A, A, A, A, A, A, 1.0, s, ws_fake, stream=0)
+    assert e.value.status == M.ERR_INVALID_ARG
+    with pytest.raises(M.MoskaError) as e:
+        M.decode_step_fp8_host(A + 2, A, A, A, A, A, A, A, A, A, A, A, A, A, A, A, A, A, A, A, 1.0, s, ws_fake, stream=0)
+    assert e.value.status == M.ERR_INVALID_ARG
