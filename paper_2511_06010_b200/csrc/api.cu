@@ -184,9 +184,14 @@ int moska_build_chunk_summaries_attn(const uint16_t* k_shared, float* summaries,
 namespace {
 // SMs the persistent tensor-core kernel gets when it runs beside unique attention: both kernels'
 // work is estimated (tensor-core items from the shape, unique attention from the token hint at
-// 7 TB/s) and the SMs are divided so that neither waits for the other.  Unique attention reaches
-// most of the HBM bandwidth from about 96 SMs; if it is the longer job the tensor-core kernel
-// hides entirely on the remaining ones.
+// 7 TB/s) and the SMs are divided so that neither waits for the other.  Unique attention keeps
+// most of the HBM bandwidth on about half of the SMs; if it is the longer job the tensor-core
+// kernel hides entirely on the remaining ones.
+// Share of the SMs left to unique attention in that case (measured on the largest workload: 45-55 %
+// is a flat optimum, 65 % is 0.5 % slower, 85 % 8 % slower; the other workloads do not care).
+#ifndef MOSKA_HBM_SM_PCT
+#define MOSKA_HBM_SM_PCT 55
+#endif
 int tc_sm_share(const moska_shape* s, bool dense, double unique_ms)
 {
     int dev = 0, n_sms = 148;
@@ -198,7 +203,7 @@ int tc_sm_share(const moska_shape* s, bool dense, double unique_ms)
         x = dense ? (n_sms * 4) / 5 : (n_sms * 35) / 100;  // no hint: tensor-heavy / HBM-heavy guess
     } else {
         const double b = unique_ms;
-        const int hbm_sms = (n_sms * 65) / 100;
+        const int hbm_sms = (n_sms * MOSKA_HBM_SM_PCT) / 100;
         if (a <= b * (n_sms - hbm_sms)) x = n_sms - hbm_sms;
         else x = (int)(a * n_sms / (a + b * 0.4 * n_sms));
     }
