@@ -14,8 +14,9 @@
  *  * All tensor arguments are DEVICE pointers owned by the caller, unless a parameter is
  *    documented as a host pointer.  The library never allocates, frees or keeps a pointer
  *    after the call returns.  Scratch memory comes from a caller-provided workspace.
- *  * Every call only enqueues work on `stream` and returns without synchronising.  Nothing
- *    produced on the device is read back by the host.
+ *  * Every call only enqueues work on `stream` and returns without synchronising, and nothing
+ *    produced on the device is read back by the host.  The exceptions say so at their
+ *    declaration: moska_device_status and the *_host forms of the step wait for the device.
  *  * bf16 tensors are passed as `const uint16_t*` (raw bfloat16 bit patterns).
  *  * Symbols: B requests, Hq query heads, Hkv KV heads, G = Hq / Hkv (1..8), D head dimension
  *    (64 or 128), C shared chunks of L tokens each, k chunks routed per (request, KV head).
