@@ -306,7 +306,7 @@ int moska_debug_check_workspace(void* ws, size_t ws_bytes, const moska_shape* sh
         return fail(MOSKA_ERR_WORKSPACE, "workspace missing, misaligned or smaller than %zu bytes",
                     ws_layout(shape).total);
     MOSKA_TRY(check_device());
-    return launch_ws_guards(ws, ws_layout(shape), true, (cudaStream_t)stream);
+    return launch_ws_guards(ws, ws_layout(shape), true, (cudaStream_t)stream, ws_layout(shape).total);
 #else
     (void)ws; (void)ws_bytes; (void)stream;
     return fail(MOSKA_ERR_UNSUPPORTED, "this build of the library has no workspace guard words "

@@ -94,7 +94,8 @@ WsLayout ws_layout(const moska_shape* s);
 // Debug build (MOSKA_DEBUG_GUARDS): writes the guard words behind every workspace region
 // (check = false) or compares them and raises MOSKA_ERR_CORRUPT in the device status word
 // (check = true).  Other builds: does nothing.
-int launch_ws_guards(void* ws, const WsLayout& lay, bool check, cudaStream_t st);
+// `ws_extent`: bytes of `ws` that exist (guard words beyond them are left alone).
+int launch_ws_guards(void* ws, const WsLayout& lay, bool check, cudaStream_t st, size_t ws_extent);
 
 constexpr int kRouteSmallC = 256;   // up to this many chunks the router keeps its scores in shared memory
 constexpr int kSmallTileRows = 16;  // query rows of one small tile (two 8-row MMA column blocks)
@@ -109,7 +110,8 @@ int launch_summaries_attn(const uint16_t* k_shared, float* summaries, float prob
 int launch_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, float* topk_score,
                  const moska_shape* s, void* ws, bool mark_groups, cudaStream_t st);
 int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
-                 const moska_shape* s, void* ws, bool premarked, cudaStream_t st);
+                 const moska_shape* s, void* ws, bool premarked, cudaStream_t st,
+                 bool grouping_regions_only = false);
 int launch_group_noalloc(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
                          const moska_shape* s, cudaStream_t st);
 int launch_shared_small(const uint16_t* q, const uint16_t* k_shared, const uint16_t* v_shared,

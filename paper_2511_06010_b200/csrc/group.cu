@@ -278,26 +278,29 @@ group_emit_kernel(const int32_t* __restrict__ topk_idx, const uint32_t* __restri
 
 }  // namespace
 
-int launch_ws_guards(void* ws, const WsLayout& lay, bool check, cudaStream_t st)
+int launch_ws_guards(void* ws, const WsLayout& lay, bool check, cudaStream_t st, size_t ws_extent)
 {
 #ifdef MOSKA_DEBUG_GUARDS
+    // only the regions that lie inside the buffer the caller really has: the built-in scratch of the
+    // allocation-free grouping ends where the grouping's regions end
     GuardRanges g;
     for (int r = 0; r < kWsRegions; ++r) {
-        g.begin[r] = lay.guard_begin[r];
-        g.end[r] = lay.guard_end[r];
+        const bool inside = lay.guard_end[r] <= ws_extent;
+        g.begin[r] = inside ? lay.guard_begin[r] : 0;
+        g.end[r] = inside ? lay.guard_end[r] : 0;
     }
     int* status = nullptr;
     MOSKA_TRY_STATUS(status_word(&status));
     ws_guard_kernel<<<kWsRegions, 256, 0, st>>>(static_cast<uint32_t*>(ws), g, check ? 1 : 0, status);
     MOSKA_LAUNCH_CHECK("ws_guard_kernel");
 #else
-    (void)ws; (void)lay; (void)check; (void)st;
+    (void)ws; (void)lay; (void)check; (void)st; (void)ws_extent;
 #endif
     return MOSKA_OK;
 }
 
 int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_entries,
-                 const moska_shape* s, void* ws, bool premarked, cudaStream_t st)
+                 const moska_shape* s, void* ws, bool premarked, cudaStream_t st, bool grouping_regions_only)
 {
     const WsLayout lay = ws_layout(s);
     char* base = static_cast<char*>(ws);
@@ -313,7 +316,7 @@ int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_ent
     // two calls run back to back inside moska_decode_step
     if (!premarked) {
         MOSKA_CUDA_TRY(cudaMemsetAsync(base, 0, lay.off_totals, st));
-        MOSKA_TRY_STATUS(launch_ws_guards(ws, lay, false, st));
+        MOSKA_TRY_STATUS(launch_ws_guards(ws, lay, false, st, grouping_regions_only ? lay.group_total : lay.total));
     }
     if (!premarked && P > 0) {
         group_mark_kernel<<<(unsigned)((P + 255) / 256), 256, 0, st>>>(topk_idx, bitmap, status, P,
@@ -334,7 +337,7 @@ int launch_group(const int32_t* topk_idx, int32_t* seg_offsets, int32_t* seg_ent
     group_emit_kernel<<<(lay.n_keys + 7) / 8, 256, 0, st>>>(topk_idx, bitmap, seg_offsets, seg_entries,
                                                             status, lay.n_keys, s->Hkv, s->C, s->k, lay.words);
     MOSKA_LAUNCH_CHECK("group_emit_kernel");
-    return launch_ws_guards(ws, lay, true, st);
+    return launch_ws_guards(ws, lay, true, st, grouping_regions_only ? lay.group_total : lay.total);
 }
 
 // ---- grouping without any caller- or library-side allocation -----------------------------------
@@ -376,7 +379,7 @@ int launch_group_noalloc(const int32_t* topk_idx, int32_t* seg_offsets, int32_t*
     }
     // launch_group clears the header and the bit sets itself, so the previous call's contents
     // never leak into this one.
-    return launch_group(topk_idx, seg_offsets, seg_entries, s, scratch, false, st);
+    return launch_group(topk_idx, seg_offsets, seg_entries, s, scratch, false, st, true);
 }
 
 }  // namespace moska

@@ -332,7 +332,7 @@ int launch_route(const uint16_t* q, const float* summaries, int32_t* topk_idx, f
     if (mark_groups) {
         const WsLayout lay = ws_layout(s);
         MOSKA_CUDA_TRY(cudaMemsetAsync(ws, 0, lay.off_totals, st));
-        MOSKA_TRY_STATUS(launch_ws_guards(ws, lay, false, st));
+        MOSKA_TRY_STATUS(launch_ws_guards(ws, lay, false, st, lay.total));
         mark = reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + lay.off_hist);
         mark_words = lay.words;
     }

@@ -54,4 +54,20 @@ for where in (n - 4, n - 256):          # last and first guard byte block of the
 layer.ws[n - 4] = 0
 layer.group()
 assert M.device_status() == 0
+# the allocation-free grouping under the debug build: its built-in buffer ends where the grouping's
+# regions end, so only their guard words exist; same segments as the call with a workspace
+w = W.scaled(W.CONFIGS[2], B=100, C=512, k=6, unique_len=16)
+sh = W.make_shared_store(w, "cuda")
+q = W.make_queries(w, sh, 0, "cuda")
+layer = MoskaLayer(w.B, w.Hq, w.Hkv, w.D, w.C, w.L, w.k, 16)
+layer.build_summaries(sh.k_shared)
+layer.route(q)
+layer.group()
+off = torch.full_like(layer.seg_offsets, -1)
+ent = torch.full_like(layer.seg_entries, -1)
+for _ in range(2):
+    M.group_by_chunk_noalloc(layer.topk_idx, off, ent, layer.shape)
+    torch.cuda.synchronize()
+    assert torch.equal(off, layer.seg_offsets) and torch.equal(ent, layer.seg_entries)
+    assert M.device_status() == 0
 print("debug build: guard words ok")
